@@ -1,0 +1,337 @@
+"""Pins for the oracle's code construction, encoder and decoder.
+
+What the paper fixes (Section 3): the code is an optimal prefix code built by recursive
+pair merging (so: a full binary tree, Kraft sum exactly 1, average length within one bit
+of the entropy, no cheaper prefix code exists), coding is lossless, and every segment
+decodes on its own from its known boundary."""
+import functools
+import heapq
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "huffman_tiebreak.txt")
+
+
+def _golden_cases():
+    out = []
+    with open(GOLDEN) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if not line:
+                continue
+            lhs, rhs = line.split("->")
+            out.append(([int(t) for t in lhs.split()], [int(t) for t in rhs.split()]))
+    return out
+
+
+def _cost(counts, lengths):
+    return sum(int(c) * int(l) for c, l in zip(counts, lengths))
+
+
+def _kraft_is_one(lengths):
+    used = [int(l) for l in lengths if l]
+    m = max(used)
+    return sum(1 << (m - l) for l in used) == (1 << m)
+
+
+# ----------------------------------------------------------------------------- lengths
+
+@pytest.mark.parametrize("counts,lengths", _golden_cases())
+def test_hand_worked_lengths(counts, lengths):
+    assert oracle.huffman_lengths(counts).tolist() == lengths
+
+
+@functools.lru_cache(maxsize=None)
+def _best_tree_cost(weights):
+    """Cheapest full binary tree over these leaf weights, trying EVERY pair at every
+    step (not just the two smallest): cost = sum of internal-node weights."""
+    if len(weights) == 1:
+        return 0
+    best = None
+    for i, j in itertools.combinations(range(len(weights)), 2):
+        merged = weights[i] + weights[j]
+        rest = tuple(sorted(w for k, w in enumerate(weights) if k != i and k != j) + [merged])
+        c = merged + _best_tree_cost(tuple(sorted(rest)))
+        best = c if best is None or c < best else best
+    return best
+
+
+def _best_kraft_cost(counts):
+    """Cheapest length vector with Kraft sum <= 1, by exhaustive enumeration."""
+    n = len(counts)
+    best = None
+    for ls in itertools.product(range(1, n), repeat=n):
+        if sum(2.0 ** -l for l in ls) <= 1.0:
+            c = _cost(counts, ls)
+            best = c if best is None or c < best else best
+    return best
+
+
+def test_optimal_against_brute_force_small_alphabets():
+    rng = np.random.default_rng(123)
+    for n in range(2, 9):
+        for trial in range(12):
+            hi = [3, 10, 1000][trial % 3]       # small ranges force many ties
+            counts = rng.integers(1, hi + 1, size=n).tolist()
+            ln = oracle.huffman_lengths(counts)
+            assert _kraft_is_one(ln)
+            assert _cost(counts, ln) == _best_tree_cost(tuple(sorted(counts))), counts
+            if n <= 6:
+                assert _cost(counts, ln) == _best_kraft_cost(counts), counts
+
+
+def _heap_huffman_cost(counts):
+    """A different construction (binary heap, arbitrary tie order): the cost is unique."""
+    h = [int(c) for c in counts if c]
+    heapq.heapify(h)
+    cost = 0
+    while len(h) > 1:
+        a, b = heapq.heappop(h), heapq.heappop(h)
+        cost += a + b
+        heapq.heappush(h, a + b)
+    return cost
+
+
+@pytest.mark.parametrize("nsym", [16, 256])
+def test_cost_kraft_and_entropy_bounds_on_weight_histograms(nsym):
+    bits = 4 if nsym == 16 else 8
+    for seed in range(4):
+        w = workloads.make_values(1 << 18, 0.02, seed).numpy()
+        q, _ = oracle.quantize_tensor(w, bits)
+        counts = oracle.histogram(q, nsym)
+        assert np.array_equal(counts, np.bincount(q, minlength=nsym).astype(np.uint64))
+        ln = oracle.huffman_lengths(counts)
+        assert np.all((ln > 0) == (counts > 0))
+        assert _kraft_is_one(ln)
+        assert _cost(counts, ln) == _heap_huffman_cost(counts)
+        p = counts[counts > 0].astype(np.float64) / counts.sum()
+        H = float(-(p * np.log2(p)).sum())
+        Lbar = _cost(counts, ln) / int(counts.sum())
+        assert H <= Lbar + 1e-12 < H + 1
+
+
+def test_random_histograms_cost_and_kraft():
+    rng = np.random.default_rng(5)
+    for trial in range(200):
+        n = int(rng.integers(2, 257))
+        counts = rng.integers(0, [2, 5, 1000, 10**9][trial % 4] + 1, size=n)
+        if np.count_nonzero(counts) < 2:
+            counts[:2] = 1
+        ln = oracle.huffman_lengths(counts)
+        assert _kraft_is_one(ln)
+        assert _cost(counts, ln) == _heap_huffman_cost(counts)
+        assert np.all((ln > 0) == (counts > 0))
+
+
+def test_textbook_length_patterns():
+    for k in range(1, 9):
+        assert oracle.huffman_lengths([7] * (1 << k)).tolist() == [k] * (1 << k)
+    # dyadic probabilities: length = -log2 p, average length equals the entropy
+    counts = [1 << 10, 1 << 9, 1 << 8, 1 << 7, 1 << 7]
+    ln = oracle.huffman_lengths(counts).tolist()
+    assert ln == [1, 2, 3, 4, 4]
+    total = sum(counts)
+    H = -sum(c / total * math.log2(c / total) for c in counts)
+    assert abs(_cost(counts, ln) / total - H) < 1e-12
+    # Fibonacci counts give the deepest possible tree: max length n - 1
+    fib = [1, 1]
+    while len(fib) < 30:
+        fib.append(fib[-1] + fib[-2])
+    ln = oracle.huffman_lengths(fib)
+    assert ln.max() == len(fib) - 1
+    fib40 = [1, 1]
+    while len(fib40) < 40:
+        fib40.append(fib40[-1] + fib40[-2])
+    with pytest.raises(oracle.OracleError) as e:          # depth 39 > 32: refused
+        oracle.huffman_lengths(fib40)
+    assert e.value.code == 4
+
+
+def test_minimum_variance_rule_gives_smallest_max_length():
+    """Leaf-before-internal on ties is the minimum-variance rule: among all optimal
+    codes it has the smallest maximum length.  Checked by enumeration."""
+    rng = np.random.default_rng(9)
+    for _ in range(40):
+        n = int(rng.integers(3, 7))
+        counts = rng.integers(1, 4, size=n).tolist()
+        ln = oracle.huffman_lengths(counts)
+        best_cost = _cost(counts, ln)
+        min_max = None
+        for ls in itertools.product(range(1, n), repeat=n):
+            if sum(2.0 ** -l for l in ls) <= 1.0 and _cost(counts, ls) == best_cost:
+                min_max = max(ls) if min_max is None else min(min_max, max(ls))
+        assert int(ln.max()) == min_max, counts
+
+
+# ----------------------------------------------------------------------------- canonical codes
+
+def _bitstr(code, length):
+    return format(int(code), "b").zfill(int(length)) if length else ""
+
+
+def test_canonical_codes_prefix_free_and_ordered():
+    rng = np.random.default_rng(1)
+    for trial in range(60):
+        n = int(rng.integers(2, 257))
+        counts = rng.integers(0, 50, size=n)
+        if np.count_nonzero(counts) < 2:
+            counts[:2] = 1
+        ln = oracle.huffman_lengths(counts)
+        cd = oracle.canonical_codes(ln)
+        words = {k: _bitstr(cd[k], ln[k]) for k in range(n) if ln[k]}
+        assert all(int(cd[k]) < (1 << int(ln[k])) for k in words)
+        ws = sorted(words.values())
+        assert len(set(ws)) == len(ws)
+        for a, b in zip(ws, ws[1:]):                 # sorted: a prefix would sit right before
+            assert not b.startswith(a)
+        # ordered by (length, symbol); numerically consecutive within a length
+        order = sorted(words, key=lambda k: (ln[k], k))
+        assert words[order[0]] == "0" * int(ln[order[0]])
+        for a, b in zip(order, order[1:]):
+            if ln[a] == ln[b]:
+                assert int(cd[b]) == int(cd[a]) + 1
+            else:
+                assert int(cd[b]) == (int(cd[a]) + 1) << (int(ln[b]) - int(ln[a]))
+        # left-justified codes increase strictly in that order, the last is all ones
+        lj = [int(cd[k]) << (32 - int(ln[k])) for k in order]
+        assert all(x < y for x, y in zip(lj, lj[1:]))
+        assert words[order[-1]] == "1" * int(ln[order[-1]])
+
+
+def test_canonical_codes_known_example():
+    # lengths 2 1 3 3: symbol 1 -> 0, symbol 0 -> 10, symbols 2, 3 -> 110, 111
+    assert oracle.canonical_codes([2, 1, 3, 3]).tolist() == [0b10, 0b0, 0b110, 0b111]
+    assert oracle.canonical_codes([0, 1, 0, 0]).tolist() == [0, 0, 0, 0]
+    with pytest.raises(oracle.OracleError):
+        oracle.canonical_codes([1, 1, 1])           # over-subscribed
+
+
+# ----------------------------------------------------------------------------- stream + index
+
+def _stream_bits(stream, nbits):
+    """Bit i of the stream = bit (31 - i % 32) of word i // 32, via NumPy unpackbits."""
+    by = np.ascontiguousarray(stream, dtype=">u4") if False else stream.astype(">u4")
+    return np.unpackbits(by.view(np.uint8))[:nbits]
+
+
+@pytest.mark.parametrize("bits,chunk", [(8, 4096), (4, 8192), (8, 64), (4, 32)])
+def test_stream_is_concatenation_of_codewords_and_index_is_consistent(bits, chunk):
+    n = 3 * chunk + chunk // 3 + 5
+    w = workloads.make_values(n, 0.02, 42 + bits).numpy()
+    c = oracle.compress(w, bits, chunk)
+    ln, cd, enc = c.lengths, c.codes, c.enc
+    text = "".join(_bitstr(cd[s], ln[s]) for s in c.q.tolist())
+    assert enc.total_bits == len(text) == int((c.counts * ln.astype(np.uint64)).sum())
+    got = "".join(map(str, _stream_bits(enc.stream, enc.total_bits).tolist()))
+    assert got == text
+    # zero padding after the last bit
+    assert not _stream_bits(enc.stream, enc.stream.size * 32)[enc.total_bits:].any()
+    # index: start of chunk k is the number of bits of the k * chunk symbols before it
+    per_sym = ln.astype(np.int64)[c.q]
+    cum = np.concatenate([[0], np.cumsum(per_sym)])
+    nch = oracle.num_chunks(n, chunk)
+    assert enc.offsets.size == nch + 1
+    for k in range(nch + 1):
+        assert int(enc.offsets[k]) == int(cum[min(k * chunk, n)])
+    sub = chunk // 32
+    for k in range(nch):
+        for j in range(32):
+            a, b = min(k * chunk + j * sub, n), min(k * chunk + (j + 1) * sub, n)
+            a, b = min(a, (k + 1) * chunk), min(b, (k + 1) * chunk)
+            assert int(enc.sub_len[k, j]) == int(cum[b] - cum[a])
+        assert int(enc.sub_len[k].sum()) == int(enc.offsets[k + 1] - enc.offsets[k])
+
+
+# ----------------------------------------------------------------------------- decoder
+
+def _dict_decode(bits_arr, start, count, table):
+    """Independent decoder: grow a bit string until it is a key of {codeword: symbol}."""
+    out, pos = [], start
+    for _ in range(count):
+        cur = ""
+        while cur not in table:
+            cur += str(int(bits_arr[pos]))
+            pos += 1
+            assert len(cur) <= 32
+        out.append(table[cur])
+    return out, pos
+
+
+@pytest.mark.parametrize("bits,chunk", [(8, 4096), (4, 8192), (8, 128)])
+def test_round_trip_and_segment_independence(bits, chunk):
+    for n in (1, 31, chunk - 1, chunk, chunk + 1, 5 * chunk + 77):
+        w = workloads.make_values(n, 0.03, n + bits).numpy()
+        c = oracle.compress(w, bits, chunk)
+        enc = c.enc
+        q, out = oracle.decode_dequant(enc.stream, enc.offsets, n, chunk, c.lengths, c.qp.scale,
+                                       c.qp.zero_point)
+        assert np.array_equal(q, c.q)                                    # lossless
+        assert np.array_equal(out, oracle.dequant(c.q, c.qp.scale, c.qp.zero_point))
+        # any subset of chunks, in any order, gives the same symbols there
+        nch = oracle.num_chunks(n, chunk)
+        ids = list(range(nch))[::-1][::2]
+        q2, _ = oracle.decode_dequant(enc.stream, enc.offsets, n, chunk, c.lengths, c.qp.scale,
+                                      c.qp.zero_point, chunk_ids=ids)
+        for k in ids:
+            assert np.array_equal(q2[k * chunk:(k + 1) * chunk], c.q[k * chunk:(k + 1) * chunk])
+        # thread-per-segment driver
+        _, out3 = oracle.decode_dequant(enc.stream, enc.offsets, n, chunk, c.lengths, c.qp.scale,
+                                        c.qp.zero_point, want_q=False, threads=3)
+        assert np.array_equal(out3, out)
+
+
+def test_decoder_against_dictionary_decoder():
+    n, chunk = 3000, 1024
+    w = workloads.make_values(n, 0.02, 77).numpy()
+    c = oracle.compress(w, 8, chunk)
+    table = {_bitstr(c.codes[s], c.lengths[s]): s for s in range(256) if c.lengths[s]}
+    bits_arr = _stream_bits(c.enc.stream, c.enc.total_bits)
+    for k in range(oracle.num_chunks(n, chunk)):
+        cnt = min(chunk, n - k * chunk)
+        syms, end = _dict_decode(bits_arr, int(c.enc.offsets[k]), cnt, table)
+        assert end == int(c.enc.offsets[k + 1])
+        assert syms == c.q[k * chunk:k * chunk + cnt].tolist()
+
+
+def test_decoder_rejects_corruption():
+    n, chunk = 20000, 4096
+    w = workloads.make_values(n, 0.02, 5).numpy()
+    c = oracle.compress(w, 8, chunk)
+    enc = c.enc
+    bad_off = enc.offsets.copy()
+    bad_off[2] += 3                                   # wrong boundary: chunk 1 ends elsewhere
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.decode_dequant(enc.stream, bad_off, n, chunk, c.lengths, c.qp.scale, c.qp.zero_point)
+    assert e.value.code == 5
+    # a single used symbol has code "0"; a 1 bit is not a codeword
+    ln = np.zeros(256, dtype=np.uint8)
+    ln[9] = 1
+    stream = np.array([0x80000000, 0], dtype=np.uint32)
+    with pytest.raises(oracle.OracleError):
+        oracle.decode_dequant(stream, np.array([0, 4], dtype=np.uint64), 4, 4096, ln, 1.0, 0)
+    q, _ = oracle.decode_dequant(np.zeros(2, dtype=np.uint32), np.array([0, 4], dtype=np.uint64), 4, 4096,
+                                 ln, 1.0, 0)
+    assert q.tolist() == [9, 9, 9, 9]
+
+
+def test_long_codes_round_trip():
+    """Fibonacci-like histogram: code lengths up to 30 bits survive encode -> decode."""
+    fib = [1, 1]
+    while len(fib) < 31:
+        fib.append(fib[-1] + fib[-2])
+    ln = oracle.huffman_lengths(fib + [0] * (256 - len(fib)))
+    assert ln.max() == 30
+    cd = oracle.canonical_codes(ln)
+    rng = np.random.default_rng(3)
+    q = np.concatenate([np.arange(31), rng.integers(0, 31, 5000), rng.integers(25, 31, 3000)]).astype(np.uint8)
+    rng.shuffle(q)
+    enc = oracle.encode(q, ln, cd, 4096)
+    q2, _ = oracle.decode_dequant(enc.stream, enc.offsets, q.size, 4096, ln, 1.0, 0)
+    assert np.array_equal(q2, q)

@@ -1,0 +1,196 @@
+"""Seeded synthetic inputs shared by the CPU oracle tests and the CUDA tests.
+
+This module holds tensor *shapes* and random *values* only.  It contains none
+of the method's arithmetic (no quantiser, no histogram, no code construction,
+no bit packing): both the oracle and the CUDA library receive the identical
+fp16 bytes produced here and do all of their own work on them.
+
+The value recipe stands in for trained checkpoints, which are not available:
+quantised LLM weights are bell-shaped with a dominant centre and long tails
+(Section 4, the weight-distribution figure), so each matrix is drawn from a
+Student-t distribution with nu = 5, scaled to a chosen standard deviation and
+rounded to fp16.  Norm-gain vectors (all positive) are included so that the
+unsigned branch of the mixed scheme (Eq. 1, left) and tensors shorter than one
+chunk are exercised as well.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+import zlib
+from typing import Iterator, List, Optional
+
+import numpy as np
+import torch
+
+NU = 5  # degrees of freedom of the Student-t draw
+
+
+@dataclasses.dataclass(frozen=True)
+class TensorSpec:
+    """One weight tensor of a synthetic model."""
+
+    name: str
+    rows: int          # out_features (or vocabulary size); 1 for vectors
+    cols: int          # in_features (or hidden size)
+    sigma: float       # target standard deviation (matrices) / gain spread (vectors)
+    seed: int
+    kind: str = "matrix"   # "matrix" (zero-mean Student-t) or "gain" (positive vector)
+
+    @property
+    def numel(self) -> int:
+        return self.rows * self.cols
+
+
+@dataclasses.dataclass(frozen=True)
+class Workload:
+    """A named list of tensors plus the symbol width and chunk size it is coded with."""
+
+    name: str
+    bits: int
+    chunk_symbols: int
+    tensors: tuple
+
+    @property
+    def numel(self) -> int:
+        return sum(t.numel for t in self.tensors)
+
+    def matrices(self) -> List[TensorSpec]:
+        return [t for t in self.tensors if t.kind == "matrix"]
+
+
+def _seed(config: str, layer: int, name: str) -> int:
+    return zlib.crc32(f"{config}/{layer}/{name}".encode()) & 0x7FFFFFFF
+
+
+def _model(config: str, config_id: int, n_layers: int, hidden: int, per_layer, extras,
+           with_gains: bool, max_layers: Optional[int]) -> List[TensorSpec]:
+    """per_layer / extras: lists of (name, rows, cols).  Sigma is drawn per layer
+    from U(0.01, 0.04) with a host generator seeded by the config id; embeddings
+    and heads take their own draw."""
+    rng = np.random.default_rng(config_id)
+    sig_layers = rng.uniform(0.01, 0.04, size=n_layers)
+    sig_extra = rng.uniform(0.01, 0.04, size=len(extras))
+    out: List[TensorSpec] = []
+    layers = n_layers if max_layers is None else min(n_layers, max_layers)
+    for (i, (name, r, c)) in enumerate(extras):
+        out.append(TensorSpec(name, r, c, float(sig_extra[i]), _seed(config, -1, name)))
+    for l in range(layers):
+        for (name, r, c) in per_layer:
+            out.append(TensorSpec(f"layers.{l}.{name}", r, c, float(sig_layers[l]),
+                                  _seed(config, l, name)))
+        if with_gains:
+            for name in ("input_norm", "post_attn_norm"):
+                out.append(TensorSpec(f"layers.{l}.{name}", 1, hidden, 0.1,
+                                      _seed(config, l, name), kind="gain"))
+    if with_gains:
+        out.append(TensorSpec("final_norm", 1, hidden, 0.1, _seed(config, n_layers, "final_norm"),
+                              kind="gain"))
+    return out
+
+
+def single_tensor(bits: int = 8, chunk_symbols: int = 4096) -> Workload:
+    """Config 1: one 1024 x 1024 tensor, sigma 0.02, seed 0."""
+    t = TensorSpec("w", 1024, 1024, 0.02, 0)
+    return Workload("single-1024x1024", bits, chunk_symbols, (t,))
+
+
+def smollm_1p7b(bits: int = 8, chunk_symbols: int = 4096, with_gains: bool = True,
+                max_layers: Optional[int] = None) -> Workload:
+    """Config 2: 24 layers, hidden 2048, MLP 8192, tied 49152 x 2048 embedding."""
+    h, m = 2048, 8192
+    per_layer = [("q_proj", h, h), ("k_proj", h, h), ("v_proj", h, h), ("o_proj", h, h),
+                 ("gate_proj", m, h), ("up_proj", m, h), ("down_proj", h, m)]
+    extras = [("embed_tokens", 49152, h)]
+    ts = _model("smollm", 2, 24, h, per_layer, extras, with_gains, max_layers)
+    return Workload("smolLM-1.7B-shaped", bits, chunk_symbols, tuple(ts))
+
+
+def phi3_mini_4k(bits: int = 4, chunk_symbols: int = 8192, with_gains: bool = True,
+                 max_layers: Optional[int] = None) -> Workload:
+    """Config 3: 32 layers, hidden 3072, fused qkv and gate_up, vocabulary 32064,
+    embedding and an untied head."""
+    h = 3072
+    per_layer = [("qkv_proj", 9216, h), ("o_proj", h, h), ("gate_up_proj", 16384, h),
+                 ("down_proj", h, 8192)]
+    extras = [("embed_tokens", 32064, h), ("lm_head", 32064, h)]
+    ts = _model("phi3", 3, 32, h, per_layer, extras, with_gains, max_layers)
+    return Workload("phi3-mini-4k-shaped", bits, chunk_symbols, tuple(ts))
+
+
+def mistral_7b(bits: int = 8, chunk_symbols: Optional[int] = None, with_gains: bool = True,
+               max_layers: Optional[int] = None) -> Workload:
+    """Config 4: 32 layers, hidden 4096, 8 kv heads of dim 128, MLP 14336,
+    vocabulary 32000, embedding and an untied head."""
+    h, kv, m = 4096, 1024, 14336
+    if chunk_symbols is None:
+        chunk_symbols = 4096 if bits == 8 else 8192
+    per_layer = [("q_proj", h, h), ("k_proj", kv, h), ("v_proj", kv, h), ("o_proj", h, h),
+                 ("gate_proj", m, h), ("up_proj", m, h), ("down_proj", h, m)]
+    extras = [("embed_tokens", 32000, h), ("lm_head", 32000, h)]
+    ts = _model("mistral", 4, 32, h, per_layer, extras, with_gains, max_layers)
+    return Workload(f"mistral-7B-shaped-uint{bits}", bits, chunk_symbols, tuple(ts))
+
+
+def mistral_layer_stack(max_layers: Optional[int] = None) -> Workload:
+    """Config 5: the seven projections of every mistral-shaped layer, 4-bit symbols,
+    stored [out_features, in_features] row-major for a batch-1 matrix-vector product."""
+    w = mistral_7b(bits=4, chunk_symbols=8192, with_gains=False, max_layers=max_layers)
+    ts = tuple(t for t in w.tensors if t.name.startswith("layers."))
+    return Workload("mistral-7B-shaped-uint4-gemv", 4, 8192, ts)
+
+
+def _generator(seed: int, device: torch.device) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    return g
+
+
+def make_values(numel: int, sigma: float, seed: int, kind: str = "matrix",
+                device: str | torch.device = "cpu", block: int = 1 << 24) -> torch.Tensor:
+    """fp16 values for one tensor, flat.  Matrices: Student-t(nu=5) as
+    N / sqrt(chi2_5 / 5), times sigma / sqrt(5/3) so the standard deviation is
+    sigma.  Gains: |1 + sigma * N(0,1)|.  Drawn block by block so the transient
+    fp32 footprint stays bounded for the largest tensors."""
+    device = torch.device(device)
+    g = _generator(seed, device)
+    out = torch.empty(numel, dtype=torch.float16, device=device)
+    scale = sigma / math.sqrt(NU / (NU - 2))
+    for lo in range(0, numel, block):
+        m = min(block, numel - lo)
+        z = torch.randn(m, generator=g, device=device, dtype=torch.float32)
+        if kind == "gain":
+            v = (1.0 + sigma * z).abs_()
+        else:
+            chi = torch.zeros(m, device=device, dtype=torch.float32)
+            for _ in range(NU):
+                e = torch.randn(m, generator=g, device=device, dtype=torch.float32)
+                chi.addcmul_(e, e)
+            v = z * torch.rsqrt(chi / NU) * scale
+        out[lo:lo + m] = v.to(torch.float16)
+    return out
+
+
+def make_tensor(spec: TensorSpec, device: str | torch.device = "cpu") -> torch.Tensor:
+    """The fp16 tensor a TensorSpec describes, shape [rows, cols] (row-major)."""
+    return make_values(spec.numel, spec.sigma, spec.seed, spec.kind, device).view(spec.rows,
+                                                                                  spec.cols)
+
+
+def make_vector(length: int, seed: int, device: str | torch.device = "cpu") -> torch.Tensor:
+    """Activation vector x ~ N(0, 1), rounded to fp16 (config 5)."""
+    device = torch.device(device)
+    g = _generator(seed, device)
+    return torch.randn(length, generator=g, device=device, dtype=torch.float32).to(torch.float16)
+
+
+def iter_tensors(w: Workload, device: str | torch.device = "cpu") -> Iterator:
+    for spec in w.tensors:
+        yield spec, make_tensor(spec, device)
+
+
+def tiny_cases() -> List[TensorSpec]:
+    """Small tensors whose sizes straddle chunk and sub-block boundaries."""
+    sizes = [1, 2, 31, 32, 33, 127, 128, 129, 4095, 4096, 4097, 8191, 8192, 8193,
+             3 * 4096 + 517, 5 * 8192 + 1]
+    return [TensorSpec(f"tiny{n}", 1, n, 0.02, 1000 + n) for n in sizes]
