@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: whole-model Huffman decode + dequantisation to fp16.
+
+A step is one pass of the whole path over one synthetic model: upload of the tensor
+descriptors, construction of the per-tensor decode tables, and the persistent decode +
+dequant kernel over every chunk of every tensor.  Default workload: mistral-7B-shaped
+weights at uint8 (7.24e9 weights, 226 + 65 tensors); `--also uint4` adds the 4-bit run.
+
+    python bench.py --gpus N --steps K --warmup W            # this library
+    python bench.py --impl reference --gpus N ...            # the CPU oracle, host cores
+
+One JSON line on stdout (rank 0).  Multi-GPU: every rank decodes its own full copy of the
+model (no data-path collective; weak scaling), launched by torch.distributed.run.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import workloads
+
+METRIC = "Huffman decode+dequant GB/s (compressed in + fp16 out)"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def pick_workload(name: str, max_layers):
+    if name == "mistral8":
+        return workloads.mistral_7b(bits=8, max_layers=max_layers)
+    if name == "mistral4":
+        return workloads.mistral_7b(bits=4, max_layers=max_layers)
+    if name == "smollm8":
+        return workloads.smollm_1p7b(max_layers=max_layers)
+    if name == "phi3_4":
+        return workloads.phi3_mini_4k(max_layers=max_layers)
+    if name == "single":
+        return workloads.single_tensor()
+    raise SystemExit(f"unknown workload {name}")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ----------------------------------------------------------------------------- this library
+
+class DeviceModel:
+    """A synthetic model compressed on the device with the library's own offline stages."""
+
+    def __init__(self, wl, E, lut_bytes: int):
+        self.wl = wl
+        self.keep = []           # device buffers
+        descs = []
+        total = sum((t.numel + 7) // 8 * 8 for t in wl.tensors)
+        self.out = torch.empty(total, dtype=torch.float16, device="cuda")
+        self.out_slices = []
+        self.n = 0
+        self.stream_bytes = 0    # ceil(total_bits / 8) per tensor
+        self.stream_buf_bytes = 0
+        self.index_bytes = 0
+        self.table_bytes = 0
+        self.max_len = 0
+        pos = 0
+        self.host_meta = []
+        for spec in wl.tensors:
+            w = workloads.make_tensor(spec, "cuda").view(-1)
+            q, qp = E.entro_quantize_tensor(w, wl.bits)
+            counts = E.entro_histogram(q, wl.bits)
+            cb = E.entro_build_codebook(counts.tolist())
+            enc = E.entro_encode(q, cb, wl.chunk_symbols, stream_words=E.entro_stream_words(counts.tolist(), cb))
+            del w, q
+            out = self.out[pos:pos + spec.numel]
+            pos += (spec.numel + 7) // 8 * 8
+            descs.append(E.make_desc(enc.stream, enc.index, spec.numel, wl.chunk_symbols, cb, qp.scale,
+                                     qp.zero_point, out))
+            self.keep.append(enc)
+            self.out_slices.append(out)
+            self.n += spec.numel
+            self.stream_bytes += (enc.total_bits + 7) // 8
+            self.stream_buf_bytes += enc.stream.numel() * 4
+            self.index_bytes += enc.index.numel()
+            self.table_bytes += lut_bytes
+            self.max_len = max(self.max_len, cb.max_len)
+        self.descs = E.desc_array(descs)
+        self.algorithmic_bytes = self.stream_bytes + self.index_bytes + self.table_bytes + 2 * self.n
+        self.bits_per_weight = 8.0 * self.stream_bytes / self.n
+
+
+def time_steps(E, model, steps, warmup, world, sampler_index):
+    import torch.distributed as dist
+    for _ in range(warmup):
+        E.entro_decode_dequant_batched(model.descs)
+    torch.cuda.synchronize()
+    assert E.entro_last_device_status() == E.OK
+    E.entro_profile_begin(steps)
+    launches0 = E.entro_kernel_launch_count()
+    sampler = ClockSampler(sampler_index)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev0.record()
+    for _ in range(steps):
+        E.entro_decode_dequant_batched(model.descs)
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    launches = E.entro_kernel_launch_count() - launches0
+    kernel_ms = E.entro_profile_read(steps)
+    E.entro_profile_begin(0)
+    assert E.entro_last_device_status() == E.OK
+    return ms, launches, kernel_ms, clocks
+
+
+def time_e2e(E, model, steps, warmup):
+    """Through the host-buffer entry point: H2D of stream + index, decode, D2H of the fp16 result."""
+    descs = model.descs
+    n_t = len(descs)
+    h_keep, io = [], (E.HostIO * n_t)()
+    h2d = d2h = 0
+    for i, enc in enumerate(model.keep):
+        hs = enc.stream.cpu().pin_memory()
+        hi = enc.index.cpu().pin_memory()
+        ho = torch.empty(model.out_slices[i].numel(), dtype=torch.float16).pin_memory()
+        h_keep += [hs, hi, ho]
+        io[i] = E.HostIO(hs.data_ptr(), hi.data_ptr(), ho.data_ptr())
+        h2d += hs.numel() * 4 + hi.numel()
+        d2h += ho.numel() * 2
+    for _ in range(warmup):
+        E.entro_decode_dequant_batched_host(descs, io)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(steps):
+        E.entro_decode_dequant_batched_host(descs, io)
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / steps
+    # spot check: the host result equals the device result of the device-resident run
+    k = min(3, n_t - 1)
+    assert torch.equal(h_keep[3 * k + 2], model.out_slices[k].cpu())
+    return ms, h2d, d2h
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_sample(wl, max_symbols):
+    """First matrices of the workload up to max_symbols, compressed BY THE ORACLE on the host."""
+    import oracle
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    items, total = [], 0
+    for spec in wl.matrices():
+        if not spec.name.startswith("layers."):
+            continue
+        if items and total + spec.numel > max_symbols:
+            break
+        w = workloads.make_tensor(spec, dev).view(-1).cpu().numpy()
+        c = oracle.compress(w, wl.bits, wl.chunk_symbols)
+        items.append((spec, c))
+        total += spec.numel
+    nbytes = 0
+    for spec, c in items:
+        nch = oracle.num_chunks(spec.numel, wl.chunk_symbols)
+        nbytes += (c.enc.total_bits + 7) // 8 + 8 * (nch + 1) + 64 * nch + 2 * spec.numel
+    return items, total, nbytes
+
+
+def oracle_pass(wl, items, threads):
+    import oracle
+    t0 = time.perf_counter()
+    for spec, c in items:
+        oracle.decode_dequant(c.enc.stream, c.enc.offsets, spec.numel, wl.chunk_symbols, c.lengths,
+                              c.qp.scale, c.qp.zero_point, want_q=False, threads=threads)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(wl, budget_cpu_s=12.0):
+    threads = os.cpu_count() or 1
+    items, nsym, nbytes = oracle_sample(wl, 120_000_000)
+    oracle_pass(wl, items[:1], threads)        # touch code and pages
+    passes, wall = 0, 0.0
+    while wall * threads < budget_cpu_s and wall < 60.0:
+        wall += oracle_pass(wl, items, threads)
+        passes += 1
+    names = ", ".join(s.name for s, _ in items)
+    return {"value": nbytes * passes / wall / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+            "weights_per_s": nsym * passes / wall,
+            "sample": f"{names} of {wl.name} ({nsym} weights), bit-serial decode + dequant, chunks dealt "
+                      f"round-robin to {threads} threads, {passes} passes in {wall:.2f} s"}
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the CPU oracle as it stands, on the host cores, rank 0 only."""
+    if rank != 0:
+        return
+    wl = pick_workload(args.workload, args.max_layers)
+    threads = os.cpu_count() or 1
+    items, nsym, nbytes = oracle_sample(wl, 45_000_000)
+    for _ in range(args.warmup):
+        oracle_pass(wl, items, threads)
+    t = 0.0
+    for _ in range(args.steps):
+        t += oracle_pass(wl, items, threads)
+    value = nbytes * args.steps / t / 1e9
+    names = ", ".join(s.name for s, _ in items)
+    sample = (f"each step: {names} of {wl.name} ({nsym} weights), bit-serial decode + dequant on "
+              f"{threads} host threads")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+        "config": {"workload": wl.name + " full-model decode (bounded sample per step)", "bits": wl.bits,
+                   "chunk_symbols": wl.chunk_symbols},
+        "weights_per_s": nsym * args.steps / t,
+        "cpu_baseline": {"value": value, "unit": "GB/s", "kind": "oracle", "cores": threads, "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ----------------------------------------------------------------------------- main
+
+def measure(E, wl, args, world, local_rank, rank, peak, with_e2e, with_cpu):
+    lut_bytes = (4 << args.lut_bits) + 1312 + 336
+    model = DeviceModel(wl, E, lut_bytes)
+    ms, launches, kernel_ms, clocks = time_steps(E, model, args.steps, args.warmup, world,
+                                                 physical_gpu_index(local_rank))
+    ms_step = ms / args.steps
+    value = world * model.algorithmic_bytes / (ms_step * 1e-3) / 1e9
+    k_ms = float(np.mean(kernel_ms)) if kernel_ms else ms_step
+    achieved = model.algorithmic_bytes / (k_ms * 1e-3) / 1e9
+    res = {
+        "value": value, "ms_per_step": ms_step, "weights_per_s": world * model.n / (ms_step * 1e-3),
+        "bytes_per_step": model.algorithmic_bytes, "bits_per_weight": model.bits_per_weight,
+        "max_code_len": model.max_len, "gpu_launches": int(launches), "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak[0],
+                     "unit": "GB/s", "frac": achieved / peak[0], "peak_source": peak[1],
+                     "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS, "kernel_ms": k_ms,
+                     "kernel_ms_min": float(np.min(kernel_ms)) if kernel_ms else None, "traffic": None},
+        "model": model,
+    }
+    if with_e2e and rank == 0 or (with_e2e and world > 1):
+        e_ms, h2d, d2h = time_e2e(E, model, max(1, min(args.e2e_steps, args.steps)), 1)
+        res["e2e"] = {"value": world * model.algorithmic_bytes / (e_ms * 1e-3) / 1e9, "unit": "GB/s",
+                      "ms_per_step": e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    if with_cpu and rank == 0 and world == 1:
+        res["cpu_baseline"] = cpu_baseline(wl)
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="own", choices=["own", "reference"])
+    ap.add_argument("--workload", default="mistral8",
+                    choices=["mistral8", "mistral4", "smollm8", "phi3_4", "single"])
+    ap.add_argument("--also", default="mistral4", help="second workload reported under 'also' ('' = none)")
+    ap.add_argument("--max-layers", type=int, default=None, help="truncate the model (for profiling runs)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--lut-bits", type=int, default=0)
+    ap.add_argument("--warps", type=int, default=0)
+    ap.add_argument("--ctas", type=int, default=0)
+    ap.add_argument("--item", type=int, default=0)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import paper_2505_02380_b200 as E   # fails loudly if the CUDA library is not built
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    E.lib()
+    if args.lut_bits or args.warps or args.ctas or args.item:
+        E.entro_set_decode_config(args.lut_bits, args.warps, args.ctas, args.item)
+    if not args.lut_bits:
+        args.lut_bits = 11
+    peak = measured_peak()
+
+    wl = pick_workload(args.workload, args.max_layers)
+    main_res = measure(E, wl, args, world, local_rank, rank, peak, not args.no_e2e, not args.no_cpu)
+    main_res.pop("model")
+    also = None
+    if args.also and args.also != args.workload:
+        torch.cuda.empty_cache()
+        wl2 = pick_workload(args.also, args.max_layers)
+        r2 = measure(E, wl2, args, world, local_rank, rank, peak, False, False)
+        r2.pop("model")
+        also = {"workload": wl2.name + " full-model decode", "bits": wl2.bits, "chunk_symbols": wl2.chunk_symbols,
+                **{k: r2[k] for k in ("value", "ms_per_step", "weights_per_s", "bytes_per_step", "bits_per_weight",
+                                       "max_code_len", "roofline", "clocks")}}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": main_res["value"], "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": main_res["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+            "config": {"workload": wl.name + " full-model decode", "bits": wl.bits,
+                       "chunk_symbols": wl.chunk_symbols, "tensors": len(wl.tensors), "weights": wl.numel,
+                       "max_layers": args.max_layers, "lut_bits": args.lut_bits,
+                       "l2": "inputs and outputs per step (GBs) are far larger than L2; no flush needed",
+                       "parallelism": f"replicas x{world}, one full model per GPU, no collective"},
+            "weights_per_s": main_res["weights_per_s"], "bytes_per_step": main_res["bytes_per_step"],
+            "bits_per_weight": main_res["bits_per_weight"], "max_code_len": main_res["max_code_len"],
+            "pct_of_nominal_8000_GBs": 100.0 * main_res["value"] / world / NOMINAL_HBM_GBS,
+            "pct_of_measured_copy": 100.0 * main_res["value"] / world / peak[0],
+            "roofline": main_res["roofline"], "clocks": main_res["clocks"],
+            "gpu_launches": main_res["gpu_launches"],
+        }
+        if "e2e" in main_res:
+            line["e2e"] = main_res["e2e"]
+        if "cpu_baseline" in main_res:
+            line["cpu_baseline"] = main_res["cpu_baseline"]
+        if also:
+            line["also"] = also
+        line["paper_context"] = ("paper: 6.66 s (uint8) / 1.66 s (uint4) to decode phi3-mini-4k on a Jetson P3450, "
+                                 "4 CPU threads, integer output (Table 3) -- other hardware, context only")
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

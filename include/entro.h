@@ -1,0 +1,231 @@
+/*
+ * entro.h -- C ABI of the B200 (sm_100a) library for EntroLLM's weight path:
+ * per-tensor quantisation, symbol histogram, canonical Huffman codebook, encoding into a
+ * bitstream with a per-chunk bit-offset index, and parallel decoding fused with
+ * dequantisation to fp16.
+ *
+ * General rules
+ *  - Pointers named *_dev are CUDA device pointers on the current device; pointers named
+ *    *_host are host pointers.  The caller owns and allocates every buffer it passes.
+ *    The library keeps a small per-device workspace of its own (decode tables, work
+ *    descriptors, a status word), allocated on first use and grown on demand.
+ *  - cuda_stream is a cudaStream_t passed as void* (NULL = the default stream).
+ *  - Every call returns an entro_status.  Nothing throws, aborts or traps.  Argument
+ *    errors are found before any kernel is launched.
+ *  - Calls that return data to the host (qp_host, counts_host, total_bits_host)
+ *    synchronise cuda_stream before returning.  Decode calls are asynchronous.
+ *  - Symbols are one per byte (values 0 .. 2^bits - 1), bits is 4 or 8.
+ *  - Calls on one device share the workspace: issue them on one stream, or order them
+ *    with events, so that no two of them overlap on the GPU.  Host-side entry is
+ *    serialised by an internal lock.
+ *
+ * Compressed format (fixed here; the paper leaves it open)
+ *  - Stream: 32-bit words; stream bit i is bit (31 - i % 32) of word i / 32; codewords are
+ *    concatenated MSB-first in row-major element order; unused bits are zero.  A stream
+ *    buffer holds ceil(total_bits / 32) + ENTRO_STREAM_SLACK_WORDS words, the slack zero,
+ *    and starts on a 16-byte boundary.
+ *  - Segments: the paper decodes independent segments with known boundaries in parallel
+ *    (Section 3, "Segmentation for parallel Huffman decoding"; Fig. 3).  Here a segment is
+ *    a chunk of chunk_symbols consecutive symbols of one tensor (the last chunk may be
+ *    short).  The index of a tensor with n_chunks = ceil(n / chunk_symbols) chunks is
+ *        uint64_t offsets[n_chunks + 1];      bit position where each chunk starts,
+ *                                             offsets[n_chunks] = total bits
+ *        uint16_t sub_len[n_chunks][32];      each chunk is cut into 32 sub-blocks of
+ *                                             chunk_symbols / 32 symbols; bit length of each
+ *    stored back to back (entro_index_bytes bytes), 8-byte aligned.
+ *  - chunk_symbols is a multiple of 32, at least 32 and at most 16384.
+ */
+#ifndef ENTRO_H
+#define ENTRO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ENTRO_MAX_SYMBOLS 256
+#define ENTRO_MAX_CODE_LEN 32
+#define ENTRO_SUB_BLOCKS 32
+#define ENTRO_STREAM_SLACK_WORDS 8
+#define ENTRO_MAX_CHUNK_SYMBOLS 16384
+
+typedef enum {
+    ENTRO_OK = 0,
+    ENTRO_ERR_INVALID_ARG = 1,
+    ENTRO_ERR_BUFFER_TOO_SMALL = 2,
+    ENTRO_ERR_NONFINITE = 3,       /* the tensor holds a NaN or an infinity */
+    ENTRO_ERR_CODE_TOO_LONG = 4,   /* an optimal code length exceeds 32 bits */
+    ENTRO_ERR_CORRUPT_STREAM = 5,  /* stream, index and codebook do not agree */
+    ENTRO_ERR_CUDA = 6,            /* a CUDA runtime call failed */
+    ENTRO_ERR_UNSUPPORTED = 7
+} entro_status;
+
+/* The paper applies "either unsigned or asymmetric quantization per layer, based on its
+ * weight distribution" (Section 3, Eq. 1).  AUTO: unsigned iff every weight is >= 0. */
+typedef enum { ENTRO_MODE_AUTO = 0, ENTRO_MODE_UNSIGNED = 1, ENTRO_MODE_ASYMMETRIC = 2 } entro_mode;
+
+typedef struct {
+    int32_t bits;        /* 4 or 8 */
+    int32_t mode;        /* resolved: ENTRO_MODE_UNSIGNED or ENTRO_MODE_ASYMMETRIC */
+    float scale;         /* s */
+    int32_t zero_point;  /* z, an integer in [0, 2^bits - 1]; 0 in unsigned mode */
+    float lo, hi;        /* tensor minimum and maximum */
+} entro_qparams;
+
+typedef struct {
+    int32_t nsym;                       /* alphabet size, 1 .. 256 */
+    int32_t max_len;                    /* longest code length in use */
+    uint8_t len[ENTRO_MAX_SYMBOLS];     /* code length per symbol, 0 = symbol unused */
+    uint32_t code[ENTRO_MAX_SYMBOLS];   /* canonical code, right-aligned in len bits */
+} entro_codebook;
+
+/* One compressed tensor for the batched decode.  Host struct; the pointers inside are
+ * device pointers. */
+typedef struct {
+    const uint32_t *stream_dev;   /* 16-byte aligned */
+    uint64_t stream_words;        /* words in the buffer, slack included */
+    const void *index_dev;        /* 8-byte aligned, entro_index_bytes(n, chunk_symbols) bytes */
+    uint64_t n;                   /* symbols (= weights) in the tensor */
+    uint32_t chunk_symbols;
+    float scale;
+    int32_t zero_point;
+    entro_codebook cb;            /* only nsym and len[] are read by the decoder */
+    void *out_fp16_dev;           /* n fp16 values, 16-byte aligned */
+} entro_tensor_desc;
+
+/*
+ * Quantise one tensor (Section 3, "Mixed Quantization Scheme", Eq. 1).
+ *   lo, hi = min, max of the weights.  qmax = 2^bits - 1.
+ *   unsigned:   s = hi / qmax, z = 0.
+ *   asymmetric: s = (hi - lo) / qmax, z = clamp(rne(-lo / s), 0, qmax).
+ *   q = clamp(rne(w / s) + z, 0, qmax), so that w_hat = s * (q - z).
+ * All arithmetic is IEEE fp32 with true division; rne is round-half-to-even.  If the
+ * computed s is not positive (constant tensor), s = 1.
+ * w_fp16_dev: n fp16 weights (device, 16-byte aligned).  q_dev: n bytes (device, 16-byte
+ * aligned), one symbol per byte.  qp_host: filled on return.  Synchronises.
+ * ENTRO_ERR_NONFINITE if a weight is NaN or infinite (q_dev is then not written).
+ */
+entro_status entro_quantize_tensor(const void *w_fp16_dev, uint64_t n, int bits, entro_mode mode,
+                                   uint8_t *q_dev, entro_qparams *qp_host, void *cuda_stream);
+
+/*
+ * Symbol frequencies, the "score" each symbol gets in Section 3 ("Huffman weight
+ * encoding").  counts_host[k] = number of symbols equal to k, k < 2^bits.  Synchronises.
+ * ENTRO_ERR_INVALID_ARG if a symbol is >= 2^bits.
+ */
+entro_status entro_histogram(const uint8_t *q_dev, uint64_t n, int bits, uint64_t *counts_host,
+                             void *cuda_stream);
+
+/*
+ * Huffman code lengths by recursive merging of the two least frequent nodes (Section 3,
+ * "Huffman weight encoding"), then canonical codes.  Pure host code.
+ * Ties: on equal weight a leaf is taken before an internal node, leaves by ascending
+ * symbol, internal nodes by creation order.  Symbols with count 0 get length 0; a single
+ * used symbol gets length 1, code 0.  Canonical codes: symbols ordered by (length,
+ * symbol), the first code is 0, each next code is (previous + 1) << (growth in length).
+ * ENTRO_ERR_CODE_TOO_LONG if a length exceeds 32; ENTRO_ERR_INVALID_ARG if all counts
+ * are zero or nsym is outside 1 .. 256.
+ */
+entro_status entro_build_codebook(const uint64_t *counts_host, int nsym, entro_codebook *cb_host);
+
+/* Words a stream buffer needs for these counts under this codebook: ceil(sum count[k] *
+ * len[k] / 32) + ENTRO_STREAM_SLACK_WORDS.  0 on a bad argument. */
+uint64_t entro_stream_words(const uint64_t *counts_host, const entro_codebook *cb_host);
+
+/* Upper bound of the same without a histogram: n symbols of max_len bits each. */
+uint64_t entro_encode_bound_words(uint64_t n, const entro_codebook *cb_host);
+
+/* Bytes of the index of an n-symbol tensor: 8 * (n_chunks + 1) + 64 * n_chunks. */
+uint64_t entro_index_bytes(uint64_t n, uint32_t chunk_symbols);
+
+/*
+ * Encode symbols into the compressed format described at the top (Section 3: variable
+ * length codes, segments with known boundaries).  stream_dev (16-byte aligned,
+ * stream_cap_words words) is zeroed and filled; index_dev (8-byte aligned) receives the
+ * offsets and sub-block lengths; *total_bits_host the stream length in bits.  Synchronises.
+ * ENTRO_ERR_BUFFER_TOO_SMALL if the stream needs more than stream_cap_words -
+ * ENTRO_STREAM_SLACK_WORDS words or the index more than index_cap_bytes;
+ * ENTRO_ERR_INVALID_ARG if a symbol has no code.
+ */
+entro_status entro_encode(const uint8_t *q_dev, uint64_t n, const entro_codebook *cb_host,
+                          uint32_t chunk_symbols, uint32_t *stream_dev, uint64_t stream_cap_words,
+                          void *index_dev, uint64_t index_cap_bytes, uint64_t *total_bits_host,
+                          void *cuda_stream);
+
+/*
+ * Parallel decode fused with dequantisation (Section 3, "Segmentation for parallel
+ * Huffman decoding": every segment decodes independently from its known boundary; Eq. 1
+ * inverted): out[i] = fp16_rne( s *_fp32 (float)(q[i] - z) ), q the decoded symbols in
+ * element order.  Asynchronous on cuda_stream.  Malformed input (index not matching the
+ * stream, a bit pattern that is no codeword) never faults: the affected chunk's output is
+ * unspecified but in bounds, and the error is reported by entro_last_device_status.
+ * n = 0: ENTRO_OK, nothing written.
+ */
+entro_status entro_decode_dequant(const uint32_t *stream_dev, uint64_t stream_words,
+                                  const void *index_dev, uint64_t n, uint32_t chunk_symbols,
+                                  const entro_codebook *cb_host, float scale, int32_t zero_point,
+                                  void *out_fp16_dev, void *cuda_stream);
+
+/*
+ * The same for a whole model in one pass: all tensors' chunks form one work list that a
+ * persistent kernel consumes (the paper balances load by dealing many segments to each
+ * thread, Section 3).  descs_host is read before the call returns.  Asynchronous.
+ */
+entro_status entro_decode_dequant_batched(const entro_tensor_desc *descs_host, int ntensors,
+                                          void *cuda_stream);
+
+/* Host-resident input and output for one tensor of entro_decode_dequant_batched_host. */
+typedef struct {
+    const uint32_t *stream_host;  /* stream_words words (pinned memory for full speed) */
+    const void *index_host;       /* entro_index_bytes bytes */
+    void *out_fp16_host;          /* n fp16 values */
+} entro_host_io;
+
+/*
+ * End-to-end form with host buffers: for every tensor, copy stream and index from
+ * io_host[i] to the device buffers named in descs_host[i], decode + dequantise, and copy
+ * the fp16 result back to io_host[i].out_fp16_host.  Copies and kernels are issued on
+ * cuda_stream; returns after everything has completed (synchronises).
+ */
+entro_status entro_decode_dequant_batched_host(const entro_tensor_desc *descs_host,
+                                               const entro_host_io *io_host, int ntensors,
+                                               void *cuda_stream);
+
+/*
+ * Synchronise cuda_stream, then report and clear what decode kernels found since the last
+ * call: ENTRO_OK or ENTRO_ERR_CORRUPT_STREAM (ENTRO_ERR_CUDA if the stream itself failed).
+ */
+entro_status entro_last_device_status(void *cuda_stream);
+
+/*
+ * Launch shape of the decode kernel; every argument may be 0 to keep its current value.
+ *   lut_bits: bits looked up at once in the shared-memory table (10 .. 12)
+ *   warps_per_cta: 4 .. 32;  ctas_per_sm: 1 .. 8;  chunks_per_item: chunks a CTA claims at once
+ * ENTRO_ERR_INVALID_ARG (nothing changed) if a value is out of range or the shape does
+ * not fit in shared memory.
+ */
+entro_status entro_set_decode_config(int lut_bits, int warps_per_cta, int ctas_per_sm,
+                                     int chunks_per_item);
+
+/*
+ * Optional timing of the decode kernel alone (CUDA events recorded on the caller's stream
+ * right before and after its launch).  entro_profile_begin(max_records) arms up to
+ * max_records recordings on the current device (0 disarms); every batched decode then
+ * fills the next record.  entro_profile_read waits for the recorded launches, writes their
+ * durations in milliseconds to ms_host (at most cap), re-arms, and returns how many it
+ * wrote (-1 on error).
+ */
+entro_status entro_profile_begin(int max_records);
+int entro_profile_read(float *ms_host, int cap);
+
+/* Kernels launched by this library on the calling thread's device since load (for
+ * launch accounting in benchmarks). */
+uint64_t entro_kernel_launch_count(void);
+
+const char *entro_status_string(entro_status st);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ENTRO_H */

@@ -1,0 +1,216 @@
+// entro_encode: symbols -> bitstream + per-chunk bit-offset index (Section 3: variable
+// length codes; segments with known boundaries).  Three passes: bit lengths of every
+// sub-block, a prefix sum over chunks, then each sub-block packs its own bits.
+#include "entro_internal.h"
+
+namespace entro {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+
+struct Code {
+    uint32_t code[ENTRO_MAX_SYMBOLS];
+    uint8_t len[ENTRO_MAX_SYMBOLS];
+};
+
+// Pass 1: one warp per chunk, one lane per sub-block.
+__global__ void __launch_bounds__(kThreads) sub_lengths_kernel(const uint8_t* __restrict__ q, uint64_t n,
+                                                               uint32_t chunk_symbols, uint32_t n_chunks,
+                                                               const Code* __restrict__ cb,
+                                                               uint16_t* __restrict__ sub_len,
+                                                               unsigned long long* __restrict__ chunk_bits,
+                                                               uint32_t* __restrict__ bad_symbol)
+{
+    __shared__ uint8_t s_len[ENTRO_MAX_SYMBOLS];
+    for (int i = threadIdx.x; i < ENTRO_MAX_SYMBOLS; i += kThreads) s_len[i] = cb->len[i];
+    __syncthreads();
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t sub = chunk_symbols / kSubBlocks;
+    for (uint32_t c = blockIdx.x * kWarps + (threadIdx.x >> 5); c < n_chunks; c += gridDim.x * kWarps) {
+        uint64_t first = (uint64_t)c * chunk_symbols + (uint64_t)lane * sub;
+        uint64_t chunk_end = min((uint64_t)(c + 1) * chunk_symbols, n);
+        uint64_t last = min(first + sub, chunk_end);
+        uint32_t bits = 0, bad = 0;
+        for (uint64_t i = first; i < last; ++i) {
+            uint32_t l = s_len[q[i]];
+            bad |= (l == 0);
+            bits += l;
+        }
+        if (bad) atomicOr(bad_symbol, 1u);
+        sub_len[(uint64_t)c * kSubBlocks + lane] = (uint16_t)bits;
+        uint32_t total = bits;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) total += __shfl_xor_sync(0xffffffffu, total, d);
+        if (lane == 0) chunk_bits[c] = total;
+    }
+}
+
+// Pass 2: exclusive prefix sum of the chunk lengths by one block; offsets[n_chunks] = total.
+__global__ void __launch_bounds__(1024) chunk_offsets_kernel(const unsigned long long* __restrict__ chunk_bits,
+                                                             uint32_t n_chunks,
+                                                             unsigned long long* __restrict__ offsets)
+{
+    __shared__ unsigned long long warp_sum[32];
+    __shared__ unsigned long long carry;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint32_t base = 0; base < n_chunks; base += 1024) {
+        uint32_t i = base + threadIdx.x;
+        unsigned long long v = i < n_chunks ? chunk_bits[i] : 0ull;
+        unsigned long long incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            unsigned long long t = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= (uint32_t)d) incl += t;
+        }
+        if (lane == 31) warp_sum[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long w = warp_sum[lane];
+            unsigned long long wi = w;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                unsigned long long t = __shfl_up_sync(0xffffffffu, wi, d);
+                if (lane >= (uint32_t)d) wi += t;
+            }
+            warp_sum[lane] = wi - w;  // exclusive
+        }
+        __syncthreads();
+        unsigned long long excl = carry + warp_sum[warp] + incl - v;
+        if (i < n_chunks) offsets[i] = excl;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry = excl + v;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) offsets[n_chunks] = carry;
+}
+
+// Pass 3: one warp per chunk; every lane writes the bits of its own sub-block.  Words that
+// a sub-block shares with a neighbour are merged with atomicOr into the zeroed stream.
+__global__ void __launch_bounds__(kThreads) pack_kernel(const uint8_t* __restrict__ q, uint64_t n,
+                                                        uint32_t chunk_symbols, uint32_t n_chunks,
+                                                        const Code* __restrict__ cb,
+                                                        const unsigned long long* __restrict__ offsets,
+                                                        const uint16_t* __restrict__ sub_len,
+                                                        uint32_t* __restrict__ stream)
+{
+    __shared__ uint32_t s_code[ENTRO_MAX_SYMBOLS];
+    __shared__ uint8_t s_len[ENTRO_MAX_SYMBOLS];
+    for (int i = threadIdx.x; i < ENTRO_MAX_SYMBOLS; i += kThreads) {
+        s_code[i] = cb->code[i];
+        s_len[i] = cb->len[i];
+    }
+    __syncthreads();
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t sub = chunk_symbols / kSubBlocks;
+    for (uint32_t c = blockIdx.x * kWarps + (threadIdx.x >> 5); c < n_chunks; c += gridDim.x * kWarps) {
+        uint32_t mine = sub_len[(uint64_t)c * kSubBlocks + lane];
+        uint32_t incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= (uint32_t)d) incl += t;
+        }
+        unsigned long long pos = offsets[c] + (incl - mine);   // first bit of this sub-block
+        uint64_t first = (uint64_t)c * chunk_symbols + (uint64_t)lane * sub;
+        uint64_t chunk_end = min((uint64_t)(c + 1) * chunk_symbols, n);
+        uint64_t last = min(first + sub, chunk_end);
+        if (first >= last) continue;
+
+        // acc holds `fill` pending bits, left-justified; word is where they go next.
+        unsigned long long word = pos >> 5;
+        uint32_t fill = (uint32_t)(pos & 31);   // bits of `word` that belong to earlier sub-blocks
+        unsigned long long acc = 0;             // bits [63 - fill ...] downwards are ours
+        bool first_word = true;
+        for (uint64_t i = first; i < last; ++i) {
+            uint32_t sym = q[i];
+            uint32_t l = s_len[sym];
+            if (l == 0) continue;               // reported by pass 1
+            acc |= (unsigned long long)s_code[sym] << (64 - fill - l);
+            fill += l;
+            if (fill >= 32) {
+                uint32_t out = (uint32_t)(acc >> 32);
+                if (first_word) atomicOr(&stream[word], out);
+                else stream[word] = out;
+                first_word = false;
+                ++word;
+                acc <<= 32;
+                fill -= 32;
+            }
+        }
+        if (fill) atomicOr(&stream[word], (uint32_t)(acc >> 32));
+    }
+}
+
+}  // namespace
+}  // namespace entro
+
+using namespace entro;
+
+extern "C" entro_status entro_encode(const uint8_t* q_dev, uint64_t n, const entro_codebook* cb,
+                                     uint32_t chunk_symbols, uint32_t* stream_dev, uint64_t stream_cap_words,
+                                     void* index_dev, uint64_t index_cap_bytes, uint64_t* total_bits_host,
+                                     void* cuda_stream)
+{
+    if (!q_dev || !cb || !stream_dev || !index_dev || !total_bits_host || n == 0) return ENTRO_ERR_INVALID_ARG;
+    if (chunk_symbols < kSubBlocks || chunk_symbols % kSubBlocks || chunk_symbols > ENTRO_MAX_CHUNK_SYMBOLS)
+        return ENTRO_ERR_INVALID_ARG;
+    if (!aligned(stream_dev, 16) || !aligned(index_dev, 8)) return ENTRO_ERR_INVALID_ARG;
+    if (!codebook_lengths_valid(cb)) return ENTRO_ERR_INVALID_ARG;
+    const uint64_t nc64 = num_chunks(n, chunk_symbols);
+    if (nc64 > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
+    const uint32_t nc = (uint32_t)nc64;
+    if (entro_index_bytes(n, chunk_symbols) > index_cap_bytes) return ENTRO_ERR_BUFFER_TOO_SMALL;
+    if (stream_cap_words <= ENTRO_STREAM_SLACK_WORDS) return ENTRO_ERR_BUFFER_TOO_SMALL;
+
+    Guard g;
+    Workspace* ws = workspace();
+    if (!ws) return ENTRO_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+
+    // workspace: [Code][chunk_bits: nc u64][flag]
+    const size_t code_bytes = (sizeof(Code) + 15) & ~(size_t)15;
+    const size_t need = code_bytes + (size_t)nc * 8 + 16;
+    if (!reserve_device(ws, need) || !reserve_pinned(ws, code_bytes + 16)) return ENTRO_ERR_CUDA;
+    Code* host_code = static_cast<Code*>(ws->pinned);
+    for (int k = 0; k < ENTRO_MAX_SYMBOLS; ++k) {
+        host_code->code[k] = k < cb->nsym ? cb->code[k] : 0;
+        host_code->len[k] = k < cb->nsym ? cb->len[k] : 0;
+    }
+    char* base = static_cast<char*>(ws->dev);
+    Code* dev_code = reinterpret_cast<Code*>(base);
+    unsigned long long* chunk_bits = reinterpret_cast<unsigned long long*>(base + code_bytes);
+    uint32_t* flag = reinterpret_cast<uint32_t*>(base + code_bytes + (size_t)nc * 8);
+    unsigned long long* offsets = static_cast<unsigned long long*>(index_dev);
+    uint16_t* sub_len = reinterpret_cast<uint16_t*>(offsets + nc + 1);
+
+    ENTRO_CUDA(cudaMemcpyAsync(dev_code, host_code, sizeof(Code), cudaMemcpyHostToDevice, s));
+    mark_pinned_in_use(ws, s);
+    ENTRO_CUDA(cudaMemsetAsync(flag, 0, 16, s));
+    int grid = (int)((nc + kWarps - 1) / kWarps);
+    int cap = ws->sm_count * 8;
+    if (grid > cap) grid = cap;
+    sub_lengths_kernel<<<grid, kThreads, 0, s>>>(q_dev, n, chunk_symbols, nc, dev_code, sub_len, chunk_bits, flag);
+    chunk_offsets_kernel<<<1, 1024, 0, s>>>(chunk_bits, nc, offsets);
+    count_launch(2);
+    ENTRO_CUDA(cudaGetLastError());
+
+    // total bits and the bad-symbol flag decide whether the pack pass may run
+    struct { unsigned long long total; uint32_t bad; uint32_t pad; } h;
+    ENTRO_CUDA(cudaMemcpyAsync(&h.total, offsets + nc, 8, cudaMemcpyDeviceToHost, s));
+    ENTRO_CUDA(cudaMemcpyAsync(&h.bad, flag, 4, cudaMemcpyDeviceToHost, s));
+    ENTRO_CUDA(cudaStreamSynchronize(s));
+    if (h.bad) return ENTRO_ERR_INVALID_ARG;
+    const uint64_t words = (h.total + 31) / 32;
+    if (words + ENTRO_STREAM_SLACK_WORDS > stream_cap_words) return ENTRO_ERR_BUFFER_TOO_SMALL;
+
+    ENTRO_CUDA(cudaMemsetAsync(stream_dev, 0, stream_cap_words * sizeof(uint32_t), s));
+    pack_kernel<<<grid, kThreads, 0, s>>>(q_dev, n, chunk_symbols, nc, dev_code, offsets, sub_len, stream_dev);
+    count_launch();
+    ENTRO_CUDA(cudaGetLastError());
+    ENTRO_CUDA(cudaStreamSynchronize(s));
+    *total_bits_host = h.total;
+    return ENTRO_OK;
+}

@@ -1,0 +1,105 @@
+// Internal declarations shared by the library's translation units (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "entro.h"
+
+namespace entro {
+
+constexpr int kSubBlocks = ENTRO_SUB_BLOCKS;
+constexpr int kMaxLutBits = 12;
+constexpr uint32_t kEscFlag = 0x8000u;        // LUT entry: code longer than the table width
+
+// Device status bits (OR-ed by kernels, read by entro_last_device_status).
+constexpr uint32_t kStatCorrupt = 1u;         // index / stream / codebook disagree
+constexpr uint32_t kStatTimeout = 2u;         // a bounded wait on a bulk copy ran out
+
+// One tensor as the decode kernels see it.
+struct DevTensor {
+    const uint32_t* stream;
+    const uint64_t* offsets;      // n_chunks + 1
+    const uint16_t* sub_len;      // n_chunks * 32
+    uint16_t* out;                // fp16 bit patterns
+    uint64_t stream_words;
+    uint64_t n;
+    uint32_t chunk_symbols;
+    uint32_t n_chunks;
+    uint32_t nsym;
+    float scale;
+    int32_t zero_point;
+    uint32_t pad[3];
+    uint8_t len[ENTRO_MAX_SYMBOLS];
+};
+static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vectors");
+
+// Per-tensor tables for codes longer than the lookup table (canonical decode by range).
+struct DecodeAux {
+    unsigned long long limit[ENTRO_MAX_CODE_LEN + 1];  // left-justified end of the codes of length <= l
+    uint32_t first_code[ENTRO_MAX_CODE_LEN + 1];
+    uint32_t offset[ENTRO_MAX_CODE_LEN + 1];           // rank of the first symbol of length l
+    uint16_t val[ENTRO_MAX_SYMBOLS];                   // fp16( s * (q - z) ) per symbol
+    uint8_t sorted[ENTRO_MAX_SYMBOLS];                 // symbols by (length, symbol)
+    uint32_t max_len;
+    uint32_t pad[3];
+};
+static_assert(sizeof(DecodeAux) % 16 == 0, "DecodeAux is copied as 16-byte vectors");
+
+struct DecodeConfig {
+    int lut_bits = 11;
+    int warps_per_cta = 16;
+    int ctas_per_sm = 2;
+    int chunks_per_item = 64;
+};
+
+// Per-device workspace owned by the library.
+struct Workspace {
+    int device = -1;
+    int sm_count = 0;
+    int max_smem_optin = 0;
+    // device
+    void* dev = nullptr;
+    size_t dev_bytes = 0;
+    uint32_t* control = nullptr;      // [0] work counter, [1] status, [2..] scratch flags
+    // pinned host
+    void* pinned = nullptr;
+    size_t pinned_bytes = 0;
+    cudaEvent_t upload_done = nullptr; // last async read of `pinned` by the device
+    bool upload_pending = false;
+    // optional timing of the decode kernel (entro_profile_begin / entro_profile_read)
+    cudaEvent_t* prof_start = nullptr;
+    cudaEvent_t* prof_stop = nullptr;
+    int prof_cap = 0;
+    int prof_used = 0;
+};
+
+// Returns the workspace of the current device (creating it), or nullptr on a CUDA error.
+Workspace* workspace();
+// Grow the device / pinned areas to at least these sizes (contents are not preserved).
+bool reserve_device(Workspace* ws, size_t bytes);
+bool reserve_pinned(Workspace* ws, size_t bytes);
+// Wait until the device has finished reading the pinned area from an earlier call.
+bool wait_pinned_free(Workspace* ws);
+void mark_pinned_in_use(Workspace* ws, cudaStream_t s);
+void lock();
+void unlock();
+void count_launch(int n = 1);
+DecodeConfig& decode_config();
+
+struct Guard {
+    Guard() { lock(); }
+    ~Guard() { unlock(); }
+};
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline uint64_t num_chunks(uint64_t n, uint32_t c) { return (n + c - 1) / c; }
+bool codebook_lengths_valid(const entro_codebook* cb);
+
+}  // namespace entro
+
+#define ENTRO_CUDA(call)                                   \
+    do {                                                   \
+        cudaError_t e__ = (call);                          \
+        if (e__ != cudaSuccess) return ENTRO_ERR_CUDA;     \
+    } while (0)
