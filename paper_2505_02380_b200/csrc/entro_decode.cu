@@ -4,11 +4,21 @@
 // Work split: a chunk (one segment) is decoded by one warp, each lane owning one of the
 // chunk's 32 sub-blocks.  The lanes' start positions come from a warp prefix sum over the
 // sub-block bit lengths stored in the index.  The warp stages the chunk's bytes into
-// shared memory with one bulk asynchronous copy, every lane then walks its own bits with a
-// shared-memory lookup table whose entries already hold the dequantised fp16 value, and
-// the fp16 results leave through a swizzled shared-memory tile as full 16-byte-per-lane
-// coalesced stores.  A persistent grid pulls work items (runs of chunks of one tensor) from
-// a global counter, so one launch covers a whole model.
+// shared memory with one bulk asynchronous copy (the next chunk's bytes are prefetched
+// into L2 meanwhile), every lane then walks its own bits with shared-memory lookup tables
+// whose entries already hold dequantised fp16 values, and the results leave through a
+// swizzled shared-memory tile as coalesced 16-byte-per-lane stores.  A persistent grid
+// pulls work items (runs of chunks of one tensor) from a global counter; the warps of a
+// CTA share out an item's chunks through a shared-memory counter.
+//
+// Tables per tensor (built by build_tables_kernel, cached in shared memory per CTA):
+//   lut1  2^K entries indexed by the next K stream bits.
+//         alphabets > 16 symbols: one symbol per entry,  value << 16 | length, or kEscFlag
+//         alphabets <= 16 symbols: four symbols per entry, nibbles << 8 | total length, or
+//         kQuadEscFlag; the fp16 values come from a 256-entry table of symbol pairs
+//   lut2  second level for codes longer than K (single-symbol mode): indexed by
+//         (window - t2) >> shift2, same entry format
+//   aux   canonical ranges per length for whatever neither table resolves
 #include <cuda_fp16.h>
 
 #include "entro_internal.h"
@@ -18,16 +28,28 @@ namespace {
 
 constexpr int kTile = 32;                 // symbols per lane between two flushes of the output tile
 constexpr int kTileBytes = 32 * kTile * 2;
-constexpr uint32_t kWaitTries = 1u << 20; // bound on polling a bulk copy
+constexpr int kUnits = kTile / 8;         // 16-byte units per tile row
+constexpr uint32_t kWaitTries = 1u << 16; // bound on polling a bulk copy (each try may suspend)
+constexpr uint32_t kLut2MaxBits = 20;     // longest code the second level resolves
 
 // ------------------------------------------------------------------ table construction
 
-// One block per tensor: canonical decode tables from the code lengths, the fp16 value of
-// every symbol, and the 2^lut_bits-entry lookup table
-//   entry = fp16(s * (q - z)) << 16 | code length          (code fits in lut_bits)
-//   entry = kEscFlag                                        (longer code, or no codeword)
+__device__ __forceinline__ uint32_t range_decode(const DecodeAux& aux, uint32_t window, uint32_t max_l, uint32_t& len)
+{
+    // smallest l with window < limit[l]; the symbol is the (code - first_code)-th of that length
+    for (uint32_t l = 1; l <= max_l; ++l) {
+        if ((unsigned long long)window < aux.limit[l]) {
+            len = l;
+            return aux.sorted[(aux.offset[l] + ((window >> (32 - l)) - aux.first_code[l])) & 0xffu];
+        }
+    }
+    len = 0;
+    return 0;
+}
+
+// One block per tensor.
 __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __restrict__ tensors, int lut_bits,
-                                                           uint32_t* __restrict__ luts, DecodeAux* __restrict__ auxs,
+                                                           TensorTables* __restrict__ tables,
                                                            uint32_t* __restrict__ control)
 {
     __shared__ DecodeAux aux;
@@ -36,6 +58,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     const int t = blockIdx.x;
     const int tid = threadIdx.x;
     const DevTensor& T = tensors[t];
+    TensorTables& out = tables[t];
     if (t == 0 && tid == 0) control[0] = 0;   // work counter of the decode kernel that follows
     if (tid <= ENTRO_MAX_CODE_LEN) count[tid] = 0;
     len[tid] = (uint32_t)tid < T.nsym ? T.len[tid] : 0;
@@ -59,6 +82,24 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
             if (count[k]) max_len = k;
         }
         aux.max_len = max_len;
+        aux.quad = T.nsym <= 16 ? 1u : 0u;
+        // second level: windows at or above the end of the codes that fit the first level
+        aux.t2 = 0;
+        aux.shift2 = 0;
+        aux.n2 = 0;
+        const unsigned long long t2 = aux.limit[lut_bits];
+        if (!aux.quad && max_len > (uint32_t)lut_bits && t2 < (1ull << 32)) {
+            uint32_t bits = max_len < kLut2MaxBits ? max_len : kLut2MaxBits;
+            for (; bits > (uint32_t)lut_bits; --bits) {
+                unsigned long long n = ((1ull << 32) - t2 + (1ull << (32 - bits)) - 1) >> (32 - bits);
+                if (n <= (unsigned long long)kLut2Entries) {
+                    aux.t2 = (uint32_t)t2;
+                    aux.shift2 = 32 - bits;
+                    aux.n2 = (uint32_t)n;
+                    break;
+                }
+            }
+        }
         aux.pad[0] = aux.pad[1] = aux.pad[2] = 0;
     }
     __syncthreads();
@@ -67,31 +108,50 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
         for (int k = 0; k < tid; ++k) rank += (len[k] == l);
         aux.sorted[aux.offset[l] + rank] = (uint8_t)tid;
     }
-    float d = (float)(tid - T.zero_point);
+    const float d = (float)(tid - T.zero_point);
     aux.val[tid] = __half_as_ushort(__float2half_rn(__fmul_rn(T.scale, d)));
     __syncthreads();
-    // unused tail of sorted[] (fewer than 256 symbols in use) is never indexed; zero it anyway
     {
         uint32_t used = aux.offset[ENTRO_MAX_CODE_LEN] + count[ENTRO_MAX_CODE_LEN];
-        if ((uint32_t)tid >= used) aux.sorted[tid] = 0;
+        if ((uint32_t)tid >= used) aux.sorted[tid] = 0;   // never indexed; keep it defined
     }
     __syncthreads();
+
     const uint32_t entries = 1u << lut_bits;
-    uint32_t* lut = luts + (size_t)t * (1u << kMaxLutBits);
-    for (uint32_t i = tid; i < entries; i += 256) {
-        const uint32_t window = i << (32 - lut_bits);
-        uint32_t e = kEscFlag;
-        for (uint32_t k = 1; k <= (uint32_t)lut_bits && k <= aux.max_len; ++k) {
-            if ((unsigned long long)window < aux.limit[k]) {
-                uint32_t sym = aux.sorted[aux.offset[k] + ((window >> (32 - k)) - aux.first_code[k])];
-                e = ((uint32_t)aux.val[sym] << 16) | k;
-                break;
+    if (aux.quad) {
+        for (uint32_t i = tid; i < entries; i += 256) {
+            uint32_t window = i << (32 - lut_bits);
+            uint32_t used = 0, nibbles = 0;
+            bool ok = true;
+            for (int k = 0; k < 4; ++k) {
+                uint32_t sl;
+                uint32_t sym = range_decode(aux, window, (uint32_t)lut_bits - used, sl);
+                if (sl == 0) {
+                    ok = false;
+                    break;
+                }
+                nibbles |= sym << (4 * k);
+                used += sl;
+                window <<= sl;   // sl <= lut_bits < 32
             }
+            out.lut1[i] = ok ? ((nibbles << 8) | used) : kQuadEscFlag;
         }
-        lut[i] = e;
+        // fp16 values of a pair of symbols: low nibble first
+        out.lut2[tid] = (uint32_t)aux.val[tid & 15] | ((uint32_t)aux.val[tid >> 4] << 16);
+    } else {
+        for (uint32_t i = tid; i < entries; i += 256) {
+            uint32_t sl;
+            uint32_t sym = range_decode(aux, i << (32 - lut_bits), (uint32_t)lut_bits, sl);
+            out.lut1[i] = sl ? (((uint32_t)aux.val[sym] << 16) | sl) : kEscFlag;
+        }
+        for (uint32_t i = tid; i < aux.n2; i += 256) {
+            uint32_t sl;
+            uint32_t sym = range_decode(aux, aux.t2 + (i << aux.shift2), 32 - aux.shift2, sl);
+            out.lut2[i] = sl ? (((uint32_t)aux.val[sym] << 16) | sl) : kEscFlag;
+        }
     }
     const uint32_t* src = reinterpret_cast<const uint32_t*>(&aux);
-    uint32_t* dst = reinterpret_cast<uint32_t*>(auxs + t);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(&out.aux);
     for (uint32_t i = tid; i < sizeof(DecodeAux) / 4; i += 256) dst[i] = src[i];
 }
 
@@ -153,21 +213,104 @@ __device__ __forceinline__ void reader_skip(Reader& r, uint32_t n)
     r.nb -= (int)n;
 }
 
-// Canonical decode of one symbol from a 32-bit window by code ranges: codes longer than the
-// lookup table, and bit patterns that are no codeword at all (flagged, one bit dropped).
-// Returns an entry in table format (value << 16 | length).
+struct Tables {
+    const uint32_t* lut1;      // shared
+    const uint32_t* lut2;      // shared
+    const DecodeAux* aux;      // shared
+    uint32_t* status;          // global
+};
+
+// One symbol from a full 32-bit window by the canonical ranges; a pattern that is no
+// codeword is flagged and dropped as a single bit.  Entry format: value << 16 | length.
 __device__ __noinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32_t window, uint32_t* status)
 {
-    const uint32_t max_len = aux->max_len;
-    uint32_t l = 1;
-    for (; l <= max_len; ++l)
-        if ((unsigned long long)window < aux->limit[l]) break;
-    if (l > max_len) {
+    uint32_t len;
+    uint32_t sym = range_decode(*aux, window, aux->max_len, len);
+    if (len == 0) {
         atomicOr(status, kStatCorrupt);
         return 1u;
     }
-    uint32_t sym = aux->sorted[(aux->offset[l] + ((window >> (32 - l)) - aux->first_code[l])) & 0xffu];
-    return ((uint32_t)aux->val[sym] << 16) | l;
+    return ((uint32_t)aux->val[sym] << 16) | len;
+}
+
+// A symbol the first level could not resolve: second level, then the ranges.
+__device__ __forceinline__ uint32_t decode_long(const Tables& tb, uint32_t window)
+{
+    const DecodeAux* aux = tb.aux;
+    if (window >= aux->t2) {
+        uint32_t i = (window - aux->t2) >> aux->shift2;
+        if (i < aux->n2) {
+            uint32_t e = tb.lut2[i];
+            if (!(e & kEscFlag)) return e;
+        }
+    }
+    return decode_by_range(aux, window, tb.status);
+}
+
+// One symbol, any tensor mode (used off the fast path).
+template <int K>
+__device__ __forceinline__ uint32_t decode_one(const Tables& tb, uint32_t window)
+{
+    if (tb.aux->quad) return decode_by_range(tb.aux, window, tb.status);
+    uint32_t e = tb.lut1[window >> (32 - K)];
+    if (e & kEscFlag) e = decode_long(tb, window);
+    return e;
+}
+
+// Out-of-line repair of a pair of lookups in which at least one hit an escape entry.  On
+// entry the window stands before the first unresolved symbol (escape entries have length
+// 0): before symbol 0 if e0 is an escape, else before symbol 1.
+struct PairFix {
+    Reader r;
+    uint32_t e0, e1;
+};
+
+template <int K>
+__device__ __noinline__ PairFix redo_pair(const uint32_t* lut1, const uint32_t* lut2, const DecodeAux* aux,
+                                         uint32_t* status, const uint32_t* words, uint32_t last, Reader r,
+                                         uint32_t e0)
+{
+    Tables tb{lut1, lut2, aux, status};
+    SmemSource src{words, last};
+    PairFix f;
+    if (e0 & kEscFlag) {
+        reader_refill(r, src);
+        e0 = decode_long(tb, r.hi);
+        reader_skip(r, e0 & 0xffu);
+    }
+    reader_refill(r, src);
+    uint32_t e1 = lut1[r.hi >> (32 - K)];
+    if (e1 & kEscFlag) e1 = decode_long(tb, r.hi);
+    reader_skip(r, e1 & 0xffu);
+    f.r = r;
+    f.e0 = e0;
+    f.e1 = e1;
+    return f;
+}
+
+// The same for a four-symbol entry: the four symbols one by one.  Returns the two pair
+// bytes (symbols 0,1 and 2,3) in e0, e1.
+__device__ __noinline__ PairFix redo_quad(const DecodeAux* aux, uint32_t* status, const uint32_t* words,
+                                         uint32_t last, Reader r)
+{
+    SmemSource src{words, last};
+    PairFix f;
+    uint32_t nib = 0;
+    for (int k = 0; k < 4; ++k) {
+        reader_refill(r, src);
+        uint32_t len;
+        uint32_t sym = range_decode(*aux, r.hi, aux->max_len, len);
+        if (len == 0) {
+            atomicOr(status, kStatCorrupt);
+            len = 1;
+        }
+        reader_skip(r, len);
+        nib |= (sym & 15u) << (4 * k);
+    }
+    f.r = r;
+    f.e0 = nib & 0xffu;
+    f.e1 = nib >> 8;
+    return f;
 }
 
 // ------------------------------------------------------------------ bulk copy + mbarrier
@@ -187,17 +330,23 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  : "memory");
 }
 
-// Bounded wait for phase `parity` of the barrier; false if the bound ran out.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+
+// Bounded wait for phase `parity` of the barrier; false if the bound ran out.  Each try may
+// suspend the thread for up to the hinted time, so waiting costs few issue slots.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
     for (uint32_t tries = 0; tries < kWaitTries; ++tries) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(20000u)
             : "memory");
         if (done) return true;
     }
@@ -207,22 +356,30 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 // ------------------------------------------------------------------ one chunk
 
 struct WarpCtx {
-    const uint32_t* lut;       // shared
-    const DecodeAux* aux;      // shared
+    Tables tb;
     uint32_t* stage;           // shared, this warp's compressed bytes
     uint4* tile;               // shared, this warp's output tile
     uint32_t bar;              // shared address of this warp's mbarrier
     uint32_t stage_bytes;
     uint32_t phase;
-    uint32_t* status;
     bool dead;                 // a bulk copy never completed: stop using the stage buffer
 };
+
+// Byte range of the stream that decoding chunk c touches, or false if the index does not
+// describe a range inside the stream buffer.  A lane may look 12 bytes past its end.
+__device__ __forceinline__ bool chunk_range(const DevTensor& T, uint64_t off0, uint64_t off1, uint64_t& byte0,
+                                            uint64_t& byte1)
+{
+    byte0 = (off0 >> 3) & ~15ull;
+    byte1 = ((off1 >> 3) + 13 + 15) & ~15ull;
+    return off1 >= off0 && off1 - off0 <= 32ull * 65535ull && byte1 <= T.stream_words * 4;
+}
 
 // General path: any symbol count per lane, words fetched straight from global memory,
 // scalar stores.  Used for the ragged last chunk of a tensor and for chunks whose bytes do
 // not fit the stage buffer.
 template <int K>
-__device__ __noinline__ void decode_chunk_general(const WarpCtx& cx, const DevTensor& T, uint32_t c, uint64_t off0,
+__device__ __noinline__ void decode_chunk_general(Tables tb, const DevTensor& T, uint32_t c, uint64_t off0,
                                                   uint32_t excl, uint32_t my_bits, uint32_t lane)
 {
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
@@ -238,13 +395,28 @@ __device__ __noinline__ void decode_chunk_general(const WarpCtx& cx, const DevTe
     uint16_t* out = T.out + chunk_first + lane_first;
     for (uint32_t i = 0; i < cnt; ++i) {
         reader_refill(r, src);
-        uint32_t e = cx.lut[r.hi >> (32 - K)];
-        if (e & kEscFlag) e = decode_by_range(cx.aux, r.hi, cx.status);
+        uint32_t e = decode_one<K>(tb, r.hi);
         reader_skip(r, e & 0xffu);
         out[i] = (uint16_t)(e >> 16);
     }
     const uint64_t used = ((uint64_t)r.next << 5) - (uint64_t)r.nb - (pos & 31);
-    if (used != my_bits) atomicOr(cx.status, kStatCorrupt);
+    if (used != my_bits) atomicOr(tb.status, kStatCorrupt);
+}
+
+// Flush the warp's output tile: each instruction writes (32 / kUnits) rows of kTile * 2
+// contiguous bytes; row r of the tile belongs to lane r's sub-block.
+__device__ __forceinline__ void flush_tile(const uint4* tile, uint16_t* out_chunk, uint32_t sub, uint32_t t0,
+                                           uint32_t lane)
+{
+#pragma unroll
+    for (int i = 0; i < kUnits; ++i) {
+        const uint32_t row = i * (32 / kUnits) + lane / kUnits;
+        const uint32_t unit = lane % kUnits;
+        const uint32_t swz = (row / (8 / kUnits)) % kUnits;
+        uint4 v = tile[row * kUnits + (unit ^ swz)];
+        uint4* dst = reinterpret_cast<uint4*>(out_chunk + (uint64_t)row * sub + t0) + unit;
+        __stcs(dst, v);
+    }
 }
 
 // Fast path: a full chunk whose bytes are staged in shared memory.
@@ -259,83 +431,103 @@ __device__ __forceinline__ void decode_chunk_staged(WarpCtx& cx, const DevTensor
     bool ok = mbar_wait(cx.bar, cx.phase);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) {
-        if (lane == 0) atomicOr(cx.status, kStatTimeout);
+        if (lane == 0) atomicOr(cx.tb.status, kStatTimeout);
         cx.dead = true;
         return;
     }
     cx.phase ^= 1u;
 
-    SmemSource src{cx.stage, copy_bytes / 4 - 1};
+    const SmemSource src{cx.stage, copy_bytes / 4 - 1};
     const uint32_t pos = (uint32_t)(off0 - byte0 * 8) + excl;     // bit position inside the stage buffer
     Reader r;
     reader_init(r, src, pos >> 5, pos & 31);
 
-    const uint32_t* lut = cx.lut;
+    const uint32_t* lut1 = cx.tb.lut1;
     // tile row = lane, 16-byte units swizzled so that both the per-lane writes and the
-    // row-wise reads below touch every bank once
-    constexpr int kUnits = kTile / 8;                             // 16-byte units per row
+    // row-wise reads of the flush touch every bank once
     const uint32_t row_swz = (lane / (8 / kUnits)) % kUnits;
     uint4* my_row = cx.tile + lane * kUnits;
     uint16_t* out_chunk = T.out + (uint64_t)c * T.chunk_symbols;
 
-    for (uint32_t t0 = 0; t0 < sub; t0 += kTile) {
+    if (cx.tb.aux->quad) {
+        const uint32_t* pair_val = cx.tb.lut2;
+        for (uint32_t t0 = 0; t0 < sub; t0 += kTile) {
+#pragma unroll 1
+            for (int g = 0; g < kUnits; ++g) {
+                uint32_t packed[4];
 #pragma unroll
-        for (int g = 0; g < kUnits; ++g) {
-            uint32_t packed[4];
-#pragma unroll
-            for (int p = 0; p < 4; ++p) {
-                reader_refill(r, src);
-                uint32_t e0 = lut[r.hi >> (32 - K)];
-                r.hi = __funnelshift_l(r.lo, r.hi, e0);
-                r.lo = __funnelshift_l(0u, r.lo, e0);
-                uint32_t e1 = lut[r.hi >> (32 - K)];
-                r.hi = __funnelshift_l(r.lo, r.hi, e1);
-                r.lo = __funnelshift_l(0u, r.lo, e1);
-                r.nb -= (int)((e0 + e1) & 0xffu);
-                if ((e0 | e1) & kEscFlag) {
-                    // An escape entry has length 0, so the window has not moved past it.
-                    if (e0 & kEscFlag) {
-                        reader_refill(r, src);
-                        e0 = decode_by_range(cx.aux, r.hi, cx.status);
-                        reader_skip(r, e0 & 0xffu);
-                        reader_refill(r, src);
-                        e1 = lut[r.hi >> (32 - K)];
-                        if (e1 & kEscFlag) e1 = decode_by_range(cx.aux, r.hi, cx.status);
-                        reader_skip(r, e1 & 0xffu);
-                    } else {
-                        reader_refill(r, src);
-                        e1 = decode_by_range(cx.aux, r.hi, cx.status);
-                        reader_skip(r, e1 & 0xffu);
+                for (int h = 0; h < 2; ++h) {
+                    reader_refill(r, src);
+                    uint32_t e = lut1[r.hi >> (32 - K)];
+                    r.hi = __funnelshift_l(r.lo, r.hi, e);
+                    r.lo = __funnelshift_l(0u, r.lo, e);
+                    r.nb -= (int)(e & 0xffu);
+                    uint32_t b0 = __byte_perm(e, 0u, 0x4441);     // byte 1: symbols 0, 1
+                    uint32_t b1 = __byte_perm(e, 0u, 0x4442);     // byte 2: symbols 2, 3
+                    if (__builtin_expect(e & kQuadEscFlag, 0)) {
+                        PairFix f = redo_quad(cx.tb.aux, cx.tb.status, src.words, src.last, r);
+                        r = f.r;
+                        b0 = f.e0;
+                        b1 = f.e1;
                     }
+                    packed[2 * h] = pair_val[b0];
+                    packed[2 * h + 1] = pair_val[b1];
                 }
-                packed[p] = __byte_perm(e0, e1, 0x7632);          // two fp16 values, first symbol low
+                my_row[g ^ row_swz] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
             }
-            my_row[g ^ row_swz] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            __syncwarp();
+            flush_tile(cx.tile, out_chunk, sub, t0, lane);
+            __syncwarp();
         }
-        __syncwarp();
-        // flush: each instruction writes (32 / kUnits) rows of (kTile * 2) contiguous bytes
+    } else {
+        for (uint32_t t0 = 0; t0 < sub; t0 += kTile) {
+#pragma unroll 1
+            for (int g = 0; g < kUnits; ++g) {
+                uint32_t packed[4];
 #pragma unroll
-        for (int i = 0; i < kUnits; ++i) {
-            const uint32_t row = i * (32 / kUnits) + lane / kUnits;
-            const uint32_t unit = lane % kUnits;
-            const uint32_t swz = (row / (8 / kUnits)) % kUnits;
-            uint4 v = cx.tile[row * kUnits + (unit ^ swz)];
-            uint4* dst = reinterpret_cast<uint4*>(out_chunk + (uint64_t)row * sub + t0) + unit;
-            __stcs(dst, v);
+                for (int p = 0; p < 4; ++p) {
+                    reader_refill(r, src);
+                    uint32_t e0 = lut1[r.hi >> (32 - K)];
+                    r.hi = __funnelshift_l(r.lo, r.hi, e0);
+                    r.lo = __funnelshift_l(0u, r.lo, e0);
+                    uint32_t e1 = lut1[r.hi >> (32 - K)];
+                    r.hi = __funnelshift_l(r.lo, r.hi, e1);
+                    r.lo = __funnelshift_l(0u, r.lo, e1);
+                    r.nb -= (int)((e0 + e1) & 0xffu);
+                    if (__builtin_expect((e0 | e1) & kEscFlag, 0)) {
+                        PairFix f = redo_pair<K>(lut1, cx.tb.lut2, cx.tb.aux, cx.tb.status, src.words, src.last, r, e0);
+                        r = f.r;
+                        e0 = f.e0;
+                        e1 = f.e1;
+                    }
+                    packed[p] = __byte_perm(e0, e1, 0x7632);      // two fp16 values, first symbol low
+                }
+                my_row[g ^ row_swz] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            }
+            __syncwarp();
+            flush_tile(cx.tile, out_chunk, sub, t0, lane);
+            __syncwarp();
         }
-        __syncwarp();
     }
     const uint32_t used = (r.next << 5) - (uint32_t)r.nb - pos;
-    if (used != my_bits) atomicOr(cx.status, kStatCorrupt);
+    if (used != my_bits) atomicOr(cx.tb.status, kStatCorrupt);
     __syncwarp();   // all lanes are done with the stage buffer before it is overwritten
 }
 
+// Decode chunk c; `next_c` (or 0xffffffff) is the chunk this warp will take afterwards, whose
+// bytes are pulled into L2 while this one is being decoded.
 template <int K>
-__device__ __forceinline__ void decode_chunk(WarpCtx& cx, const DevTensor& T, uint32_t c, uint32_t lane)
+__device__ __forceinline__ void decode_chunk(WarpCtx& cx, const DevTensor& T, uint32_t c, uint32_t next_c,
+                                             uint32_t lane)
 {
     const uint64_t off0 = T.offsets[c];
     const uint64_t off1 = T.offsets[c + 1];
     const uint32_t my_bits = T.sub_len[(uint64_t)c * kSubBlocks + lane];
+    if (next_c < T.n_chunks && lane == 0) {
+        uint64_t b0, b1;
+        if (chunk_range(T, T.offsets[next_c], T.offsets[next_c + 1], b0, b1))
+            bulk_prefetch_l2(reinterpret_cast<const char*>(T.stream) + b0, (uint32_t)(b1 - b0));
+    }
     uint32_t incl = my_bits;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -345,11 +537,9 @@ __device__ __forceinline__ void decode_chunk(WarpCtx& cx, const DevTensor& T, ui
     const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
     const uint32_t excl = incl - my_bits;
 
-    // the index must describe a range inside the stream buffer
-    const uint64_t byte0 = (off0 >> 3) & ~15ull;
-    const uint64_t byte1 = ((off1 >> 3) + 13 + 15) & ~15ull;      // a lane may look 12 bytes past its end
-    if (off1 < off0 || off1 - off0 != total || byte1 > T.stream_words * 4) {
-        if (lane == 0) atomicOr(cx.status, kStatCorrupt);
+    uint64_t byte0, byte1;
+    if (!chunk_range(T, off0, off1, byte0, byte1) || off1 - off0 != total) {
+        if (lane == 0) atomicOr(cx.tb.status, kStatCorrupt);
         return;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
@@ -358,7 +548,7 @@ __device__ __forceinline__ void decode_chunk(WarpCtx& cx, const DevTensor& T, ui
     if (full && (sub % kTile) == 0 && copy_bytes <= cx.stage_bytes && !cx.dead)
         decode_chunk_staged<K>(cx, T, c, off0, byte0, (uint32_t)copy_bytes, excl, my_bits, lane);
     else
-        decode_chunk_general<K>(cx, T, c, off0, excl, my_bits, lane);
+        decode_chunk_general<K>(cx.tb, T, c, off0, excl, my_bits, lane);
 }
 
 // ------------------------------------------------------------------ persistent kernel
@@ -368,33 +558,33 @@ __device__ __forceinline__ void decode_chunk(WarpCtx& cx, const DevTensor& T, ui
 template <int K>
 __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __restrict__ tensors, int ntensors,
                                                          const uint32_t* __restrict__ item_start,
-                                                         const uint32_t* __restrict__ luts,
-                                                         const DecodeAux* __restrict__ auxs, uint32_t chunks_per_item,
-                                                         uint32_t stage_bytes, uint32_t* __restrict__ control)
+                                                         const TensorTables* __restrict__ tables,
+                                                         uint32_t chunks_per_item, uint32_t stage_bytes,
+                                                         uint32_t* __restrict__ control)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    // layout: [lut][aux][tensor][per-warp tile][per-warp stage][mbarriers][item slots]
-    uint32_t* s_lut = reinterpret_cast<uint32_t*>(smem);
-    DecodeAux* s_aux = reinterpret_cast<DecodeAux*>(smem + (4u << K));
-    DevTensor* s_tensor = reinterpret_cast<DevTensor*>(smem + (4u << K) + sizeof(DecodeAux));
-    unsigned char* p = smem + (4u << K) + sizeof(DecodeAux) + sizeof(DevTensor);
+    // layout: [lut1][lut2][aux][tensor][per-warp tile][per-warp stage][mbarriers][item + claim slots]
+    uint32_t* s_lut1 = reinterpret_cast<uint32_t*>(smem);
+    uint32_t* s_lut2 = s_lut1 + (1u << K);
+    DecodeAux* s_aux = reinterpret_cast<DecodeAux*>(s_lut2 + kLut2Entries);
+    DevTensor* s_tensor = reinterpret_cast<DevTensor*>(s_aux + 1);
+    unsigned char* p = reinterpret_cast<unsigned char*>(s_tensor + 1);
     p = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(p) + 127) & ~(uintptr_t)127);
     const uint32_t warps = blockDim.x >> 5;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     unsigned char* tiles = p;
     unsigned char* stages = tiles + (size_t)warps * kTileBytes;
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(stages + (size_t)warps * stage_bytes);
-    volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(bars + warps);
+    volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(bars + warps);   // [2]
+    uint32_t* s_claim = const_cast<uint32_t*>(s_item) + 2;                            // [2]
 
     WarpCtx cx;
-    cx.lut = s_lut;
-    cx.aux = s_aux;
+    cx.tb = Tables{s_lut1, s_lut2, s_aux, control + 1};
     cx.tile = reinterpret_cast<uint4*>(tiles + (size_t)warp * kTileBytes);
     cx.stage = reinterpret_cast<uint32_t*>(stages + (size_t)warp * stage_bytes);
     cx.bar = smem_addr(bars + warp);
     cx.stage_bytes = stage_bytes;
     cx.phase = 0;
-    cx.status = control + 1;
     cx.dead = false;
 
     if (lane == 0) mbar_init(cx.bar, 1);
@@ -402,7 +592,10 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
     const uint32_t total_items = item_start[ntensors];
-    if (threadIdx.x == 0) s_item[0] = atomicAdd(control, 1u);
+    if (threadIdx.x == 0) {
+        s_item[0] = atomicAdd(control, 1u);
+        s_claim[0] = 0;
+    }
     __syncthreads();
     int cur = -1;
     uint32_t slot = 0;
@@ -410,7 +603,10 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
         const uint32_t item = s_item[slot];
         if (item >= total_items) break;
         // claim the next item early; it is read after the barrier that ends this one
-        if (threadIdx.x == 0) s_item[slot ^ 1u] = atomicAdd(control, 1u);
+        if (threadIdx.x == 0) {
+            s_item[slot ^ 1u] = atomicAdd(control, 1u);
+            s_claim[slot ^ 1u] = 0;
+        }
         // tensor of this item: last t with item_start[t] <= item
         int lo = 0, hi = ntensors - 1;
         while (lo < hi) {
@@ -420,10 +616,14 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
         }
         if (lo != cur) {
             cur = lo;
-            const uint4* gl = reinterpret_cast<const uint4*>(luts + (size_t)cur * (1u << kMaxLutBits));
-            uint4* sl = reinterpret_cast<uint4*>(s_lut);
-            for (uint32_t i = threadIdx.x; i < (1u << K) / 4; i += blockDim.x) sl[i] = __ldg(gl + i);
-            const uint4* ga = reinterpret_cast<const uint4*>(auxs + cur);
+            const TensorTables* tt = tables + cur;
+            const uint4* g1 = reinterpret_cast<const uint4*>(tt->lut1);
+            uint4* s1 = reinterpret_cast<uint4*>(s_lut1);
+            for (uint32_t i = threadIdx.x; i < (1u << K) / 4; i += blockDim.x) s1[i] = __ldg(g1 + i);
+            const uint4* g2 = reinterpret_cast<const uint4*>(tt->lut2);
+            uint4* s2 = reinterpret_cast<uint4*>(s_lut2);
+            for (uint32_t i = threadIdx.x; i < kLut2Entries / 4; i += blockDim.x) s2[i] = __ldg(g2 + i);
+            const uint4* ga = reinterpret_cast<const uint4*>(&tt->aux);
             uint4* sa = reinterpret_cast<uint4*>(s_aux);
             for (uint32_t i = threadIdx.x; i < sizeof(DecodeAux) / 16; i += blockDim.x) sa[i] = __ldg(ga + i);
             const uint4* gt = reinterpret_cast<const uint4*>(tensors + cur);
@@ -433,9 +633,19 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
         }
         const DevTensor& T = *s_tensor;
         const uint32_t first = (item - __ldg(item_start + cur)) * chunks_per_item;
-        const uint32_t last = min(first + chunks_per_item, T.n_chunks);
-        for (uint32_t c = first + warp; c < last; c += warps) decode_chunk<K>(cx, T, c, lane);
-        __syncthreads();   // tables may be replaced, and s_item[slot ^ 1] is now visible
+        const uint32_t count = min(chunks_per_item, T.n_chunks - first);
+        // the warps share out the item's chunks; each keeps one claim ahead for the L2 prefetch
+        uint32_t k = 0;
+        if (lane == 0) k = atomicAdd(&s_claim[slot], 1u);
+        k = __shfl_sync(0xffffffffu, k, 0);
+        while (k < count) {
+            uint32_t kn = 0;
+            if (lane == 0) kn = atomicAdd(&s_claim[slot], 1u);
+            kn = __shfl_sync(0xffffffffu, kn, 0);
+            decode_chunk<K>(cx, T, first + k, kn < count ? first + kn : 0xffffffffu, lane);
+            k = kn;
+        }
+        __syncthreads();   // tables may be replaced; s_item / s_claim [slot ^ 1] are now visible
         slot ^= 1u;
     }
     // A warp that gave up on a bulk copy lets it land (bounded) before its buffer goes away.
@@ -450,12 +660,11 @@ struct Shape {
 // Shared memory of one CTA for a launch shape; stage_bytes == 0 if it cannot fit.
 Shape shape_for(const DecodeConfig& cfg, int max_smem, uint32_t want_stage)
 {
-    size_t fixed = (4u << cfg.lut_bits) + sizeof(DecodeAux) + sizeof(DevTensor) + 128;
+    size_t fixed = (4u << cfg.lut_bits) + 4u * kLut2Entries + sizeof(DecodeAux) + sizeof(DevTensor) + 128;
     size_t per_warp_fixed = kTileBytes + 8;
     size_t tail = 16;
     size_t budget = (size_t)max_smem / cfg.ctas_per_sm;
     if (cfg.ctas_per_sm > 1) budget -= 1024;   // per-CTA reservation of the driver
-    if (budget > (size_t)max_smem) budget = max_smem;
     Shape s{0, 0};
     if (budget < fixed + tail + cfg.warps_per_cta * (per_warp_fixed + 512)) return s;
     size_t avail = (budget - fixed - tail) / cfg.warps_per_cta - per_warp_fixed;
@@ -468,8 +677,8 @@ Shape shape_for(const DecodeConfig& cfg, int max_smem, uint32_t want_stage)
 
 template <int K>
 entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
-                           const uint32_t* item_start, uint32_t total_items, const uint32_t* luts,
-                           const DecodeAux* auxs, uint32_t want_stage, cudaStream_t s)
+                           const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
+                           uint32_t want_stage, cudaStream_t s)
 {
     Shape sh = shape_for(cfg, ws->max_smem_optin, want_stage);
     if (sh.stage_bytes == 0) return ENTRO_ERR_UNSUPPORTED;
@@ -482,7 +691,7 @@ entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTens
     if (grid > total_items) grid = total_items;
     const bool timed = ws->prof_used < ws->prof_cap;
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_start[ws->prof_used], s));
-    decode_kernel<K><<<grid, cfg.warps_per_cta * 32, sh.smem, s>>>(tensors, ntensors, item_start, luts, auxs,
+    decode_kernel<K><<<grid, cfg.warps_per_cta * 32, sh.smem, s>>>(tensors, ntensors, item_start, tables,
                                                                    (uint32_t)cfg.chunks_per_item, sh.stage_bytes,
                                                                    ws->control);
     count_launch();
@@ -511,7 +720,6 @@ entro_status validate_desc(const entro_tensor_desc& d)
 entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs, int ntensors, cudaStream_t s)
 {
     const DecodeConfig cfg = decode_config();
-    // keep only tensors that have symbols
     int live = 0;
     for (int i = 0; i < ntensors; ++i) {
         entro_status st = validate_desc(descs[i]);
@@ -523,10 +731,9 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     const size_t tensors_bytes = (size_t)live * sizeof(DevTensor);
     const size_t items_bytes = (((size_t)live + 1) * 4 + 15) & ~(size_t)15;
     const size_t upload_bytes = tensors_bytes + items_bytes;
-    const size_t aux_bytes = (size_t)live * sizeof(DecodeAux);
-    const size_t lut_bytes = (size_t)live * (4u << kMaxLutBits);
+    const size_t tables_bytes = (size_t)live * sizeof(TensorTables);
     if (!reserve_pinned(ws, upload_bytes)) return ENTRO_ERR_CUDA;
-    if (!reserve_device(ws, upload_bytes + aux_bytes + lut_bytes)) return ENTRO_ERR_CUDA;
+    if (!reserve_device(ws, upload_bytes + tables_bytes)) return ENTRO_ERR_CUDA;
 
     DevTensor* ht = static_cast<DevTensor*>(ws->pinned);
     uint32_t* hitems = reinterpret_cast<uint32_t*>(static_cast<char*>(ws->pinned) + tensors_bytes);
@@ -554,9 +761,10 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
         hitems[k] = (uint32_t)items;
         items += (nc + cfg.chunks_per_item - 1) / cfg.chunks_per_item;
         if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
-        // stage buffer: the chunk at one byte per symbol (an 8-bit alphabet cannot average
-        // more for long), or 5/8 of that for alphabets of 16 symbols and fewer
-        uint32_t want = d.cb.nsym <= 16 ? (d.chunk_symbols * 5) / 8 : d.chunk_symbols;
+        // stage buffer: room for a chunk at one byte per symbol (an 8-bit alphabet averages
+        // less), or 3/8 of a byte for alphabets of 16 symbols and fewer; chunks that need
+        // more take the general path
+        uint32_t want = d.cb.nsym <= 16 ? (d.chunk_symbols * 3) / 8 : d.chunk_symbols;
         want = ((want + 127) & ~127u) + 128;
         if (want > want_stage) want_stage = want;
         ++k;
@@ -566,17 +774,16 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     char* base = static_cast<char*>(ws->dev);
     DevTensor* dt = reinterpret_cast<DevTensor*>(base);
     uint32_t* ditems = reinterpret_cast<uint32_t*>(base + tensors_bytes);
-    DecodeAux* dauxs = reinterpret_cast<DecodeAux*>(base + upload_bytes);
-    uint32_t* dluts = reinterpret_cast<uint32_t*>(base + upload_bytes + aux_bytes);
+    TensorTables* dtables = reinterpret_cast<TensorTables*>(base + upload_bytes);
     ENTRO_CUDA(cudaMemcpyAsync(dt, ht, upload_bytes, cudaMemcpyHostToDevice, s));
     mark_pinned_in_use(ws, s);
-    build_tables_kernel<<<live, 256, 0, s>>>(dt, cfg.lut_bits, dluts, dauxs, ws->control);
+    build_tables_kernel<<<live, 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     switch (cfg.lut_bits) {
-        case 10: return launch_decode<10>(ws, cfg, dt, live, ditems, (uint32_t)items, dluts, dauxs, want_stage, s);
-        case 11: return launch_decode<11>(ws, cfg, dt, live, ditems, (uint32_t)items, dluts, dauxs, want_stage, s);
-        case 12: return launch_decode<12>(ws, cfg, dt, live, ditems, (uint32_t)items, dluts, dauxs, want_stage, s);
+        case 10: return launch_decode<10>(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, want_stage, s);
+        case 11: return launch_decode<11>(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, want_stage, s);
+        case 12: return launch_decode<12>(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, want_stage, s);
     }
     return ENTRO_ERR_UNSUPPORTED;
 }

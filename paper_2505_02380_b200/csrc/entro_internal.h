@@ -34,7 +34,10 @@ struct DevTensor {
 };
 static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vectors");
 
-// Per-tensor tables for codes longer than the lookup table (canonical decode by range).
+constexpr int kLut2Entries = 2048;            // capacity of the second-level table
+constexpr uint32_t kQuadEscFlag = 0x80000000u; // four-symbol entry: the four codes do not fit
+
+// Per-tensor tables beside the first-level lookup table.
 struct DecodeAux {
     unsigned long long limit[ENTRO_MAX_CODE_LEN + 1];  // left-justified end of the codes of length <= l
     uint32_t first_code[ENTRO_MAX_CODE_LEN + 1];
@@ -42,15 +45,27 @@ struct DecodeAux {
     uint16_t val[ENTRO_MAX_SYMBOLS];                   // fp16( s * (q - z) ) per symbol
     uint8_t sorted[ENTRO_MAX_SYMBOLS];                 // symbols by (length, symbol)
     uint32_t max_len;
+    uint32_t quad;     // 1: first-level entries decode four symbols (alphabets of <= 16 symbols)
+    uint32_t t2;       // second level covers windows >= t2 (left-justified), in steps of 1 << shift2
+    uint32_t shift2;
+    uint32_t n2;       // entries in use in the second-level table (0 = none)
     uint32_t pad[3];
 };
 static_assert(sizeof(DecodeAux) % 16 == 0, "DecodeAux is copied as 16-byte vectors");
+
+// Everything the decode kernel loads into shared memory when it switches tensor.
+struct TensorTables {
+    uint32_t lut1[1u << kMaxLutBits];
+    uint32_t lut2[kLut2Entries];   // single-symbol mode: second level; four-symbol mode: [0, 256) pair values
+    DecodeAux aux;
+};
+static_assert(sizeof(TensorTables) % 16 == 0, "TensorTables is copied as 16-byte vectors");
 
 struct DecodeConfig {
     int lut_bits = 11;
     int warps_per_cta = 16;
     int ctas_per_sm = 2;
-    int chunks_per_item = 64;
+    int chunks_per_item = 256;
 };
 
 // Per-device workspace owned by the library.
