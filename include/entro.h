@@ -49,6 +49,7 @@ extern "C" {
 #define ENTRO_SUB_BLOCKS 32
 #define ENTRO_STREAM_SLACK_WORDS 8
 #define ENTRO_MAX_CHUNK_SYMBOLS 16384
+#define ENTRO_STATIC_MAX_TENSORS 8
 
 typedef enum {
     ENTRO_OK = 0,
@@ -58,7 +59,8 @@ typedef enum {
     ENTRO_ERR_CODE_TOO_LONG = 4,   /* an optimal code length exceeds 32 bits */
     ENTRO_ERR_CORRUPT_STREAM = 5,  /* stream, index and codebook do not agree */
     ENTRO_ERR_CUDA = 6,            /* a CUDA runtime call failed */
-    ENTRO_ERR_UNSUPPORTED = 7
+    ENTRO_ERR_UNSUPPORTED = 7,
+    ENTRO_ERR_TOO_MANY_TENSORS = 8 /* more tensors than entro_decode_dequant_static has room for */
 } entro_status;
 
 /* The paper applies "either unsigned or asymmetric quantization per layer, based on its
@@ -191,6 +193,37 @@ typedef struct {
 entro_status entro_decode_dequant_batched_host(const entro_tensor_desc *descs_host,
                                                const entro_host_io *io_host, int ntensors,
                                                void *cuda_stream);
+
+/*
+ * entro_decode_dequant_batched for callers that cannot allocate device memory.  (The paper
+ * has no counterpart; this entry point exists for the sake of the host application.)
+ *
+ * The other decode calls keep their descriptors and decode tables in a workspace that the
+ * library obtains with cudaMalloc / cudaMallocHost on first use and re-allocates when a
+ * larger model arrives.  That is unusable where the application has already handed all
+ * device memory to its own pool, where an allocation (which synchronises the whole device)
+ * would stall kernels running on other streams, or where the CUDA allocator must not be
+ * entered at all.  This variant calls no allocator: descriptors travel as kernel
+ * arguments, and tables, work counter and status word live in an array that is part of the
+ * library's device image (about 210 KB, held on every GPU that loads the library until
+ * the process exits).
+ *
+ *  - At most ENTRO_STATIC_MAX_TENSORS tensors with n > 0 per call; more returns
+ *    ENTRO_ERR_TOO_MANY_TENSORS and launches nothing.  Decode a larger model in slices.
+ *  - The first call on each device looks up the array's device address (that device must
+ *    be current, as for every call); make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps what the previous call left:
+ *    each call rewrites what it uses and clears its counter and status first.  Two calls
+ *    whose kernels overlap on the GPU (different streams, no event between them) race on
+ *    it; keep them on one stream or order them.
+ *  - status_dev: NULL, or a device pointer to one uint32_t that receives 0 if every chunk
+ *    decoded cleanly and a non-zero value if stream, index and codebook disagreed
+ *    (written asynchronously on cuda_stream; entro_last_device_status does not see this
+ *    call).  Output, alignment rules and error behaviour are otherwise those of
+ *    entro_decode_dequant_batched.  Asynchronous.
+ */
+entro_status entro_decode_dequant_static(const entro_tensor_desc *descs_host, int ntensors,
+                                         uint32_t *status_dev, void *cuda_stream);
 
 /*
  * Synchronise cuda_stream, then report and clear what decode kernels found since the last

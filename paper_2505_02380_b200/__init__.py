@@ -23,7 +23,8 @@ STREAM_SLACK_WORDS = 8
 MODE_AUTO, MODE_UNSIGNED, MODE_ASYMMETRIC = 0, 1, 2
 
 OK, ERR_INVALID_ARG, ERR_BUFFER_TOO_SMALL, ERR_NONFINITE, ERR_CODE_TOO_LONG, ERR_CORRUPT_STREAM, ERR_CUDA, \
-    ERR_UNSUPPORTED = range(8)
+    ERR_UNSUPPORTED, ERR_TOO_MANY_TENSORS = range(9)
+STATIC_MAX_TENSORS = 8
 
 
 class EntroError(RuntimeError):
@@ -95,6 +96,7 @@ def lib():
         L.entro_decode_dequant.argtypes = [vp, u64, vp, u64, u32, C.POINTER(Codebook), C.c_float, C.c_int32, vp, vp]
         L.entro_decode_dequant_batched.argtypes = [C.POINTER(TensorDesc), i32, vp]
         L.entro_decode_dequant_batched_host.argtypes = [C.POINTER(TensorDesc), C.POINTER(HostIO), i32, vp]
+        L.entro_decode_dequant_static.argtypes = [C.POINTER(TensorDesc), i32, vp, vp]
         L.entro_last_device_status.argtypes = [vp]
         L.entro_set_decode_config.argtypes = [i32, i32, i32, i32]
         L.entro_profile_begin.argtypes = [i32]
@@ -113,7 +115,8 @@ def lib():
 # Every symbol include/entro.h declares.
 EXPORTS = ["entro_quantize_tensor", "entro_histogram", "entro_build_codebook", "entro_stream_words",
            "entro_encode_bound_words", "entro_index_bytes", "entro_encode", "entro_decode_dequant",
-           "entro_decode_dequant_batched", "entro_decode_dequant_batched_host", "entro_last_device_status",
+           "entro_decode_dequant_batched", "entro_decode_dequant_batched_host", "entro_decode_dequant_static",
+           "entro_last_device_status",
            "entro_set_decode_config", "entro_profile_begin", "entro_profile_read", "entro_kernel_launch_count",
            "entro_status_string"]
 
@@ -255,6 +258,18 @@ def entro_decode_dequant_batched_host(descs, io, stream: Optional[torch.cuda.Str
     """descs, io: ctypes arrays of TensorDesc / HostIO of equal length.  Synchronises."""
     _check(lib().entro_decode_dequant_batched_host(descs, io, len(descs), _stream(stream)),
            "entro_decode_dequant_batched_host")
+
+
+def entro_decode_dequant_static(descs, status: Optional[torch.Tensor] = None,
+                                stream: Optional[torch.cuda.Stream] = None) -> None:
+    """The batched decode for callers that cannot allocate device memory: at most
+    STATIC_MAX_TENSORS tensors, no allocator call inside the library.  status: an int32
+    device tensor of one element that receives 0 (clean) or non-zero (corrupt input).
+    Asynchronous."""
+    if isinstance(descs, list):
+        descs = desc_array(descs)
+    sp = None if status is None else _dev(status, torch.int32)
+    _check(lib().entro_decode_dequant_static(descs, len(descs), sp, _stream(stream)), "entro_decode_dequant_static")
 
 
 def entro_last_device_status(stream: Optional[torch.cuda.Stream] = None) -> int:

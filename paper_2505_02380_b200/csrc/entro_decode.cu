@@ -861,6 +861,156 @@ extern "C" entro_status entro_decode_dequant_batched_host(const entro_tensor_des
     return ENTRO_OK;
 }
 
+// ------------------------------------------------------------------ decode without allocation
+
+namespace entro {
+namespace {
+
+// Everything the decode of up to ENTRO_STATIC_MAX_TENSORS tensors needs besides the
+// caller's buffers.  One instance per device that loads the library, held until exit.
+struct StaticScratch {
+    DevTensor tensors[ENTRO_STATIC_MAX_TENSORS];
+    uint32_t item_start[16];          // ENTRO_STATIC_MAX_TENSORS + 1 in use
+    uint32_t control[16];             // [0] work counter, [1] status
+    TensorTables tables[ENTRO_STATIC_MAX_TENSORS];
+};
+static_assert(ENTRO_STATIC_MAX_TENSORS + 1 <= 16, "item_start holds one entry per tensor plus the total");
+
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+// In host code g_static_scratch is only a handle for the runtime; the device address is
+// looked up once per device and kept here.
+struct StaticDevice {
+    StaticScratch* scratch = nullptr;
+    int sm_count = 0;
+    int max_smem_optin = 0;
+    bool ready = false;
+};
+StaticDevice g_static_device[64];
+
+struct StaticUpload {
+    DevTensor tensors[ENTRO_STATIC_MAX_TENSORS];
+    uint32_t item_start[16];
+    int live;
+};
+
+// Copies the descriptors from the kernel's parameter space into the scratch and clears the
+// words that must start at zero (the previous call's contents are still there).
+__global__ void __launch_bounds__(256) static_upload_kernel(const __grid_constant__ StaticUpload up,
+                                                            StaticScratch* __restrict__ sc)
+{
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(up.tensors);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(sc->tensors);
+    const uint32_t words = (uint32_t)up.live * (uint32_t)(sizeof(DevTensor) / 4);
+    for (uint32_t i = threadIdx.x; i < words; i += blockDim.x) dst[i] = src[i];
+    if (threadIdx.x < 16) {
+        sc->item_start[threadIdx.x] = up.item_start[threadIdx.x];
+        sc->control[threadIdx.x] = 0;
+    }
+}
+
+entro_status static_device(StaticDevice** out)
+{
+    int dev = -1;
+    ENTRO_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return ENTRO_ERR_UNSUPPORTED;
+    StaticDevice* sd = &g_static_device[dev];
+    if (!sd->ready) {
+        void* p = nullptr;
+        ENTRO_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        ENTRO_CUDA(cudaDeviceGetAttribute(&sd->sm_count, cudaDevAttrMultiProcessorCount, dev));
+        ENTRO_CUDA(cudaDeviceGetAttribute(&sd->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        sd->scratch = static_cast<StaticScratch*>(p);
+        sd->ready = true;
+    }
+    *out = sd;
+    return ENTRO_OK;
+}
+
+}  // namespace
+}  // namespace entro
+
+extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* descs_host, int ntensors,
+                                                    uint32_t* status_dev, void* cuda_stream)
+{
+    if (ntensors < 0 || (ntensors > 0 && !descs_host)) return ENTRO_ERR_INVALID_ARG;
+    if (status_dev && !aligned(status_dev, 4)) return ENTRO_ERR_INVALID_ARG;
+    int live = 0;
+    for (int i = 0; i < ntensors; ++i) {
+        entro_status st = validate_desc(descs_host[i]);
+        if (st != ENTRO_OK) return st;
+        if (descs_host[i].n) live++;
+    }
+    if (live > ENTRO_STATIC_MAX_TENSORS) return ENTRO_ERR_TOO_MANY_TENSORS;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    Guard g;
+    StaticDevice* sd = nullptr;
+    entro_status st = static_device(&sd);
+    if (st != ENTRO_OK) return st;
+    if (live == 0) {
+        if (status_dev) ENTRO_CUDA(cudaMemsetAsync(status_dev, 0, sizeof(uint32_t), s));
+        return ENTRO_OK;
+    }
+    const DecodeConfig cfg = decode_config();
+
+    StaticUpload up;
+    uint64_t items = 0;
+    uint32_t want_stage = 0;
+    int k = 0;
+    for (int i = 0; i < ntensors; ++i) {
+        const entro_tensor_desc& d = descs_host[i];
+        if (!d.n) continue;
+        DevTensor& t = up.tensors[k];
+        const uint64_t nc = num_chunks(d.n, d.chunk_symbols);
+        t.stream = d.stream_dev;
+        t.offsets = static_cast<const uint64_t*>(d.index_dev);
+        t.sub_len = reinterpret_cast<const uint16_t*>(t.offsets + nc + 1);
+        t.out = static_cast<uint16_t*>(d.out_fp16_dev);
+        t.stream_words = d.stream_words;
+        t.n = d.n;
+        t.chunk_symbols = d.chunk_symbols;
+        t.n_chunks = (uint32_t)nc;
+        t.nsym = (uint32_t)d.cb.nsym;
+        t.scale = d.scale;
+        t.zero_point = d.zero_point;
+        t.pad[0] = t.pad[1] = t.pad[2] = 0;
+        for (int j = 0; j < ENTRO_MAX_SYMBOLS; ++j) t.len[j] = j < d.cb.nsym ? d.cb.len[j] : 0;
+        up.item_start[k] = (uint32_t)items;
+        items += (nc + cfg.chunks_per_item - 1) / cfg.chunks_per_item;
+        if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
+        uint32_t want = d.cb.nsym <= 16 ? (d.chunk_symbols * 3) / 8 : d.chunk_symbols;
+        want = ((want + 127) & ~127u) + 128;
+        if (want > want_stage) want_stage = want;
+        ++k;
+    }
+    for (int j = live; j < 16; ++j) up.item_start[j] = (uint32_t)items;
+    up.live = live;
+
+    StaticScratch* sc = sd->scratch;
+    static_upload_kernel<<<1, 256, 0, s>>>(up, sc);
+    count_launch();
+    ENTRO_CUDA(cudaGetLastError());
+    build_tables_kernel<<<live, 256, 0, s>>>(sc->tensors, cfg.lut_bits, sc->tables, sc->control);
+    count_launch();
+    ENTRO_CUDA(cudaGetLastError());
+    // launch_decode reads only these fields of a workspace; no timing records are taken here
+    Workspace ws;
+    cudaGetDevice(&ws.device);
+    ws.sm_count = sd->sm_count;
+    ws.max_smem_optin = sd->max_smem_optin;
+    ws.control = sc->control;
+    switch (cfg.lut_bits) {
+        case 10: st = launch_decode<10>(&ws, cfg, sc->tensors, live, sc->item_start, (uint32_t)items, sc->tables, want_stage, s); break;
+        case 11: st = launch_decode<11>(&ws, cfg, sc->tensors, live, sc->item_start, (uint32_t)items, sc->tables, want_stage, s); break;
+        case 12: st = launch_decode<12>(&ws, cfg, sc->tensors, live, sc->item_start, (uint32_t)items, sc->tables, want_stage, s); break;
+        default: st = ENTRO_ERR_UNSUPPORTED;
+    }
+    if (st != ENTRO_OK) return st;
+    if (status_dev)
+        ENTRO_CUDA(cudaMemcpyAsync(status_dev, sc->control + 1, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
+    return ENTRO_OK;
+}
+
 extern "C" entro_status entro_set_decode_config(int lut_bits, int warps_per_cta, int ctas_per_sm, int chunks_per_item)
 {
     Guard g;

@@ -171,6 +171,7 @@ extern "C" const char* entro_status_string(entro_status st)
         case ENTRO_ERR_CORRUPT_STREAM: return "stream, index and codebook do not agree";
         case ENTRO_ERR_CUDA: return "a CUDA call failed";
         case ENTRO_ERR_UNSUPPORTED: return "unsupported";
+        case ENTRO_ERR_TOO_MANY_TENSORS: return "more tensors than the static scratch holds";
     }
     return "unknown status";
 }
