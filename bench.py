@@ -127,11 +127,13 @@ def physical_gpu_index(local_rank: int) -> int:
 class DeviceModel:
     """A synthetic model compressed on the device with the library's own offline stages."""
 
-    def __init__(self, wl, E, lut_bytes: int):
+    def __init__(self, wl, E, lut_bits: int):
         self.wl = wl
         self.keep = []           # device buffers
         descs = []
-        total = sum((t.numel + 7) // 8 * 8 for t in wl.tensors)
+        # per-tensor decode tables read from HBM: canonical ranges + the lookup table of the tensor's mode
+        lut_bytes = 1312 + (2048 if wl.bits == 8 else (17 << lut_bits))
+        total = sum((t.numel + 15) // 16 * 16 for t in wl.tensors)
         self.out = torch.empty(total, dtype=torch.float16, device="cuda")
         self.out_slices = []
         self.n = 0
@@ -150,7 +152,7 @@ class DeviceModel:
             enc = E.entro_encode(q, cb, wl.chunk_symbols, stream_words=E.entro_stream_words(counts.tolist(), cb))
             del w, q
             out = self.out[pos:pos + spec.numel]
-            pos += (spec.numel + 7) // 8 * 8
+            pos += (spec.numel + 15) // 16 * 16
             descs.append(E.make_desc(enc.stream, enc.index, spec.numel, wl.chunk_symbols, cb, qp.scale,
                                      qp.zero_point, out))
             self.keep.append(enc)
@@ -309,8 +311,7 @@ def run_reference(args, rank, world):
 # ----------------------------------------------------------------------------- main
 
 def measure(E, wl, args, world, local_rank, rank, peak, with_e2e, with_cpu):
-    lut_bytes = (4 << args.lut_bits) + 1312 + 336
-    model = DeviceModel(wl, E, lut_bytes)
+    model = DeviceModel(wl, E, args.lut_bits)
     ms, launches, kernel_ms, clocks = time_steps(E, model, args.steps, args.warmup, world,
                                                  physical_gpu_index(local_rank))
     ms_step = ms / args.steps
@@ -373,7 +374,7 @@ def main():
     if args.lut_bits or args.warps or args.ctas or args.item:
         E.entro_set_decode_config(args.lut_bits, args.warps, args.ctas, args.item)
     if not args.lut_bits:
-        args.lut_bits = 11
+        args.lut_bits = E.DEFAULT_DECODE_CONFIG[0]
     peak = measured_peak()
 
     wl = pick_workload(args.workload, args.max_layers)

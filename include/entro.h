@@ -205,7 +205,7 @@ entro_status entro_decode_dequant_batched_host(const entro_tensor_desc *descs_ho
  * would stall kernels running on other streams, or where the CUDA allocator must not be
  * entered at all.  This variant calls no allocator: descriptors travel as kernel
  * arguments, and tables, work counter and status word live in an array that is part of the
- * library's device image (about 210 KB, held on every GPU that loads the library until
+ * library's device image (about 575 KB, held on every GPU that loads the library until
  * the process exits).
  *
  *  - At most ENTRO_STATIC_MAX_TENSORS tensors with n > 0 per call; more returns
@@ -233,7 +233,7 @@ entro_status entro_last_device_status(void *cuda_stream);
 
 /*
  * Launch shape of the decode kernel; every argument may be 0 to keep its current value.
- *   lut_bits: bits looked up at once in the shared-memory table (10 .. 12)
+ *   lut_bits: window of the eight-symbol table used for alphabets of <= 16 symbols (10 .. 12)
  *   warps_per_cta: 4 .. 32;  ctas_per_sm: 1 .. 8;  chunks_per_item: chunks a CTA claims at once
  * ENTRO_ERR_INVALID_ARG (nothing changed) if a value is out of range or the shape does
  * not fit in shared memory.

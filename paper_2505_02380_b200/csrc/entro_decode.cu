@@ -3,22 +3,28 @@
 //
 // Work split: a chunk (one segment) is decoded by one warp, each lane owning one of the
 // chunk's 32 sub-blocks.  The lanes' start positions come from a warp prefix sum over the
-// sub-block bit lengths stored in the index.  The warp stages the chunk's bytes into
-// shared memory with one bulk asynchronous copy (the next chunk's bytes are prefetched
-// into L2 meanwhile), every lane then walks its own bits with shared-memory lookup tables
-// whose entries already hold dequantised fp16 values, and the results leave through a
-// swizzled shared-memory tile as coalesced 16-byte-per-lane stores.  A persistent grid
-// pulls work items (runs of chunks of one tensor) from a global counter; the warps of a
-// CTA share out an item's chunks through a shared-memory counter.
+// sub-block bit lengths stored in the index.  A persistent grid pulls work items (runs of
+// chunks of one tensor) from a global counter; the warps of a CTA share out an item's
+// chunks through a shared-memory counter.  Every warp runs a three-deep pipeline: while it
+// decodes chunk i, the bytes of chunk i + 1 are arriving in its shared-memory ring through
+// one bulk asynchronous copy, and the index entries of chunk i + 2 are on their way into
+// registers.  Lanes walk their bits with lookup tables whose entries already hold the
+// dequantised fp16 values and store 16 values (32 bytes, one full sector) at a time.
 //
-// Tables per tensor (built by build_tables_kernel, cached in shared memory per CTA):
-//   lut1  2^K entries indexed by the next K stream bits.
-//         alphabets > 16 symbols: one symbol per entry,  value << 16 | length, or kEscFlag
-//         alphabets <= 16 symbols: four symbols per entry, nibbles << 8 | total length, or
-//         kQuadEscFlag; the fp16 values come from a 256-entry table of symbol pairs
-//   lut2  second level for codes longer than K (single-symbol mode): indexed by
-//         (window - t2) >> shift2, same entry format
-//   aux   canonical ranges per length for whatever neither table resolves
+// Tables per tensor (built by build_tables_kernel, copied into shared memory per CTA):
+//   alphabets > 16 symbols, one symbol per lookup.  Canonical codes grow longer towards the
+//     all-ones end of the code space, so the table is indexed like a floating-point number:
+//     by the count of leading one bits of the window and the kExpBits bits after the first
+//     zero.  Converting the inverted window to float yields exactly that index (exponent |
+//     top mantissa bits) in one instruction, and 32 << kExpBits cells resolve every code
+//     whose length is at most leading ones + 1 + kExpBits - on bell-shaped histograms all
+//     of them, where a direct table of the same size would miss the tail.  The shared-
+//     memory copy is replicated 32 times, cell-major, so lane l only ever touches bank l:
+//     no bank conflicts whatever the data.
+//   alphabets <= 16 symbols, eight symbols per lookup: the next K bits index a table of
+//     16-byte entries (eight fp16 values) and a byte table (bits used, 0 = no eight whole
+//     codes in K bits).
+//   aux   canonical ranges per length, for whatever the tables do not resolve.
 #include <cuda_fp16.h>
 
 #include "entro_internal.h"
@@ -26,11 +32,18 @@
 namespace entro {
 namespace {
 
-constexpr int kTile = 32;                 // symbols per lane between two flushes of the output tile
-constexpr int kTileBytes = 32 * kTile * 2;
-constexpr int kUnits = kTile / 8;         // 16-byte units per tile row
-constexpr uint32_t kWaitTries = 1u << 16; // bound on polling a bulk copy (each try may suspend)
-constexpr uint32_t kLut2MaxBits = 20;     // longest code the second level resolves
+extern __shared__ __align__(1024) unsigned char smem[];
+
+constexpr uint32_t kNone = 0xffffffffu;
+constexpr uint32_t kWaitTries = 1u << 16;  // bound on polling a bulk copy (each try may suspend)
+constexpr uint32_t kEscLen = 0x40u;        // length field of a cell the table cannot resolve
+constexpr uint32_t kOverRead = 2064;       // a lane fed garbage may read this far past its chunk's bytes
+
+// Shared-memory bytes of the lookup tables for a K-bit eight-symbol table.
+__host__ __device__ constexpr uint32_t lut_bytes(int K)
+{
+    return (17u << K) > (uint32_t)kExpEntries * 128u ? (17u << K) : (uint32_t)kExpEntries * 128u;
+}
 
 // ------------------------------------------------------------------ table construction
 
@@ -69,6 +82,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     if (tid == 0) {
         unsigned long long code = 0;   // reaches 2^32 after the last length of a complete code
         uint32_t off = 0, max_len = 0;
+        float mean_len = 0.f;          // sum over codes of len * 2^-len: the code's own estimate of its mean length
         aux.limit[0] = 0;
         aux.first_code[0] = 0;
         aux.offset[0] = 0;
@@ -80,27 +94,13 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
             off += count[k];
             aux.limit[k] = code << (32 - k);
             if (count[k]) max_len = k;
+            mean_len += (float)count[k] * (float)k * exp2f(-(float)k);
         }
         aux.max_len = max_len;
-        aux.quad = T.nsym <= 16 ? 1u : 0u;
-        // second level: windows at or above the end of the codes that fit the first level
-        aux.t2 = 0;
-        aux.shift2 = 0;
-        aux.n2 = 0;
-        const unsigned long long t2 = aux.limit[lut_bits];
-        if (!aux.quad && max_len > (uint32_t)lut_bits && t2 < (1ull << 32)) {
-            uint32_t bits = max_len < kLut2MaxBits ? max_len : kLut2MaxBits;
-            for (; bits > (uint32_t)lut_bits; --bits) {
-                unsigned long long n = ((1ull << 32) - t2 + (1ull << (32 - bits)) - 1) >> (32 - bits);
-                if (n <= (unsigned long long)kLut2Entries) {
-                    aux.t2 = (uint32_t)t2;
-                    aux.shift2 = 32 - bits;
-                    aux.n2 = (uint32_t)n;
-                    break;
-                }
-            }
-        }
-        aux.pad[0] = aux.pad[1] = aux.pad[2] = 0;
+        aux.oct = T.nsym <= 16 ? 1u : 0u;
+        // four lookups per window refill while their lengths almost always sum to <= 32 bits
+        aux.group = mean_len <= 4.75f ? 4u : 2u;
+        aux.pad = 0;
     }
     __syncthreads();
     if (l) {
@@ -117,37 +117,54 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     }
     __syncthreads();
 
-    const uint32_t entries = 1u << lut_bits;
-    if (aux.quad) {
+    if (aux.oct) {
+        const uint32_t entries = 1u << lut_bits;
         for (uint32_t i = tid; i < entries; i += 256) {
             uint32_t window = i << (32 - lut_bits);
-            uint32_t used = 0, nibbles = 0;
+            uint32_t used = 0;
+            uint32_t v[8];
             bool ok = true;
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < 8; ++k) {
                 uint32_t sl;
                 uint32_t sym = range_decode(aux, window, (uint32_t)lut_bits - used, sl);
                 if (sl == 0) {
                     ok = false;
                     break;
                 }
-                nibbles |= sym << (4 * k);
+                v[k] = aux.val[sym];
                 used += sl;
                 window <<= sl;   // sl <= lut_bits < 32
             }
-            out.lut1[i] = ok ? ((nibbles << 8) | used) : kQuadEscFlag;
+            uint4 e = make_uint4(0u, 0u, 0u, 0u);
+            if (ok) e = make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
+            out.oct_val[i] = e;
+            out.oct_len[i] = ok ? (uint8_t)used : (uint8_t)0;
         }
-        // fp16 values of a pair of symbols: low nibble first
-        out.lut2[tid] = (uint32_t)aux.val[tid & 15] | ((uint32_t)aux.val[tid >> 4] << 16);
     } else {
-        for (uint32_t i = tid; i < entries; i += 256) {
-            uint32_t sl;
-            uint32_t sym = range_decode(aux, i << (32 - lut_bits), (uint32_t)lut_bits, sl);
-            out.lut1[i] = sl ? (((uint32_t)aux.val[sym] << 16) | sl) : kEscFlag;
-        }
-        for (uint32_t i = tid; i < aux.n2; i += 256) {
-            uint32_t sl;
-            uint32_t sym = range_decode(aux, aux.t2 + (i << aux.shift2), 32 - aux.shift2, sl);
-            out.lut2[i] = sl ? (((uint32_t)aux.val[sym] << 16) | sl) : kEscFlag;
+        // cell (e5, mant): windows that start with r ones and a zero, followed by the bits ~mant
+        for (uint32_t i = tid; i < (uint32_t)kExpEntries; i += 256) {
+            const uint32_t e5 = i >> kExpBits, mant = i & ((1u << kExpBits) - 1u);
+            const uint32_t r = (30u - e5) & 31u;
+            const uint32_t avail = 31u - r;                               // window bits after the zero
+            const uint32_t mb = avail < (uint32_t)kExpBits ? avail : (uint32_t)kExpBits;
+            uint32_t entry = kEscLen;
+            if ((mant & ((1u << (kExpBits - mb)) - 1u)) == 0u) {          // else no window maps here
+                const uint32_t mt = mant >> (kExpBits - mb);
+                const uint32_t vb = ~mt & ((1u << mb) - 1u);
+                const uint32_t ones = r ? (0xffffffffu << (32u - r)) : 0u;
+                const uint32_t v_lo = ones | (vb << (avail - mb));
+                uint32_t sl;
+                uint32_t sym = range_decode(aux, v_lo, aux.max_len, sl);
+                bool ok = sl != 0 && sl <= r + 1u + mb;
+                if (ok && i == 0) {
+                    // the window of 32 ones converts to 0.0f and lands in this cell as well
+                    uint32_t sl1;
+                    uint32_t sym1 = range_decode(aux, 0xffffffffu, aux.max_len, sl1);
+                    ok = sl1 == sl && sym1 == sym;
+                }
+                if (ok) entry = ((uint32_t)aux.val[sym] << 16) | sl;
+            }
+            out.exp_lut[i] = entry;
         }
     }
     const uint32_t* src = reinterpret_cast<const uint32_t*>(&aux);
@@ -157,42 +174,70 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
 
 // ------------------------------------------------------------------ bit reader
 
-// 64-bit window, left-justified: `nb` valid bits, the rest zero.  `next` is the index of
-// the next 32-bit word to pull in.
-struct Reader {
+// 64-bit window, left-justified: `nb` valid bits, zeros below.  With kInv the window holds
+// the complement of the stream bits (what the exponent-indexed table wants).
+struct Win {
+    uint32_t hi, lo;
+    int nb;
+    const uint32_t* next;     // shared memory: next word to pull in
+};
+
+template <bool kInv>
+__device__ __forceinline__ void win_init(Win& r, const uint32_t* words, uint32_t bit_pos)
+{
+    const uint32_t* p = words + (bit_pos >> 5);
+    const uint32_t bit = bit_pos & 31u;
+    uint32_t w0 = p[0], w1 = p[1];
+    if (kInv) {
+        w0 = ~w0;
+        w1 = ~w1;
+    }
+    r.hi = __funnelshift_l(w1, w0, bit);
+    r.lo = w1 << bit;
+    r.nb = 64 - (int)bit;
+    r.next = p + 2;
+}
+
+// Top up to more than 32 valid bits.  With nb <= 32 the low word is empty.
+template <bool kInv>
+__device__ __forceinline__ void win_refill(Win& r)
+{
+    if (r.nb <= 32) {
+        uint32_t w = *r.next++;
+        if (kInv) w = ~w;
+        r.hi |= __funnelshift_rc(w, 0u, (uint32_t)r.nb);
+        r.lo = __funnelshift_lc(0u, w, (uint32_t)(32 - r.nb));
+        r.nb += 32;
+    }
+}
+
+// Drop n bits, 0 <= n <= 32.
+__device__ __forceinline__ void win_skip(Win& r, uint32_t n)
+{
+    r.hi = __funnelshift_lc(r.lo, r.hi, n);
+    r.lo = __funnelshift_lc(0u, r.lo, n);
+    r.nb -= (int)n;
+}
+
+__device__ __forceinline__ uint32_t win_used_bits(const Win& r, const uint32_t* words, uint32_t bit_pos)
+{
+    return (uint32_t)(r.next - words) * 32u - (uint32_t)r.nb - bit_pos;
+}
+
+// The same over global memory, word by word, for chunks that are not staged.
+struct GlobalWin {
     uint32_t hi, lo;
     int nb;
     uint32_t next;
-};
-
-struct SmemSource {
-    const uint32_t* words;
-    uint32_t last;            // highest index that may be read
-    __device__ __forceinline__ uint32_t get(uint32_t i) const { return words[min(i, last)]; }
-};
-
-struct GlobalSource {
     const uint32_t* words;
     uint64_t count;           // words readable from `words`
     __device__ __forceinline__ uint32_t get(uint32_t i) const { return i < count ? __ldg(words + i) : 0u; }
 };
 
-template <class Src>
-__device__ __forceinline__ void reader_init(Reader& r, const Src& src, uint32_t word, uint32_t bit)
-{
-    uint32_t w0 = src.get(word), w1 = src.get(word + 1);
-    r.hi = __funnelshift_l(w1, w0, bit);          // bit < 32
-    r.lo = __funnelshift_l(0u, w1, bit);
-    r.nb = 64 - (int)bit;
-    r.next = word + 2;
-}
-
-// Top up to more than 32 valid bits.  With nb <= 32 the low word is empty.
-template <class Src>
-__device__ __forceinline__ void reader_refill(Reader& r, const Src& src)
+__device__ __forceinline__ void gwin_refill(GlobalWin& r)
 {
     if (r.nb <= 32) {
-        uint32_t w = src.get(r.next);
+        uint32_t w = r.get(r.next);
         r.next++;
         r.hi |= __funnelshift_rc(w, 0u, (uint32_t)r.nb);
         r.lo = __funnelshift_lc(0u, w, (uint32_t)(32 - r.nb));
@@ -200,28 +245,19 @@ __device__ __forceinline__ void reader_refill(Reader& r, const Src& src)
     }
 }
 
-// Drop `n` bits, 0 <= n <= 32.
-__device__ __forceinline__ void reader_skip(Reader& r, uint32_t n)
+// ------------------------------------------------------------------ lookups
+
+// Cell of the exponent-indexed table for an inverted window, in this lane's copy.
+// lane4 = 4 * lane.  The table starts at the beginning of shared memory.
+__device__ __forceinline__ uint32_t exp_lookup(uint32_t lane4, uint32_t inv_window)
 {
-    if (n >= 32) {
-        r.hi = r.lo;
-        r.lo = 0;
-    } else {
-        r.hi = __funnelshift_l(r.lo, r.hi, n);
-        r.lo <<= n;
-    }
-    r.nb -= (int)n;
+    const uint32_t fb = __float_as_uint(__uint2float_rz(inv_window));
+    const uint32_t a = ((fb >> (16 - kExpBits)) & (((32u << kExpBits) - 1u) << 7)) | lane4;
+    return *reinterpret_cast<const uint32_t*>(smem + a);
 }
 
-struct Tables {
-    const uint32_t* lut1;      // shared
-    const uint32_t* lut2;      // shared
-    const DecodeAux* aux;      // shared
-    uint32_t* status;          // global
-};
-
-// One symbol from a full 32-bit window by the canonical ranges; a pattern that is no
-// codeword is flagged and dropped as a single bit.  Entry format: value << 16 | length.
+// One symbol from a full 32-bit window (true stream bits) by the canonical ranges; a pattern
+// that is no codeword is flagged and dropped as a single bit.  -> value << 16 | length.
 __device__ __noinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32_t window, uint32_t* status)
 {
     uint32_t len;
@@ -233,84 +269,62 @@ __device__ __noinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32_t 
     return ((uint32_t)aux->val[sym] << 16) | len;
 }
 
-// A symbol the first level could not resolve: second level, then the ranges.
-__device__ __forceinline__ uint32_t decode_long(const Tables& tb, uint32_t window)
-{
-    const DecodeAux* aux = tb.aux;
-    if (window >= aux->t2) {
-        uint32_t i = (window - aux->t2) >> aux->shift2;
-        if (i < aux->n2) {
-            uint32_t e = tb.lut2[i];
-            if (!(e & kEscFlag)) return e;
-        }
-    }
-    return decode_by_range(aux, window, tb.status);
-}
-
-// One symbol, any tensor mode (used off the fast path).
-template <int K>
-__device__ __forceinline__ uint32_t decode_one(const Tables& tb, uint32_t window)
-{
-    if (tb.aux->quad) return decode_by_range(tb.aux, window, tb.status);
-    uint32_t e = tb.lut1[window >> (32 - K)];
-    if (e & kEscFlag) e = decode_long(tb, window);
-    return e;
-}
-
-// Out-of-line repair of a pair of lookups in which at least one hit an escape entry.  On
-// entry the window stands before the first unresolved symbol (escape entries have length
-// 0): before symbol 0 if e0 is an escape, else before symbol 1.
-struct PairFix {
-    Reader r;
-    uint32_t e0, e1;
+struct SlowOut {
+    Win r;
+    uint32_t e[4];
 };
 
-template <int K>
-__device__ __noinline__ PairFix redo_pair(const uint32_t* lut1, const uint32_t* lut2, const DecodeAux* aux,
-                                         uint32_t* status, const uint32_t* words, uint32_t last, Reader r,
-                                         uint32_t e0)
+// A group of `count` (2 or 4) symbols of an 8-bit alphabet that the fast path gave up on:
+// symbol by symbol, any code length.  -> values in the high halves of e[].
+__device__ __noinline__ SlowOut single_slow(const DecodeAux* aux, uint32_t* status, uint32_t lane4, Win r, int count)
 {
-    Tables tb{lut1, lut2, aux, status};
-    SmemSource src{words, last};
-    PairFix f;
-    if (e0 & kEscFlag) {
-        reader_refill(r, src);
-        e0 = decode_long(tb, r.hi);
-        reader_skip(r, e0 & 0xffu);
+    SlowOut o;
+    for (int k = 0; k < 4; ++k) o.e[k] = 0;
+    for (int k = 0; k < count; ++k) {
+        win_refill<true>(r);
+        uint32_t e = exp_lookup(lane4, r.hi);
+        if ((e & 0xffffu) > 32u) e = decode_by_range(aux, ~r.hi, status);
+        win_skip(r, e & 0xffffu);
+        o.e[k] = e;
     }
-    reader_refill(r, src);
-    uint32_t e1 = lut1[r.hi >> (32 - K)];
-    if (e1 & kEscFlag) e1 = decode_long(tb, r.hi);
-    reader_skip(r, e1 & 0xffu);
-    f.r = r;
-    f.e0 = e0;
-    f.e1 = e1;
-    return f;
+    o.r = r;
+    return o;
 }
 
-// The same for a four-symbol entry: the four symbols one by one.  Returns the two pair
-// bytes (symbols 0,1 and 2,3) in e0, e1.
-__device__ __noinline__ PairFix redo_quad(const DecodeAux* aux, uint32_t* status, const uint32_t* words,
-                                         uint32_t last, Reader r)
+struct OctOut {
+    Win r;
+    uint4 v;
+};
+
+// Eight symbols of a 4-bit alphabet whose codes do not fit the table's window.
+__device__ __noinline__ OctOut oct_slow(const DecodeAux* aux, uint32_t* status, Win r)
 {
-    SmemSource src{words, last};
-    PairFix f;
-    uint32_t nib = 0;
-    for (int k = 0; k < 4; ++k) {
-        reader_refill(r, src);
-        uint32_t len;
-        uint32_t sym = range_decode(*aux, r.hi, aux->max_len, len);
-        if (len == 0) {
-            atomicOr(status, kStatCorrupt);
-            len = 1;
-        }
-        reader_skip(r, len);
-        nib |= (sym & 15u) << (4 * k);
+    uint32_t h[8];
+    for (int k = 0; k < 8; ++k) {
+        win_refill<false>(r);
+        uint32_t e = decode_by_range(aux, r.hi, status);
+        win_skip(r, e & 0xffu);
+        h[k] = e >> 16;
     }
-    f.r = r;
-    f.e0 = nib & 0xffu;
-    f.e1 = nib >> 8;
-    return f;
+    OctOut o;
+    o.r = r;
+    o.v = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+    return o;
+}
+
+// ------------------------------------------------------------------ output
+
+// 16 fp16 values (32 bytes) of this lane's row, write-once data.
+__device__ __forceinline__ void store16(uint16_t* dst, const uint32_t (&v)[8], bool aligned32)
+{
+    if (aligned32) {
+        asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(v[0]), "r"(v[1]), "r"(v[2]),
+                     "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                     : "memory");
+    } else {
+        __stcs(reinterpret_cast<uint4*>(dst), make_uint4(v[0], v[1], v[2], v[3]));
+        __stcs(reinterpret_cast<uint4*>(dst) + 1, make_uint4(v[4], v[5], v[6], v[7]));
+    }
 }
 
 // ------------------------------------------------------------------ bulk copy + mbarrier
@@ -328,11 +342,6 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
-}
-
-__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 
 // Bounded wait for phase `parity` of the barrier; false if the bound ran out.  Each try may
@@ -356,30 +365,124 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 // ------------------------------------------------------------------ one chunk
 
 struct WarpCtx {
-    Tables tb;
-    uint32_t* stage;           // shared, this warp's compressed bytes
-    uint4* tile;               // shared, this warp's output tile
-    uint32_t bar;              // shared address of this warp's mbarrier
+    const DecodeAux* aux;      // shared
+    uint32_t* status;          // global
+    unsigned char* stage;      // shared: this warp's ring for compressed bytes
     uint32_t stage_bytes;
-    uint32_t phase;
-    bool dead;                 // a bulk copy never completed: stop using the stage buffer
+    uint32_t bar;              // shared address of this warp's two mbarriers
+    uint32_t tickets;          // bulk copies issued so far
+    bool dead;                 // a bulk copy never completed: stop staging
 };
 
-// Byte range of the stream that decoding chunk c touches, or false if the index does not
-// describe a range inside the stream buffer.  A lane may look 12 bytes past its end.
-__device__ __forceinline__ bool chunk_range(const DevTensor& T, uint64_t off0, uint64_t off1, uint64_t& byte0,
-                                            uint64_t& byte1)
+// Chunk whose index entries have been requested from global memory.
+struct Pending {
+    uint32_t c;                // chunk within the tensor, or kNone
+    uint64_t off;              // even lanes: offsets[c], odd lanes: offsets[c + 1]
+    uint32_t bits;             // this lane's sub-block length
+};
+
+enum : uint32_t { kStaged = 0, kGeneral = 1, kSkip = 2 };
+
+// Chunk ready to decode.
+struct Ready {
+    uint32_t c;                // or kNone
+    uint32_t kind;
+    uint32_t pos;              // staged: this lane's first bit within the staged bytes; general: bits before it in the chunk
+    uint32_t my_bits;
+    uint32_t at;               // staged: byte offset in the ring
+    uint32_t bytes;            // staged: bytes copied
+    uint32_t ticket;           // staged: which barrier and phase
+    uint32_t src_lo, src_hi;   // staged: byte offset in the stream, until the copy has been issued
+    bool issued;
+};
+
+__device__ __forceinline__ Pending fetch_index(const DevTensor& T, uint32_t c, uint32_t lane)
 {
-    byte0 = (off0 >> 3) & ~15ull;
-    byte1 = ((off1 >> 3) + 13 + 15) & ~15ull;
-    return off1 >= off0 && off1 - off0 <= 32ull * 65535ull && byte1 <= T.stream_words * 4;
+    Pending p;
+    p.c = c;
+    p.off = 0;
+    p.bits = 0;
+    if (c != kNone) {
+        p.off = T.offsets[c + (lane & 1u)];
+        p.bits = T.sub_len[(uint64_t)c * kSubBlocks + lane];
+    }
+    return p;
 }
 
-// General path: any symbol count per lane, words fetched straight from global memory,
-// scalar stores.  Used for the ragged last chunk of a tensor and for chunks whose bytes do
-// not fit the stage buffer.
-template <int K>
-__device__ __noinline__ void decode_chunk_general(Tables tb, const DevTensor& T, uint32_t c, uint64_t off0,
+__device__ __forceinline__ void issue_copy(WarpCtx& cx, const DevTensor& T, Ready& r, uint32_t lane)
+{
+    if (lane == 0) {
+        const uint64_t byte0 = ((uint64_t)r.src_hi << 32) | r.src_lo;
+        bulk_load(smem_addr(cx.stage + r.at), reinterpret_cast<const char*>(T.stream) + byte0, r.bytes,
+                  cx.bar + 8u * (r.ticket & 1u));
+    }
+    r.issued = true;
+}
+
+// Turn a fetched index entry into a decodable chunk: lane start positions by prefix sum,
+// consistency checks, a place in the ring next to `prev` (the chunk decoded before this
+// one, possibly still undecoded), and the bulk copy if that place is free already.
+__device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, const Pending& p, const Ready& prev,
+                                         uint32_t lane)
+{
+    Ready r;
+    r.c = p.c;
+    r.kind = kSkip;
+    r.pos = r.at = r.bytes = r.ticket = r.src_lo = r.src_hi = 0;
+    r.my_bits = p.bits;
+    r.issued = false;
+    if (p.c == kNone) return r;
+    const uint64_t off0 = __shfl_sync(0xffffffffu, p.off, 0);
+    const uint64_t off1 = __shfl_sync(0xffffffffu, p.off, 1);
+    uint32_t incl = p.bits;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= (uint32_t)d) incl += t;
+    }
+    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+    const uint32_t excl = incl - p.bits;
+    // bytes the chunk's decode touches: from the 16-byte boundary below its first bit to
+    // 13 bytes past its last (a window looks ahead), rounded up to 16
+    const uint64_t byte0 = (off0 >> 3) & ~15ull;
+    const uint64_t byte1 = ((off1 >> 3) + 13 + 15) & ~15ull;
+    if (off1 < off0 || off1 - off0 != (uint64_t)total || byte1 > T.stream_words * 4) {
+        if (lane == 0) atomicOr(cx.status, kStatCorrupt);
+        return r;
+    }
+    const uint32_t sub = T.chunk_symbols / kSubBlocks;
+    const bool full = (uint64_t)(p.c + 1) * T.chunk_symbols <= T.n;
+    const uint64_t bytes = byte1 - byte0;
+    if (!full || (sub & 15u) || bytes > cx.stage_bytes || cx.dead) {
+        r.kind = kGeneral;
+        r.pos = excl;
+        return r;
+    }
+    r.kind = kStaged;
+    r.bytes = (uint32_t)bytes;
+    r.pos = (uint32_t)(off0 - byte0 * 8) + excl;
+    r.src_lo = (uint32_t)byte0;
+    r.src_hi = (uint32_t)(byte0 >> 32);
+    r.ticket = cx.tickets++;
+    // ring placement: behind the previous chunk's bytes, else at the start if that does not
+    // overlap them, else at the start once the previous chunk has been decoded
+    bool now = true;
+    if (prev.c != kNone && prev.kind == kStaged) {
+        const uint32_t end = prev.at + prev.bytes;
+        if (end + r.bytes <= cx.stage_bytes) r.at = end;
+        else if (r.bytes <= prev.at) r.at = 0;
+        else {
+            r.at = 0;
+            now = false;
+        }
+    }
+    if (now) issue_copy(cx, T, r, lane);
+    return r;
+}
+
+// Any symbol count per lane, words fetched straight from global memory, scalar stores: the
+// ragged last chunk of a tensor, odd chunk sizes, chunks larger than the ring.
+__device__ __noinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t* status, const DevTensor& T, uint32_t c,
                                                   uint32_t excl, uint32_t my_bits, uint32_t lane)
 {
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
@@ -387,168 +490,136 @@ __device__ __noinline__ void decode_chunk_general(Tables tb, const DevTensor& T,
     const uint64_t chunk_syms = min((uint64_t)T.chunk_symbols, T.n - chunk_first);
     const uint64_t lane_first = (uint64_t)lane * sub;
     const uint32_t cnt = lane_first >= chunk_syms ? 0u : (uint32_t)min((uint64_t)sub, chunk_syms - lane_first);
-    const uint64_t pos = off0 + excl;
+    const uint64_t pos = T.offsets[c] + excl;
     const uint64_t word0 = pos >> 5;
-    GlobalSource src{T.stream + word0, word0 < T.stream_words ? T.stream_words - word0 : 0ull};
-    Reader r;
-    reader_init(r, src, 0u, (uint32_t)(pos & 31));
+    GlobalWin r;
+    r.words = T.stream + word0;
+    r.count = word0 < T.stream_words ? T.stream_words - word0 : 0ull;
+    const uint32_t bit = (uint32_t)(pos & 31);
+    const uint32_t w0 = r.get(0), w1 = r.get(1);
+    r.hi = __funnelshift_l(w1, w0, bit);
+    r.lo = w1 << bit;
+    r.nb = 64 - (int)bit;
+    r.next = 2;
+    const bool oct = aux->oct != 0;
     uint16_t* out = T.out + chunk_first + lane_first;
     for (uint32_t i = 0; i < cnt; ++i) {
-        reader_refill(r, src);
-        uint32_t e = decode_one<K>(tb, r.hi);
-        reader_skip(r, e & 0xffu);
+        gwin_refill(r);
+        uint32_t e = kEscLen;
+        if (!oct) e = exp_lookup(lane * 4u, ~r.hi);
+        if ((e & 0xffffu) > 32u) e = decode_by_range(aux, r.hi, status);
+        const uint32_t n = e & 0xffffu;
+        r.hi = __funnelshift_lc(r.lo, r.hi, n);
+        r.lo = __funnelshift_lc(0u, r.lo, n);
+        r.nb -= (int)n;
         out[i] = (uint16_t)(e >> 16);
     }
-    const uint64_t used = ((uint64_t)r.next << 5) - (uint64_t)r.nb - (pos & 31);
-    if (used != my_bits) atomicOr(tb.status, kStatCorrupt);
+    const uint64_t used = ((uint64_t)r.next << 5) - (uint64_t)r.nb - bit;
+    if (used != my_bits) atomicOr(status, kStatCorrupt);
 }
 
-// Flush the warp's output tile: each instruction writes (32 / kUnits) rows of kTile * 2
-// contiguous bytes; row r of the tile belongs to lane r's sub-block.
-__device__ __forceinline__ void flush_tile(const uint4* tile, uint16_t* out_chunk, uint32_t sub, uint32_t t0,
-                                           uint32_t lane)
+// 8-bit alphabets: G lookups per refill.  The lookups of a group read the window at the
+// running sum of the lengths before them; the group stands if that sum ends at 32 bits or
+// less (the refill guarantees 33), which also rules out an unresolved cell (length 64).
+template <int G>
+__device__ __forceinline__ void rows_single(Win& r, const WarpCtx& cx, uint32_t lane4, uint16_t* out_row, uint32_t sub,
+                                            bool aligned32)
 {
+    for (uint32_t t0 = 0; t0 < sub; t0 += 16) {
+        uint32_t pk[8];
 #pragma unroll
-    for (int i = 0; i < kUnits; ++i) {
-        const uint32_t row = i * (32 / kUnits) + lane / kUnits;
-        const uint32_t unit = lane % kUnits;
-        const uint32_t swz = (row / (8 / kUnits)) % kUnits;
-        uint4 v = tile[row * kUnits + (unit ^ swz)];
-        uint4* dst = reinterpret_cast<uint4*>(out_chunk + (uint64_t)row * sub + t0) + unit;
-        __stcs(dst, v);
+        for (int g = 0; g < 16 / G; ++g) {
+            win_refill<true>(r);
+            uint32_t e[4];
+            e[0] = exp_lookup(lane4, r.hi);
+            uint32_t s = e[0];
+#pragma unroll
+            for (int k = 1; k < G; ++k) {
+                e[k] = exp_lookup(lane4, __funnelshift_l(r.lo, r.hi, s));   // shift = low 5 bits of s
+                s += e[k];
+            }
+            const uint32_t S = s & 0xffffu;
+            if (__builtin_expect(S > 32u, 0)) {
+                SlowOut o = single_slow(cx.aux, cx.status, lane4, r, G);
+                r = o.r;
+#pragma unroll
+                for (int k = 0; k < G; ++k) e[k] = o.e[k];
+            } else {
+                win_skip(r, S);
+            }
+#pragma unroll
+            for (int k = 0; k < G; k += 2) pk[(g * G + k) / 2] = __byte_perm(e[k], e[k + 1], 0x7632);
+        }
+        store16(out_row + t0, pk, aligned32);
     }
 }
 
-// Fast path: a full chunk whose bytes are staged in shared memory.
+// 4-bit alphabets: eight symbols per lookup.
 template <int K>
-__device__ __forceinline__ void decode_chunk_staged(WarpCtx& cx, const DevTensor& T, uint32_t c, uint64_t off0,
-                                                    uint64_t byte0, uint32_t copy_bytes, uint32_t excl,
-                                                    uint32_t my_bits, uint32_t lane)
+__device__ __forceinline__ void rows_oct(Win& r, const WarpCtx& cx, uint16_t* out_row, uint32_t sub, bool aligned32)
 {
-    const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    if (lane == 0)
-        bulk_load(smem_addr(cx.stage), reinterpret_cast<const char*>(T.stream) + byte0, copy_bytes, cx.bar);
-    bool ok = mbar_wait(cx.bar, cx.phase);
-    ok = __all_sync(0xffffffffu, ok);
-    if (!ok) {
-        if (lane == 0) atomicOr(cx.tb.status, kStatTimeout);
-        cx.dead = true;
+    for (uint32_t t0 = 0; t0 < sub; t0 += 16) {
+        uint32_t pk[8];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            win_refill<false>(r);
+            const uint32_t idx = r.hi >> (32 - K);
+            uint4 v = *reinterpret_cast<const uint4*>(smem + idx * 16u);
+            const uint32_t n = *(smem + (16u << K) + idx);
+            if (__builtin_expect(n == 0u, 0)) {
+                OctOut o = oct_slow(cx.aux, cx.status, r);
+                r = o.r;
+                v = o.v;
+            } else {
+                r.hi = __funnelshift_l(r.lo, r.hi, n);
+                r.lo <<= n;
+                r.nb -= (int)n;
+            }
+            pk[4 * h] = v.x;
+            pk[4 * h + 1] = v.y;
+            pk[4 * h + 2] = v.z;
+            pk[4 * h + 3] = v.w;
+        }
+        store16(out_row + t0, pk, aligned32);
+    }
+}
+
+template <int K>
+__device__ __forceinline__ void decode_ready(WarpCtx& cx, const DevTensor& T, Ready& r, uint32_t lane)
+{
+    if (r.kind == kSkip) return;
+    if (r.kind == kStaged) {
+        if (!r.issued) issue_copy(cx, T, r, lane);
+        bool ok = mbar_wait(cx.bar + 8u * (r.ticket & 1u), (r.ticket >> 1) & 1u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) {
+            if (lane == 0) atomicOr(cx.status, kStatTimeout);
+            cx.dead = true;
+            // fall back to global memory; this lane's bits before it: pos minus the chunk's first bit
+            const uint32_t first = __shfl_sync(0xffffffffu, r.pos, 0);
+            r.kind = kGeneral;
+            r.pos -= first;
+        }
+    }
+    if (r.kind == kGeneral) {
+        decode_chunk_general(cx.aux, cx.status, T, r.c, r.pos, r.my_bits, lane);
         return;
     }
-    cx.phase ^= 1u;
-
-    const SmemSource src{cx.stage, copy_bytes / 4 - 1};
-    const uint32_t pos = (uint32_t)(off0 - byte0 * 8) + excl;     // bit position inside the stage buffer
-    Reader r;
-    reader_init(r, src, pos >> 5, pos & 31);
-
-    const uint32_t* lut1 = cx.tb.lut1;
-    // tile row = lane, 16-byte units swizzled so that both the per-lane writes and the
-    // row-wise reads of the flush touch every bank once
-    const uint32_t row_swz = (lane / (8 / kUnits)) % kUnits;
-    uint4* my_row = cx.tile + lane * kUnits;
-    uint16_t* out_chunk = T.out + (uint64_t)c * T.chunk_symbols;
-
-    if (cx.tb.aux->quad) {
-        const uint32_t* pair_val = cx.tb.lut2;
-        for (uint32_t t0 = 0; t0 < sub; t0 += kTile) {
-#pragma unroll 1
-            for (int g = 0; g < kUnits; ++g) {
-                uint32_t packed[4];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    reader_refill(r, src);
-                    uint32_t e = lut1[r.hi >> (32 - K)];
-                    r.hi = __funnelshift_l(r.lo, r.hi, e);
-                    r.lo = __funnelshift_l(0u, r.lo, e);
-                    r.nb -= (int)(e & 0xffu);
-                    uint32_t b0 = __byte_perm(e, 0u, 0x4441);     // byte 1: symbols 0, 1
-                    uint32_t b1 = __byte_perm(e, 0u, 0x4442);     // byte 2: symbols 2, 3
-                    if (__builtin_expect(e & kQuadEscFlag, 0)) {
-                        PairFix f = redo_quad(cx.tb.aux, cx.tb.status, src.words, src.last, r);
-                        r = f.r;
-                        b0 = f.e0;
-                        b1 = f.e1;
-                    }
-                    packed[2 * h] = pair_val[b0];
-                    packed[2 * h + 1] = pair_val[b1];
-                }
-                my_row[g ^ row_swz] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-            }
-            __syncwarp();
-            flush_tile(cx.tile, out_chunk, sub, t0, lane);
-            __syncwarp();
-        }
+    const uint32_t sub = T.chunk_symbols / kSubBlocks;
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(cx.stage + r.at);
+    uint16_t* out_row = T.out + (uint64_t)r.c * T.chunk_symbols + (uint64_t)lane * sub;
+    const bool aligned32 = (reinterpret_cast<uintptr_t>(T.out) & 31u) == 0;
+    Win w;
+    if (cx.aux->oct) {
+        win_init<false>(w, words, r.pos);
+        rows_oct<K>(w, cx, out_row, sub, aligned32);
     } else {
-        for (uint32_t t0 = 0; t0 < sub; t0 += kTile) {
-#pragma unroll 1
-            for (int g = 0; g < kUnits; ++g) {
-                uint32_t packed[4];
-#pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    reader_refill(r, src);
-                    uint32_t e0 = lut1[r.hi >> (32 - K)];
-                    r.hi = __funnelshift_l(r.lo, r.hi, e0);
-                    r.lo = __funnelshift_l(0u, r.lo, e0);
-                    uint32_t e1 = lut1[r.hi >> (32 - K)];
-                    r.hi = __funnelshift_l(r.lo, r.hi, e1);
-                    r.lo = __funnelshift_l(0u, r.lo, e1);
-                    r.nb -= (int)((e0 + e1) & 0xffu);
-                    if (__builtin_expect((e0 | e1) & kEscFlag, 0)) {
-                        PairFix f = redo_pair<K>(lut1, cx.tb.lut2, cx.tb.aux, cx.tb.status, src.words, src.last, r, e0);
-                        r = f.r;
-                        e0 = f.e0;
-                        e1 = f.e1;
-                    }
-                    packed[p] = __byte_perm(e0, e1, 0x7632);      // two fp16 values, first symbol low
-                }
-                my_row[g ^ row_swz] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-            }
-            __syncwarp();
-            flush_tile(cx.tile, out_chunk, sub, t0, lane);
-            __syncwarp();
-        }
+        win_init<true>(w, words, r.pos);
+        if (cx.aux->group == 4u) rows_single<4>(w, cx, lane * 4u, out_row, sub, aligned32);
+        else rows_single<2>(w, cx, lane * 4u, out_row, sub, aligned32);
     }
-    const uint32_t used = (r.next << 5) - (uint32_t)r.nb - pos;
-    if (used != my_bits) atomicOr(cx.tb.status, kStatCorrupt);
-    __syncwarp();   // all lanes are done with the stage buffer before it is overwritten
-}
-
-// Decode chunk c; `next_c` (or 0xffffffff) is the chunk this warp will take afterwards, whose
-// bytes are pulled into L2 while this one is being decoded.
-template <int K>
-__device__ __forceinline__ void decode_chunk(WarpCtx& cx, const DevTensor& T, uint32_t c, uint32_t next_c,
-                                             uint32_t lane)
-{
-    const uint64_t off0 = T.offsets[c];
-    const uint64_t off1 = T.offsets[c + 1];
-    const uint32_t my_bits = T.sub_len[(uint64_t)c * kSubBlocks + lane];
-    if (next_c < T.n_chunks && lane == 0) {
-        uint64_t b0, b1;
-        if (chunk_range(T, T.offsets[next_c], T.offsets[next_c + 1], b0, b1))
-            bulk_prefetch_l2(reinterpret_cast<const char*>(T.stream) + b0, (uint32_t)(b1 - b0));
-    }
-    uint32_t incl = my_bits;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= (uint32_t)d) incl += t;
-    }
-    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
-    const uint32_t excl = incl - my_bits;
-
-    uint64_t byte0, byte1;
-    if (!chunk_range(T, off0, off1, byte0, byte1) || off1 - off0 != total) {
-        if (lane == 0) atomicOr(cx.tb.status, kStatCorrupt);
-        return;
-    }
-    const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    const bool full = (uint64_t)(c + 1) * T.chunk_symbols <= T.n;
-    const uint64_t copy_bytes = byte1 - byte0;
-    if (full && (sub % kTile) == 0 && copy_bytes <= cx.stage_bytes && !cx.dead)
-        decode_chunk_staged<K>(cx, T, c, off0, byte0, (uint32_t)copy_bytes, excl, my_bits, lane);
-    else
-        decode_chunk_general<K>(cx.tb, T, c, off0, excl, my_bits, lane);
+    if (win_used_bits(w, words, r.pos) != r.my_bits) atomicOr(cx.status, kStatCorrupt);
+    __syncwarp();   // all lanes are done with these bytes before the ring reuses them
 }
 
 // ------------------------------------------------------------------ persistent kernel
@@ -562,32 +633,31 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                                                          uint32_t chunks_per_item, uint32_t stage_bytes,
                                                          uint32_t* __restrict__ control)
 {
-    extern __shared__ __align__(128) unsigned char smem[];
-    // layout: [lut1][lut2][aux][tensor][per-warp tile][per-warp stage][mbarriers][item + claim slots]
-    uint32_t* s_lut1 = reinterpret_cast<uint32_t*>(smem);
-    uint32_t* s_lut2 = s_lut1 + (1u << K);
-    DecodeAux* s_aux = reinterpret_cast<DecodeAux*>(s_lut2 + kLut2Entries);
+    // layout: [tables][aux][tensor][per-warp rings][over-read pad][mbarriers][item + claim slots]
+    DecodeAux* s_aux = reinterpret_cast<DecodeAux*>(smem + lut_bytes(K));
     DevTensor* s_tensor = reinterpret_cast<DevTensor*>(s_aux + 1);
     unsigned char* p = reinterpret_cast<unsigned char*>(s_tensor + 1);
     p = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(p) + 127) & ~(uintptr_t)127);
     const uint32_t warps = blockDim.x >> 5;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned char* tiles = p;
-    unsigned char* stages = tiles + (size_t)warps * kTileBytes;
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(stages + (size_t)warps * stage_bytes);
-    volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(bars + warps);   // [2]
-    uint32_t* s_claim = const_cast<uint32_t*>(s_item) + 2;                            // [2]
+    unsigned char* stages = p;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(stages + (size_t)warps * stage_bytes + kOverRead);
+    volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(bars + 2 * warps);   // [2]
+    uint32_t* s_claim = const_cast<uint32_t*>(s_item) + 2;                                // [2]
 
     WarpCtx cx;
-    cx.tb = Tables{s_lut1, s_lut2, s_aux, control + 1};
-    cx.tile = reinterpret_cast<uint4*>(tiles + (size_t)warp * kTileBytes);
-    cx.stage = reinterpret_cast<uint32_t*>(stages + (size_t)warp * stage_bytes);
-    cx.bar = smem_addr(bars + warp);
+    cx.aux = s_aux;
+    cx.status = control + 1;
+    cx.stage = stages + (size_t)warp * stage_bytes;
     cx.stage_bytes = stage_bytes;
-    cx.phase = 0;
+    cx.bar = smem_addr(bars + 2 * warp);
+    cx.tickets = 0;
     cx.dead = false;
 
-    if (lane == 0) mbar_init(cx.bar, 1);
+    if (lane == 0) {
+        mbar_init(cx.bar, 1);
+        mbar_init(cx.bar + 8u, 1);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
@@ -617,39 +687,55 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
         if (lo != cur) {
             cur = lo;
             const TensorTables* tt = tables + cur;
-            const uint4* g1 = reinterpret_cast<const uint4*>(tt->lut1);
-            uint4* s1 = reinterpret_cast<uint4*>(s_lut1);
-            for (uint32_t i = threadIdx.x; i < (1u << K) / 4; i += blockDim.x) s1[i] = __ldg(g1 + i);
-            const uint4* g2 = reinterpret_cast<const uint4*>(tt->lut2);
-            uint4* s2 = reinterpret_cast<uint4*>(s_lut2);
-            for (uint32_t i = threadIdx.x; i < kLut2Entries / 4; i += blockDim.x) s2[i] = __ldg(g2 + i);
             const uint4* ga = reinterpret_cast<const uint4*>(&tt->aux);
             uint4* sa = reinterpret_cast<uint4*>(s_aux);
             for (uint32_t i = threadIdx.x; i < sizeof(DecodeAux) / 16; i += blockDim.x) sa[i] = __ldg(ga + i);
             const uint4* gt = reinterpret_cast<const uint4*>(tensors + cur);
             uint4* st = reinterpret_cast<uint4*>(s_tensor);
             for (uint32_t i = threadIdx.x; i < sizeof(DevTensor) / 16; i += blockDim.x) st[i] = __ldg(gt + i);
+            if (__ldg(&tt->aux.oct)) {
+                const uint4* g1 = tt->oct_val;
+                uint4* s1 = reinterpret_cast<uint4*>(smem);
+                for (uint32_t i = threadIdx.x; i < (1u << K); i += blockDim.x) s1[i] = __ldg(g1 + i);
+                const uint4* g2 = reinterpret_cast<const uint4*>(tt->oct_len);
+                uint4* s2 = reinterpret_cast<uint4*>(smem + (16u << K));
+                for (uint32_t i = threadIdx.x; i < (1u << K) / 16; i += blockDim.x) s2[i] = __ldg(g2 + i);
+            } else {
+                // 32 copies, cell-major: word (cell * 32 + lane) belongs to lane's bank
+                uint32_t* s1 = reinterpret_cast<uint32_t*>(smem);
+                for (uint32_t cell = warp; cell < (uint32_t)kExpEntries; cell += warps)
+                    s1[cell * 32u + lane] = __ldg(tt->exp_lut + cell);
+            }
             __syncthreads();
         }
         const DevTensor& T = *s_tensor;
         const uint32_t first = (item - __ldg(item_start + cur)) * chunks_per_item;
         const uint32_t count = min(chunks_per_item, T.n_chunks - first);
-        // the warps share out the item's chunks; each keeps one claim ahead for the L2 prefetch
-        uint32_t k = 0;
-        if (lane == 0) k = atomicAdd(&s_claim[slot], 1u);
-        k = __shfl_sync(0xffffffffu, k, 0);
-        while (k < count) {
-            uint32_t kn = 0;
-            if (lane == 0) kn = atomicAdd(&s_claim[slot], 1u);
-            kn = __shfl_sync(0xffffffffu, kn, 0);
-            decode_chunk<K>(cx, T, first + k, kn < count ? first + kn : 0xffffffffu, lane);
-            k = kn;
+
+        // the warps share out the item's chunks; each runs: fetch index (i + 2), copy (i + 1), decode (i)
+        auto claim = [&]() -> uint32_t {
+            uint32_t k = 0;
+            if (lane == 0) k = atomicAdd(&s_claim[slot], 1u);
+            k = __shfl_sync(0xffffffffu, k, 0);
+            return k < count ? first + k : kNone;
+        };
+        Ready r0;
+        r0.c = kNone;
+        r0.kind = kSkip;
+        r0.at = r0.bytes = 0;
+        Pending p2 = fetch_index(T, claim(), lane);
+        while (true) {
+            Ready r1 = prepare(cx, T, p2, r0, lane);
+            p2 = fetch_index(T, r1.c == kNone ? kNone : claim(), lane);
+            if (r0.c != kNone) decode_ready<K>(cx, T, r0, lane);
+            if (r1.c == kNone) break;
+            r0 = r1;
         }
         __syncthreads();   // tables may be replaced; s_item / s_claim [slot ^ 1] are now visible
         slot ^= 1u;
     }
     // A warp that gave up on a bulk copy lets it land (bounded) before its buffer goes away.
-    if (cx.dead) (void)mbar_wait(cx.bar, cx.phase);
+    if (cx.dead && cx.tickets) (void)mbar_wait(cx.bar + 8u * ((cx.tickets - 1) & 1u), ((cx.tickets - 1) >> 1) & 1u);
 }
 
 struct Shape {
@@ -658,18 +744,18 @@ struct Shape {
 };
 
 // Shared memory of one CTA for a launch shape; stage_bytes == 0 if it cannot fit.
-Shape shape_for(const DecodeConfig& cfg, int max_smem, uint32_t want_stage)
+Shape shape_for(const DecodeConfig& cfg, int max_smem)
 {
-    size_t fixed = (4u << cfg.lut_bits) + 4u * kLut2Entries + sizeof(DecodeAux) + sizeof(DevTensor) + 128;
-    size_t per_warp_fixed = kTileBytes + 8;
+    size_t fixed = lut_bytes(cfg.lut_bits) + sizeof(DecodeAux) + sizeof(DevTensor) + 128 + kOverRead;
+    size_t per_warp_fixed = 16;   // two mbarriers
     size_t tail = 16;
     size_t budget = (size_t)max_smem / cfg.ctas_per_sm;
     if (cfg.ctas_per_sm > 1) budget -= 1024;   // per-CTA reservation of the driver
     Shape s{0, 0};
-    if (budget < fixed + tail + cfg.warps_per_cta * (per_warp_fixed + 512)) return s;
+    if (budget < fixed + tail + cfg.warps_per_cta * (per_warp_fixed + 1024)) return s;
     size_t avail = (budget - fixed - tail) / cfg.warps_per_cta - per_warp_fixed;
     uint32_t stage = (uint32_t)(avail & ~(size_t)127);
-    if (stage > want_stage) stage = want_stage;
+    if (stage > 32768u) stage = 32768u;
     s.stage_bytes = stage;
     s.smem = fixed + tail + cfg.warps_per_cta * (per_warp_fixed + stage);
     return s;
@@ -678,9 +764,9 @@ Shape shape_for(const DecodeConfig& cfg, int max_smem, uint32_t want_stage)
 template <int K>
 entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
                            const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
-                           uint32_t want_stage, cudaStream_t s)
+                           cudaStream_t s)
 {
-    Shape sh = shape_for(cfg, ws->max_smem_optin, want_stage);
+    Shape sh = shape_for(cfg, ws->max_smem_optin);
     if (sh.stage_bytes == 0) return ENTRO_ERR_UNSUPPORTED;
     static int configured_smem[64] = {0};
     if ((int)sh.smem > configured_smem[ws->device]) {
@@ -700,6 +786,18 @@ entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTens
     return ENTRO_OK;
 }
 
+entro_status launch_decode_any(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
+                               const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
+                               cudaStream_t s)
+{
+    switch (cfg.lut_bits) {
+        case 10: return launch_decode<10>(ws, cfg, tensors, ntensors, item_start, total_items, tables, s);
+        case 11: return launch_decode<11>(ws, cfg, tensors, ntensors, item_start, total_items, tables, s);
+        case 12: return launch_decode<12>(ws, cfg, tensors, ntensors, item_start, total_items, tables, s);
+    }
+    return ENTRO_ERR_UNSUPPORTED;
+}
+
 entro_status validate_desc(const entro_tensor_desc& d)
 {
     if (d.n == 0) return ENTRO_OK;
@@ -712,6 +810,26 @@ entro_status validate_desc(const entro_tensor_desc& d)
     if (num_chunks(d.n, d.chunk_symbols) > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
     if (d.stream_words < ENTRO_STREAM_SLACK_WORDS + 1) return ENTRO_ERR_INVALID_ARG;
     return ENTRO_OK;
+}
+
+// Device-side form of a descriptor; returns the tensor's number of work items.
+uint64_t fill_dev_tensor(const entro_tensor_desc& d, const DecodeConfig& cfg, DevTensor& t)
+{
+    const uint64_t nc = num_chunks(d.n, d.chunk_symbols);
+    t.stream = d.stream_dev;
+    t.offsets = static_cast<const uint64_t*>(d.index_dev);
+    t.sub_len = reinterpret_cast<const uint16_t*>(t.offsets + nc + 1);
+    t.out = static_cast<uint16_t*>(d.out_fp16_dev);
+    t.stream_words = d.stream_words;
+    t.n = d.n;
+    t.chunk_symbols = d.chunk_symbols;
+    t.n_chunks = (uint32_t)nc;
+    t.nsym = (uint32_t)d.cb.nsym;
+    t.scale = d.scale;
+    t.zero_point = d.zero_point;
+    t.pad[0] = t.pad[1] = t.pad[2] = 0;
+    for (int j = 0; j < ENTRO_MAX_SYMBOLS; ++j) t.len[j] = j < d.cb.nsym ? d.cb.len[j] : 0;
+    return (nc + cfg.chunks_per_item - 1) / cfg.chunks_per_item;
 }
 
 }  // namespace
@@ -738,35 +856,12 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     DevTensor* ht = static_cast<DevTensor*>(ws->pinned);
     uint32_t* hitems = reinterpret_cast<uint32_t*>(static_cast<char*>(ws->pinned) + tensors_bytes);
     uint64_t items = 0;
-    uint32_t want_stage = 0;
     int k = 0;
     for (int i = 0; i < ntensors; ++i) {
-        const entro_tensor_desc& d = descs[i];
-        if (!d.n) continue;
-        DevTensor& t = ht[k];
-        const uint64_t nc = num_chunks(d.n, d.chunk_symbols);
-        t.stream = d.stream_dev;
-        t.offsets = static_cast<const uint64_t*>(d.index_dev);
-        t.sub_len = reinterpret_cast<const uint16_t*>(t.offsets + nc + 1);
-        t.out = static_cast<uint16_t*>(d.out_fp16_dev);
-        t.stream_words = d.stream_words;
-        t.n = d.n;
-        t.chunk_symbols = d.chunk_symbols;
-        t.n_chunks = (uint32_t)nc;
-        t.nsym = (uint32_t)d.cb.nsym;
-        t.scale = d.scale;
-        t.zero_point = d.zero_point;
-        t.pad[0] = t.pad[1] = t.pad[2] = 0;
-        for (int j = 0; j < ENTRO_MAX_SYMBOLS; ++j) t.len[j] = j < d.cb.nsym ? d.cb.len[j] : 0;
+        if (!descs[i].n) continue;
         hitems[k] = (uint32_t)items;
-        items += (nc + cfg.chunks_per_item - 1) / cfg.chunks_per_item;
+        items += fill_dev_tensor(descs[i], cfg, ht[k]);
         if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
-        // stage buffer: room for a chunk at one byte per symbol (an 8-bit alphabet averages
-        // less), or 3/8 of a byte for alphabets of 16 symbols and fewer; chunks that need
-        // more take the general path
-        uint32_t want = d.cb.nsym <= 16 ? (d.chunk_symbols * 3) / 8 : d.chunk_symbols;
-        want = ((want + 127) & ~127u) + 128;
-        if (want > want_stage) want_stage = want;
         ++k;
     }
     hitems[live] = (uint32_t)items;
@@ -780,12 +875,7 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     build_tables_kernel<<<live, 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
-    switch (cfg.lut_bits) {
-        case 10: return launch_decode<10>(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, want_stage, s);
-        case 11: return launch_decode<11>(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, want_stage, s);
-        case 12: return launch_decode<12>(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, want_stage, s);
-    }
-    return ENTRO_ERR_UNSUPPORTED;
+    return launch_decode_any(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, s);
 }
 
 }  // namespace entro
@@ -955,32 +1045,12 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
 
     StaticUpload up;
     uint64_t items = 0;
-    uint32_t want_stage = 0;
     int k = 0;
     for (int i = 0; i < ntensors; ++i) {
-        const entro_tensor_desc& d = descs_host[i];
-        if (!d.n) continue;
-        DevTensor& t = up.tensors[k];
-        const uint64_t nc = num_chunks(d.n, d.chunk_symbols);
-        t.stream = d.stream_dev;
-        t.offsets = static_cast<const uint64_t*>(d.index_dev);
-        t.sub_len = reinterpret_cast<const uint16_t*>(t.offsets + nc + 1);
-        t.out = static_cast<uint16_t*>(d.out_fp16_dev);
-        t.stream_words = d.stream_words;
-        t.n = d.n;
-        t.chunk_symbols = d.chunk_symbols;
-        t.n_chunks = (uint32_t)nc;
-        t.nsym = (uint32_t)d.cb.nsym;
-        t.scale = d.scale;
-        t.zero_point = d.zero_point;
-        t.pad[0] = t.pad[1] = t.pad[2] = 0;
-        for (int j = 0; j < ENTRO_MAX_SYMBOLS; ++j) t.len[j] = j < d.cb.nsym ? d.cb.len[j] : 0;
+        if (!descs_host[i].n) continue;
         up.item_start[k] = (uint32_t)items;
-        items += (nc + cfg.chunks_per_item - 1) / cfg.chunks_per_item;
+        items += fill_dev_tensor(descs_host[i], cfg, up.tensors[k]);
         if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
-        uint32_t want = d.cb.nsym <= 16 ? (d.chunk_symbols * 3) / 8 : d.chunk_symbols;
-        want = ((want + 127) & ~127u) + 128;
-        if (want > want_stage) want_stage = want;
         ++k;
     }
     for (int j = live; j < 16; ++j) up.item_start[j] = (uint32_t)items;
@@ -995,16 +1065,11 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
     ENTRO_CUDA(cudaGetLastError());
     // launch_decode reads only these fields of a workspace; no timing records are taken here
     Workspace ws;
-    cudaGetDevice(&ws.device);
+    ENTRO_CUDA(cudaGetDevice(&ws.device));
     ws.sm_count = sd->sm_count;
     ws.max_smem_optin = sd->max_smem_optin;
     ws.control = sc->control;
-    switch (cfg.lut_bits) {
-        case 10: st = launch_decode<10>(&ws, cfg, sc->tensors, live, sc->item_start, (uint32_t)items, sc->tables, want_stage, s); break;
-        case 11: st = launch_decode<11>(&ws, cfg, sc->tensors, live, sc->item_start, (uint32_t)items, sc->tables, want_stage, s); break;
-        case 12: st = launch_decode<12>(&ws, cfg, sc->tensors, live, sc->item_start, (uint32_t)items, sc->tables, want_stage, s); break;
-        default: st = ENTRO_ERR_UNSUPPORTED;
-    }
+    st = launch_decode_any(&ws, cfg, sc->tensors, live, sc->item_start, (uint32_t)items, sc->tables, s);
     if (st != ENTRO_OK) return st;
     if (status_dev)
         ENTRO_CUDA(cudaMemcpyAsync(status_dev, sc->control + 1, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
@@ -1022,10 +1087,11 @@ extern "C" entro_status entro_set_decode_config(int lut_bits, int warps_per_cta,
     if (c.lut_bits < 10 || c.lut_bits > kMaxLutBits || c.warps_per_cta < 4 || c.warps_per_cta > 32 ||
         c.ctas_per_sm < 1 || c.ctas_per_sm > 8 || c.chunks_per_item < 1 || c.chunks_per_item > 65536)
         return ENTRO_ERR_INVALID_ARG;
-    Workspace* ws = workspace();
-    if (ws) {
-        // smallest useful stage buffer is 1 KiB
-        Shape sh = shape_for(c, ws->max_smem_optin, 1024);
+    int dev = -1, max_smem = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) == cudaSuccess) {
+        // the ring of a warp must hold at least 1 KiB
+        Shape sh = shape_for(c, max_smem);
         if (sh.stage_bytes < 1024) return ENTRO_ERR_INVALID_ARG;
     }
     decode_config() = c;

@@ -9,8 +9,9 @@
 namespace entro {
 
 constexpr int kSubBlocks = ENTRO_SUB_BLOCKS;
-constexpr int kMaxLutBits = 12;
-constexpr uint32_t kEscFlag = 0x8000u;        // LUT entry: code longer than the table width
+constexpr int kMaxLutBits = 12;               // widest window of the eight-symbol table
+constexpr int kExpBits = 4;                   // mantissa bits of the exponent-indexed table
+constexpr int kExpEntries = 32 << kExpBits;
 
 // Device status bits (OR-ed by kernels, read by entro_last_device_status).
 constexpr uint32_t kStatCorrupt = 1u;         // index / stream / codebook disagree
@@ -34,10 +35,7 @@ struct DevTensor {
 };
 static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vectors");
 
-constexpr int kLut2Entries = 2048;            // capacity of the second-level table
-constexpr uint32_t kQuadEscFlag = 0x80000000u; // four-symbol entry: the four codes do not fit
-
-// Per-tensor tables beside the first-level lookup table.
+// Per-tensor canonical-code description beside the lookup tables.
 struct DecodeAux {
     unsigned long long limit[ENTRO_MAX_CODE_LEN + 1];  // left-justified end of the codes of length <= l
     uint32_t first_code[ENTRO_MAX_CODE_LEN + 1];
@@ -45,27 +43,26 @@ struct DecodeAux {
     uint16_t val[ENTRO_MAX_SYMBOLS];                   // fp16( s * (q - z) ) per symbol
     uint8_t sorted[ENTRO_MAX_SYMBOLS];                 // symbols by (length, symbol)
     uint32_t max_len;
-    uint32_t quad;     // 1: first-level entries decode four symbols (alphabets of <= 16 symbols)
-    uint32_t t2;       // second level covers windows >= t2 (left-justified), in steps of 1 << shift2
-    uint32_t shift2;
-    uint32_t n2;       // entries in use in the second-level table (0 = none)
-    uint32_t pad[3];
+    uint32_t oct;      // 1: eight symbols per lookup (alphabets of <= 16 symbols)
+    uint32_t group;    // one-symbol lookups per window refill: 4 or 2
+    uint32_t pad;
 };
 static_assert(sizeof(DecodeAux) % 16 == 0, "DecodeAux is copied as 16-byte vectors");
 
 // Everything the decode kernel loads into shared memory when it switches tensor.
 struct TensorTables {
-    uint32_t lut1[1u << kMaxLutBits];
-    uint32_t lut2[kLut2Entries];   // single-symbol mode: second level; four-symbol mode: [0, 256) pair values
+    uint4 oct_val[1u << kMaxLutBits];      // eight fp16 values per window (oct mode)
+    uint8_t oct_len[1u << kMaxLutBits];    // bits they use, 0 = not eight whole codes
+    uint32_t exp_lut[kExpEntries];         // value << 16 | length, or length 64 (one-symbol mode)
     DecodeAux aux;
 };
 static_assert(sizeof(TensorTables) % 16 == 0, "TensorTables is copied as 16-byte vectors");
 
 struct DecodeConfig {
-    int lut_bits = 11;
-    int warps_per_cta = 16;
-    int ctas_per_sm = 2;
-    int chunks_per_item = 256;
+    int lut_bits = 12;
+    int warps_per_cta = 32;
+    int ctas_per_sm = 1;
+    int chunks_per_item = 512;
 };
 
 // Per-device workspace owned by the library.

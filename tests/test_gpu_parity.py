@@ -178,7 +178,7 @@ def test_decode_single_symbol_alphabet_and_two_symbols():
 
 
 @pytest.mark.parametrize("lut_bits,warps,ctas,per_item", [(10, 8, 2, 8), (12, 16, 1, 64), (11, 32, 1, 7),
-                                                          (11, 4, 4, 1), (11, 16, 2, 64)])
+                                                          (11, 4, 2, 1), (12, 16, 2, 64)])
 def test_decode_launch_shapes(lut_bits, warps, ctas, per_item):
     """The result does not depend on table width, CTA shape or work-item size."""
     try:
@@ -189,7 +189,7 @@ def test_decode_launch_shapes(lut_bits, warps, ctas, per_item):
             assert np.array_equal(gpu_decode_from_oracle_stream(c, n, chunk), expected_out(c))
         assert_status_ok()
     finally:
-        E.entro_set_decode_config(11, 16, 2, 64)
+        E.entro_set_decode_config(*E.DEFAULT_DECODE_CONFIG)
 
 
 def test_batched_decode_mixed_tensors():
