@@ -31,9 +31,13 @@
  *  - Bitstream: codewords concatenated MSB-first in row-major element order, stored in
  *    32-bit words, stream bit i being bit (31 - i % 32) of word i / 32.
  *  - Segments (Section 3, segmentation for parallel decoding): fixed-size chunks of
- *    chunk_symbols symbols of one tensor, offsets[c] = bit position where chunk c
- *    starts, offsets[n_chunks] = total bits; each chunk is cut into 32 equal
- *    sub-blocks whose bit lengths are recorded as well.
+ *    chunk_symbols consecutive symbols of one tensor, offsets[c] = bit position where
+ *    chunk c starts, offsets[n_chunks] = total bits.  The paper fixes that segments have
+ *    known boundaries and decode independently, not the order of the codewords inside
+ *    one.  Here a chunk's symbols are taken in groups of 8 consecutive symbols (the last
+ *    group may be short); sub-block l (0 <= l < 32) is the groups l, l + 32, l + 64, ...
+ *    in that order; the chunk's codewords are stored sub-block after sub-block, and
+ *    the bit length of every sub-block is recorded as well.
  */
 #include <math.h>
 #include <pthread.h>
@@ -55,6 +59,7 @@
 #define MAX_SYMBOLS 256
 #define MAX_LEN 32
 #define SUB_BLOCKS 32
+#define GROUP 8        /* symbols per group inside a chunk */
 
 /* ------------------------------------------------------------------ fp16 <-> fp32 */
 
@@ -340,14 +345,22 @@ int oracle_encode(const uint8_t *q, uint64_t n, const uint8_t *len, const uint32
     const uint64_t nchunks = oracle_num_chunks(n, chunk_symbols);
     memset(sub_len, 0, nchunks * SUB_BLOCKS * sizeof(uint16_t));
     uint64_t pos = 0;
-    for (uint64_t i = 0; i < n; ++i) {
-        uint64_t c = i / chunk_symbols;
-        uint32_t within = (uint32_t)(i % chunk_symbols);
-        if (within == 0) offsets[c] = pos;
-        int l = len[q[i]];
-        uint32_t cw = code[q[i]];
-        for (int b = l - 1; b >= 0; --b) put_bit(stream, pos++, (cw >> b) & 1);
-        sub_len[c * SUB_BLOCKS + within / sub] += (uint16_t)l;
+    (void)sub;
+    for (uint64_t c = 0; c < nchunks; ++c) {
+        const uint64_t first = c * chunk_symbols;
+        const uint64_t m = (first + chunk_symbols <= n) ? chunk_symbols : n - first;   /* symbols in this chunk */
+        offsets[c] = pos;
+        for (uint32_t l = 0; l < SUB_BLOCKS; ++l) {
+            for (uint64_t g = l; g * GROUP < m; g += SUB_BLOCKS) {
+                for (uint64_t k = 0; k < GROUP && g * GROUP + k < m; ++k) {
+                    const uint8_t sym = q[first + g * GROUP + k];
+                    const int ln = len[sym];
+                    const uint32_t cw = code[sym];
+                    for (int b = ln - 1; b >= 0; --b) put_bit(stream, pos++, (cw >> b) & 1);
+                    sub_len[c * SUB_BLOCKS + l] += (uint16_t)ln;
+                }
+            }
+        }
     }
     offsets[nchunks] = pos;
     *total_bits = pos;
@@ -432,9 +445,17 @@ static int decode_dequant_chunk(const uint32_t *stream, const uint64_t *offsets,
     int rc = oracle_decode_symbols(stream, offsets[nchunks], offsets[c], cnt, t, buf, &end);
     if (rc) return rc;
     if (end != offsets[c + 1]) return ORACLE_ERR_CORRUPT;
-    for (uint64_t i = 0; i < cnt; ++i) {
-        if (q_out) q_out[first + i] = buf[i];
-        if (out) out[first + i] = oracle_dequant_one(buf[i], s, z);
+    /* buf holds the symbols in stored order: sub-block after sub-block */
+    uint64_t stored = 0;
+    for (uint32_t l = 0; l < SUB_BLOCKS; ++l) {
+        for (uint64_t g = l; g * GROUP < cnt; g += SUB_BLOCKS) {
+            for (uint64_t k = 0; k < GROUP && g * GROUP + k < cnt; ++k) {
+                const uint64_t i = first + g * GROUP + k;
+                if (q_out) q_out[i] = buf[stored];
+                if (out) out[i] = oracle_dequant_one(buf[stored], s, z);
+                ++stored;
+            }
+        }
     }
     return ORACLE_OK;
 }

@@ -221,13 +221,38 @@ def _stream_bits(stream, nbits):
     return np.unpackbits(by.view(np.uint8))[:nbits]
 
 
-@pytest.mark.parametrize("bits,chunk", [(8, 4096), (4, 8192), (8, 64), (4, 32)])
+def _stored_order(n, chunk):
+    """Independent statement of the storage order: element indices in the order their
+    codewords appear in the stream, and the sub-block each belongs to.  Inside a chunk the
+    symbols form groups of 8; group g belongs to sub-block g % 32; a sub-block holds its
+    groups in increasing g; sub-blocks follow each other 0 .. 31."""
+    i = np.arange(n, dtype=np.int64)
+    c, r = i // chunk, i % chunk
+    g = r // 8
+    lane, rnd, k = g % 32, g // 32, r % 8
+    order = np.lexsort((k, rnd, lane, c))          # last key is the primary one
+    return order, lane
+
+
+def test_stored_order_small_example_by_hand():
+    """chunk = 32 * 8 * 2 = 512: lane 0 holds elements 0..7 then 256..263, lane 1 holds 8..15 then 264..271."""
+    order, lane = _stored_order(512 + 20, 512)
+    assert order[:16].tolist() == list(range(0, 8)) + list(range(256, 264))
+    assert order[16:32].tolist() == list(range(8, 16)) + list(range(264, 272))
+    assert order[496:512].tolist() == list(range(248, 256)) + list(range(504, 512))
+    # ragged second chunk of 20 symbols: groups 0, 1 full, group 2 has 4 symbols, lanes 0..2
+    assert order[512:].tolist() == list(range(512, 532))
+    assert lane[512:].tolist() == [0] * 8 + [1] * 8 + [2] * 4
+
+
+@pytest.mark.parametrize("bits,chunk", [(8, 4096), (4, 8192), (8, 64), (4, 32), (8, 512)])
 def test_stream_is_concatenation_of_codewords_and_index_is_consistent(bits, chunk):
     n = 3 * chunk + chunk // 3 + 5
     w = workloads.make_values(n, 0.02, 42 + bits).numpy()
     c = oracle.compress(w, bits, chunk)
     ln, cd, enc = c.lengths, c.codes, c.enc
-    text = "".join(_bitstr(cd[s], ln[s]) for s in c.q.tolist())
+    order, lane = _stored_order(n, chunk)
+    text = "".join(_bitstr(cd[s], ln[s]) for s in c.q[order].tolist())
     assert enc.total_bits == len(text) == int((c.counts * ln.astype(np.uint64)).sum())
     got = "".join(map(str, _stream_bits(enc.stream, enc.total_bits).tolist()))
     assert got == text
@@ -240,12 +265,11 @@ def test_stream_is_concatenation_of_codewords_and_index_is_consistent(bits, chun
     assert enc.offsets.size == nch + 1
     for k in range(nch + 1):
         assert int(enc.offsets[k]) == int(cum[min(k * chunk, n)])
-    sub = chunk // 32
+    # sub-block lengths: bits of the elements that belong to each sub-block
     for k in range(nch):
-        for j in range(32):
-            a, b = min(k * chunk + j * sub, n), min(k * chunk + (j + 1) * sub, n)
-            a, b = min(a, (k + 1) * chunk), min(b, (k + 1) * chunk)
-            assert int(enc.sub_len[k, j]) == int(cum[b] - cum[a])
+        a, b = k * chunk, min((k + 1) * chunk, n)
+        want = np.bincount(lane[a:b], weights=per_sym[a:b], minlength=32).astype(np.int64)
+        assert enc.sub_len[k].astype(np.int64).tolist() == want.tolist()
         assert int(enc.sub_len[k].sum()) == int(enc.offsets[k + 1] - enc.offsets[k])
 
 
@@ -293,11 +317,12 @@ def test_decoder_against_dictionary_decoder():
     c = oracle.compress(w, 8, chunk)
     table = {_bitstr(c.codes[s], c.lengths[s]): s for s in range(256) if c.lengths[s]}
     bits_arr = _stream_bits(c.enc.stream, c.enc.total_bits)
+    order, _ = _stored_order(n, chunk)
     for k in range(oracle.num_chunks(n, chunk)):
         cnt = min(chunk, n - k * chunk)
         syms, end = _dict_decode(bits_arr, int(c.enc.offsets[k]), cnt, table)
         assert end == int(c.enc.offsets[k + 1])
-        assert syms == c.q[k * chunk:k * chunk + cnt].tolist()
+        assert syms == c.q[order[k * chunk:k * chunk + cnt]].tolist()
 
 
 def test_decoder_rejects_corruption():
