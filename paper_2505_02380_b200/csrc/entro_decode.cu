@@ -9,7 +9,9 @@
 // decodes chunk i, the bytes of chunk i + 1 are arriving in its shared-memory ring through
 // one bulk asynchronous copy, and the index entries of chunk i + 2 are on their way into
 // registers.  Lanes walk their bits with lookup tables whose entries already hold the
-// dequantised fp16 values and store 16 values (32 bytes, one full sector) at a time.
+// dequantised fp16 values.  A sub-block is the chunk's 8-symbol groups l, l + 32, ..., so
+// when every lane has decoded one group the warp's 32 16-byte stores cover 512
+// contiguous bytes: four full lines per store instruction, no staging of the output.
 //
 // Tables per tensor (built by build_tables_kernel, copied into shared memory per CTA):
 //   alphabets > 16 symbols, one symbol per lookup.  Canonical codes grow longer towards the
@@ -174,11 +176,14 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
 
 // ------------------------------------------------------------------ bit reader
 
-// 64-bit window, left-justified: `nb` valid bits, zeros below.  With kInv the window holds
-// the complement of the stream bits (what the exponent-indexed table wants).
+// 64-bit window, left-justified, zeros below the valid bits.  `k` is 32 minus the number
+// of valid bits, kept modulo 2^16 in the low half of the register (the high half may hold
+// anything): negative (bit 15 set) while more than 32 bits are valid, else the left shift
+// that puts the next word behind the valid bits.  With kInv the window holds the
+// complement of the stream bits (what the exponent-indexed table wants).
 struct Win {
     uint32_t hi, lo;
-    int nb;
+    uint32_t k;
     const uint32_t* next;     // shared memory: next word to pull in
 };
 
@@ -194,34 +199,43 @@ __device__ __forceinline__ void win_init(Win& r, const uint32_t* words, uint32_t
     }
     r.hi = __funnelshift_l(w1, w0, bit);
     r.lo = w1 << bit;
-    r.nb = 64 - (int)bit;
+    r.k = bit - 32u;          // 64 - bit valid bits
     r.next = p + 2;
 }
 
-// Top up to more than 32 valid bits.  With nb <= 32 the low word is empty.
+// Top up to more than 32 valid bits.  With 32 or fewer the low word is empty.
 template <bool kInv>
 __device__ __forceinline__ void win_refill(Win& r)
 {
-    if (r.nb <= 32) {
+    if (!(r.k & 0x8000u)) {
         uint32_t w = *r.next++;
         if (kInv) w = ~w;
-        r.hi |= __funnelshift_rc(w, 0u, (uint32_t)r.nb);
-        r.lo = __funnelshift_lc(0u, w, (uint32_t)(32 - r.nb));
-        r.nb += 32;
+        r.hi |= __funnelshift_l(w, 0u, r.k);      // w >> (32 - k), nothing for k = 0
+        r.lo = __funnelshift_l(0u, w, r.k);       // w << k
+        r.k -= 32u;
     }
 }
 
-// Drop n bits, 0 <= n <= 32.
+// Drop n bits, 0 <= n <= 31 in the low five bits of n; n's low half is the true count.
 __device__ __forceinline__ void win_skip(Win& r, uint32_t n)
+{
+    r.hi = __funnelshift_l(r.lo, r.hi, n);
+    r.lo = __funnelshift_l(0u, r.lo, n);
+    r.k += n;
+}
+
+// Drop n bits, 0 <= n <= 32.
+__device__ __forceinline__ void win_skip_any(Win& r, uint32_t n)
 {
     r.hi = __funnelshift_lc(r.lo, r.hi, n);
     r.lo = __funnelshift_lc(0u, r.lo, n);
-    r.nb -= (int)n;
+    r.k += n;
 }
 
 __device__ __forceinline__ uint32_t win_used_bits(const Win& r, const uint32_t* words, uint32_t bit_pos)
 {
-    return (uint32_t)(r.next - words) * 32u - (uint32_t)r.nb - bit_pos;
+    const int valid = 32 - (int)(short)(r.k & 0xffffu);
+    return (uint32_t)(r.next - words) * 32u - (uint32_t)valid - bit_pos;
 }
 
 // The same over global memory, word by word, for chunks that are not staged.
@@ -284,7 +298,7 @@ __device__ __noinline__ SlowOut single_slow(const DecodeAux* aux, uint32_t* stat
         win_refill<true>(r);
         uint32_t e = exp_lookup(lane4, r.hi);
         if ((e & 0xffffu) > 32u) e = decode_by_range(aux, ~r.hi, status);
-        win_skip(r, e & 0xffffu);
+        win_skip_any(r, e & 0xffffu);
         o.e[k] = e;
     }
     o.r = r;
@@ -303,28 +317,13 @@ __device__ __noinline__ OctOut oct_slow(const DecodeAux* aux, uint32_t* status, 
     for (int k = 0; k < 8; ++k) {
         win_refill<false>(r);
         uint32_t e = decode_by_range(aux, r.hi, status);
-        win_skip(r, e & 0xffu);
+        win_skip_any(r, e & 0xffu);
         h[k] = e >> 16;
     }
     OctOut o;
     o.r = r;
     o.v = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
     return o;
-}
-
-// ------------------------------------------------------------------ output
-
-// 16 fp16 values (32 bytes) of this lane's row, write-once data.
-__device__ __forceinline__ void store16(uint16_t* dst, const uint32_t (&v)[8], bool aligned32)
-{
-    if (aligned32) {
-        asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(v[0]), "r"(v[1]), "r"(v[2]),
-                     "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-                     : "memory");
-    } else {
-        __stcs(reinterpret_cast<uint4*>(dst), make_uint4(v[0], v[1], v[2], v[3]));
-        __stcs(reinterpret_cast<uint4*>(dst) + 1, make_uint4(v[4], v[5], v[6], v[7]));
-    }
 }
 
 // ------------------------------------------------------------------ bulk copy + mbarrier
@@ -383,18 +382,23 @@ struct Pending {
 
 enum : uint32_t { kStaged = 0, kGeneral = 1, kSkip = 2 };
 
-// Chunk ready to decode.
+// Chunk ready to decode.  meta packs what the staging needs: ring offset / 16 (12 bits),
+// bytes / 16 (12 bits), ticket modulo 4 (2 bits), kind (2 bits), copy issued (1 bit).
 struct Ready {
     uint32_t c;                // or kNone
-    uint32_t kind;
     uint32_t pos;              // staged: this lane's first bit within the staged bytes; general: bits before it in the chunk
     uint32_t my_bits;
-    uint32_t at;               // staged: byte offset in the ring
-    uint32_t bytes;            // staged: bytes copied
-    uint32_t ticket;           // staged: which barrier and phase
-    uint32_t src_lo, src_hi;   // staged: byte offset in the stream, until the copy has been issued
-    bool issued;
+    uint32_t meta;
+    __device__ __forceinline__ uint32_t at() const { return (meta & 0xfffu) << 4; }
+    __device__ __forceinline__ uint32_t bytes() const { return ((meta >> 12) & 0xfffu) << 4; }
+    __device__ __forceinline__ uint32_t ticket() const { return (meta >> 24) & 3u; }
+    __device__ __forceinline__ uint32_t kind() const { return (meta >> 26) & 3u; }
+    __device__ __forceinline__ bool issued() const { return (meta >> 28) & 1u; }
 };
+__device__ __forceinline__ uint32_t ready_meta(uint32_t at, uint32_t bytes, uint32_t ticket, uint32_t kind)
+{
+    return (at >> 4) | ((bytes >> 4) << 12) | ((ticket & 3u) << 24) | (kind << 26);
+}
 
 __device__ __forceinline__ Pending fetch_index(const DevTensor& T, uint32_t c, uint32_t lane)
 {
@@ -409,14 +413,12 @@ __device__ __forceinline__ Pending fetch_index(const DevTensor& T, uint32_t c, u
     return p;
 }
 
-__device__ __forceinline__ void issue_copy(WarpCtx& cx, const DevTensor& T, Ready& r, uint32_t lane)
+__device__ __forceinline__ void issue_copy(WarpCtx& cx, const DevTensor& T, Ready& r, uint64_t byte0, uint32_t lane)
 {
-    if (lane == 0) {
-        const uint64_t byte0 = ((uint64_t)r.src_hi << 32) | r.src_lo;
-        bulk_load(smem_addr(cx.stage + r.at), reinterpret_cast<const char*>(T.stream) + byte0, r.bytes,
-                  cx.bar + 8u * (r.ticket & 1u));
-    }
-    r.issued = true;
+    if (lane == 0)
+        bulk_load(smem_addr(cx.stage + r.at()), reinterpret_cast<const char*>(T.stream) + byte0, r.bytes(),
+                  cx.bar + 8u * (r.ticket() & 1u));
+    r.meta |= 1u << 28;
 }
 
 // Turn a fetched index entry into a decodable chunk: lane start positions by prefix sum,
@@ -427,10 +429,9 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, const 
 {
     Ready r;
     r.c = p.c;
-    r.kind = kSkip;
-    r.pos = r.at = r.bytes = r.ticket = r.src_lo = r.src_hi = 0;
+    r.pos = 0;
     r.my_bits = p.bits;
-    r.issued = false;
+    r.meta = ready_meta(0, 0, 0, kSkip);
     if (p.c == kNone) return r;
     const uint64_t off0 = __shfl_sync(0xffffffffu, p.off, 0);
     const uint64_t off1 = __shfl_sync(0xffffffffu, p.off, 1);
@@ -454,29 +455,22 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, const 
     const bool full = (uint64_t)(p.c + 1) * T.chunk_symbols <= T.n;
     const uint64_t bytes = byte1 - byte0;
     if (!full || (sub & 15u) || bytes > cx.stage_bytes || cx.dead) {
-        r.kind = kGeneral;
+        r.meta = ready_meta(0, 0, 0, kGeneral);
         r.pos = excl;
         return r;
     }
-    r.kind = kStaged;
-    r.bytes = (uint32_t)bytes;
     r.pos = (uint32_t)(off0 - byte0 * 8) + excl;
-    r.src_lo = (uint32_t)byte0;
-    r.src_hi = (uint32_t)(byte0 >> 32);
-    r.ticket = cx.tickets++;
     // ring placement: behind the previous chunk's bytes, else at the start if that does not
     // overlap them, else at the start once the previous chunk has been decoded
+    uint32_t at = 0;
     bool now = true;
-    if (prev.c != kNone && prev.kind == kStaged) {
-        const uint32_t end = prev.at + prev.bytes;
-        if (end + r.bytes <= cx.stage_bytes) r.at = end;
-        else if (r.bytes <= prev.at) r.at = 0;
-        else {
-            r.at = 0;
-            now = false;
-        }
+    if (prev.c != kNone && prev.kind() == kStaged) {
+        const uint32_t end = prev.at() + prev.bytes();
+        if (end + (uint32_t)bytes <= cx.stage_bytes) at = end;
+        else if ((uint32_t)bytes > prev.at()) now = false;
     }
-    if (now) issue_copy(cx, T, r, lane);
+    r.meta = ready_meta(at, (uint32_t)bytes, cx.tickets++, kStaged);
+    if (now) issue_copy(cx, T, r, byte0, lane);
     return r;
 }
 
@@ -485,11 +479,8 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, const 
 __device__ __noinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t* status, const DevTensor& T, uint32_t c,
                                                   uint32_t excl, uint32_t my_bits, uint32_t lane)
 {
-    const uint32_t sub = T.chunk_symbols / kSubBlocks;
     const uint64_t chunk_first = (uint64_t)c * T.chunk_symbols;
-    const uint64_t chunk_syms = min((uint64_t)T.chunk_symbols, T.n - chunk_first);
-    const uint64_t lane_first = (uint64_t)lane * sub;
-    const uint32_t cnt = lane_first >= chunk_syms ? 0u : (uint32_t)min((uint64_t)sub, chunk_syms - lane_first);
+    const uint32_t m = (uint32_t)min((uint64_t)T.chunk_symbols, T.n - chunk_first);   // symbols in the chunk
     const uint64_t pos = T.offsets[c] + excl;
     const uint64_t word0 = pos >> 5;
     GlobalWin r;
@@ -502,121 +493,118 @@ __device__ __noinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t
     r.nb = 64 - (int)bit;
     r.next = 2;
     const bool oct = aux->oct != 0;
-    uint16_t* out = T.out + chunk_first + lane_first;
-    for (uint32_t i = 0; i < cnt; ++i) {
-        gwin_refill(r);
-        uint32_t e = kEscLen;
-        if (!oct) e = exp_lookup(lane * 4u, ~r.hi);
-        if ((e & 0xffffu) > 32u) e = decode_by_range(aux, r.hi, status);
-        const uint32_t n = e & 0xffffu;
-        r.hi = __funnelshift_lc(r.lo, r.hi, n);
-        r.lo = __funnelshift_lc(0u, r.lo, n);
-        r.nb -= (int)n;
-        out[i] = (uint16_t)(e >> 16);
+    uint16_t* out = T.out + chunk_first;
+    // this lane's symbols: groups lane, lane + 32, ... of 8 consecutive symbols
+    for (uint32_t g = lane; g * 8u < m; g += kSubBlocks) {
+        const uint32_t end = min(g * 8u + 8u, m);
+        for (uint32_t i = g * 8u; i < end; ++i) {
+            gwin_refill(r);
+            uint32_t e = kEscLen;
+            if (!oct) e = exp_lookup(lane * 4u, ~r.hi);
+            if ((e & 0xffffu) > 32u) e = decode_by_range(aux, r.hi, status);
+            const uint32_t n = e & 0xffffu;
+            r.hi = __funnelshift_lc(r.lo, r.hi, n);
+            r.lo = __funnelshift_lc(0u, r.lo, n);
+            r.nb -= (int)n;
+            out[i] = (uint16_t)(e >> 16);
+        }
     }
     const uint64_t used = ((uint64_t)r.next << 5) - (uint64_t)r.nb - bit;
     if (used != my_bits) atomicOr(status, kStatCorrupt);
 }
 
 // 8-bit alphabets: G lookups per refill.  The lookups of a group read the window at the
-// running sum of the lengths before them; the group stands if that sum ends at 32 bits or
-// less (the refill guarantees 33), which also rules out an unresolved cell (length 64).
+// running sum of the lengths before them; the group stands if that sum ends below 32 bits
+// (the refill guarantees 33), which also rules out an unresolved cell (length 64).
+// out_lane: this lane's first group; consecutive groups of a lane are 32 groups apart.
 template <int G>
-__device__ __forceinline__ void rows_single(Win& r, const WarpCtx& cx, uint32_t lane4, uint16_t* out_row, uint32_t sub,
-                                            bool aligned32)
+__device__ __forceinline__ void rows_single(Win& r, const WarpCtx& cx, uint32_t lane4, uint16_t* out_lane, uint32_t sub)
 {
     for (uint32_t t0 = 0; t0 < sub; t0 += 16) {
-        uint32_t pk[8];
 #pragma unroll
-        for (int g = 0; g < 16 / G; ++g) {
-            win_refill<true>(r);
-            uint32_t e[4];
-            e[0] = exp_lookup(lane4, r.hi);
-            uint32_t s = e[0];
+        for (int half = 0; half < 2; ++half) {
+            uint32_t pk[4];
 #pragma unroll
-            for (int k = 1; k < G; ++k) {
-                e[k] = exp_lookup(lane4, __funnelshift_l(r.lo, r.hi, s));   // shift = low 5 bits of s
-                s += e[k];
+            for (int g = 0; g < 8 / G; ++g) {
+                win_refill<true>(r);
+                uint32_t e[4];
+                e[0] = exp_lookup(lane4, r.hi);
+                uint32_t s = e[0];
+#pragma unroll
+                for (int k = 1; k < G; ++k) {
+                    e[k] = exp_lookup(lane4, __funnelshift_l(r.lo, r.hi, s));   // shift = low 5 bits of s
+                    s += e[k];
+                }
+                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) {
+                    SlowOut o = single_slow(cx.aux, cx.status, lane4, r, G);
+                    r = o.r;
+#pragma unroll
+                    for (int k = 0; k < G; ++k) e[k] = o.e[k];
+                } else {
+                    win_skip(r, s);
+                }
+#pragma unroll
+                for (int k = 0; k < G; k += 2) pk[(g * G + k) / 2] = __byte_perm(e[k], e[k + 1], 0x7632);
             }
-            const uint32_t S = s & 0xffffu;
-            if (__builtin_expect(S > 32u, 0)) {
-                SlowOut o = single_slow(cx.aux, cx.status, lane4, r, G);
-                r = o.r;
-#pragma unroll
-                for (int k = 0; k < G; ++k) e[k] = o.e[k];
-            } else {
-                win_skip(r, S);
-            }
-#pragma unroll
-            for (int k = 0; k < G; k += 2) pk[(g * G + k) / 2] = __byte_perm(e[k], e[k + 1], 0x7632);
+            __stcs(reinterpret_cast<uint4*>(out_lane + (size_t)(t0 + 8 * half) * kSubBlocks),
+                   make_uint4(pk[0], pk[1], pk[2], pk[3]));
         }
-        store16(out_row + t0, pk, aligned32);
     }
 }
 
 // 4-bit alphabets: eight symbols per lookup.
 template <int K>
-__device__ __forceinline__ void rows_oct(Win& r, const WarpCtx& cx, uint16_t* out_row, uint32_t sub, bool aligned32)
+__device__ __forceinline__ void rows_oct(Win& r, const WarpCtx& cx, uint16_t* out_lane, uint32_t sub)
 {
-    for (uint32_t t0 = 0; t0 < sub; t0 += 16) {
-        uint32_t pk[8];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            win_refill<false>(r);
-            const uint32_t idx = r.hi >> (32 - K);
-            uint4 v = *reinterpret_cast<const uint4*>(smem + idx * 16u);
-            const uint32_t n = *(smem + (16u << K) + idx);
-            if (__builtin_expect(n == 0u, 0)) {
-                OctOut o = oct_slow(cx.aux, cx.status, r);
-                r = o.r;
-                v = o.v;
-            } else {
-                r.hi = __funnelshift_l(r.lo, r.hi, n);
-                r.lo <<= n;
-                r.nb -= (int)n;
-            }
-            pk[4 * h] = v.x;
-            pk[4 * h + 1] = v.y;
-            pk[4 * h + 2] = v.z;
-            pk[4 * h + 3] = v.w;
+    for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
+        win_refill<false>(r);
+        const uint32_t idx = r.hi >> (32 - K);
+        uint4 v = *reinterpret_cast<const uint4*>(smem + idx * 16u);
+        const uint32_t n = *(smem + (16u << K) + idx);
+        if (__builtin_expect(n == 0u, 0)) {
+            OctOut o = oct_slow(cx.aux, cx.status, r);
+            r = o.r;
+            v = o.v;
+        } else {
+            win_skip(r, n);
         }
-        store16(out_row + t0, pk, aligned32);
+        __stcs(reinterpret_cast<uint4*>(out_lane + (size_t)t0 * kSubBlocks), v);
     }
 }
 
 template <int K>
 __device__ __forceinline__ void decode_ready(WarpCtx& cx, const DevTensor& T, Ready& r, uint32_t lane)
 {
-    if (r.kind == kSkip) return;
-    if (r.kind == kStaged) {
-        if (!r.issued) issue_copy(cx, T, r, lane);
-        bool ok = mbar_wait(cx.bar + 8u * (r.ticket & 1u), (r.ticket >> 1) & 1u);
+    uint32_t kind = r.kind();
+    if (kind == kSkip) return;
+    if (kind == kStaged) {
+        if (!r.issued()) issue_copy(cx, T, r, (T.offsets[r.c] >> 3) & ~15ull, lane);
+        bool ok = mbar_wait(cx.bar + 8u * (r.ticket() & 1u), (r.ticket() >> 1) & 1u);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) {
             if (lane == 0) atomicOr(cx.status, kStatTimeout);
             cx.dead = true;
             // fall back to global memory; this lane's bits before it: pos minus the chunk's first bit
             const uint32_t first = __shfl_sync(0xffffffffu, r.pos, 0);
-            r.kind = kGeneral;
+            kind = kGeneral;
             r.pos -= first;
         }
     }
-    if (r.kind == kGeneral) {
+    if (kind == kGeneral) {
         decode_chunk_general(cx.aux, cx.status, T, r.c, r.pos, r.my_bits, lane);
         return;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    const uint32_t* words = reinterpret_cast<const uint32_t*>(cx.stage + r.at);
-    uint16_t* out_row = T.out + (uint64_t)r.c * T.chunk_symbols + (uint64_t)lane * sub;
-    const bool aligned32 = (reinterpret_cast<uintptr_t>(T.out) & 31u) == 0;
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(cx.stage + r.at());
+    uint16_t* out_lane = T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u;
     Win w;
     if (cx.aux->oct) {
         win_init<false>(w, words, r.pos);
-        rows_oct<K>(w, cx, out_row, sub, aligned32);
+        rows_oct<K>(w, cx, out_lane, sub);
     } else {
         win_init<true>(w, words, r.pos);
-        if (cx.aux->group == 4u) rows_single<4>(w, cx, lane * 4u, out_row, sub, aligned32);
-        else rows_single<2>(w, cx, lane * 4u, out_row, sub, aligned32);
+        if (cx.aux->group == 4u) rows_single<4>(w, cx, lane * 4u, out_lane, sub);
+        else rows_single<2>(w, cx, lane * 4u, out_lane, sub);
     }
     if (win_used_bits(w, words, r.pos) != r.my_bits) atomicOr(cx.status, kStatCorrupt);
     __syncwarp();   // all lanes are done with these bytes before the ring reuses them
@@ -721,8 +709,8 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
         };
         Ready r0;
         r0.c = kNone;
-        r0.kind = kSkip;
-        r0.at = r0.bytes = 0;
+        r0.pos = r0.my_bits = 0;
+        r0.meta = ready_meta(0, 0, 0, kSkip);
         Pending p2 = fetch_index(T, claim(), lane);
         while (true) {
             Ready r1 = prepare(cx, T, p2, r0, lane);

@@ -1,6 +1,8 @@
 // entro_encode: symbols -> bitstream + per-chunk bit-offset index (Section 3: variable
 // length codes; segments with known boundaries).  Three passes: bit lengths of every
 // sub-block, a prefix sum over chunks, then each sub-block packs its own bits.
+// Sub-block l of a chunk is the chunk's 8-symbol groups l, l + 32, l + 64, ... in that
+// order (the last group of a chunk may be short).
 #include "entro_internal.h"
 
 namespace entro {
@@ -14,6 +16,28 @@ struct Code {
     uint8_t len[ENTRO_MAX_SYMBOLS];
 };
 
+constexpr uint32_t kGroup = 8;    // symbols per group
+
+// Calls f(symbol) for every symbol of sub-block `lane` of the chunk that starts at element
+// `first` and holds m symbols, in stored order.
+template <class F>
+__device__ __forceinline__ void for_each_symbol(const uint8_t* __restrict__ q, uint64_t first, uint32_t m,
+                                                uint32_t lane, F f)
+{
+    for (uint32_t g = lane; g * kGroup < m; g += kSubBlocks) {
+        const uint32_t base = g * kGroup;
+        if (base + kGroup <= m) {
+            const uint2 v = *reinterpret_cast<const uint2*>(q + first + base);   // q is 16-byte aligned, base a multiple of 8
+#pragma unroll
+            for (int k = 0; k < 4; ++k) f((v.x >> (8 * k)) & 0xffu);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) f((v.y >> (8 * k)) & 0xffu);
+        } else {
+            for (uint32_t k = base; k < m; ++k) f((uint32_t)q[first + k]);
+        }
+    }
+}
+
 // Pass 1: one warp per chunk, one lane per sub-block.
 __global__ void __launch_bounds__(kThreads) sub_lengths_kernel(const uint8_t* __restrict__ q, uint64_t n,
                                                                uint32_t chunk_symbols, uint32_t n_chunks,
@@ -26,17 +50,15 @@ __global__ void __launch_bounds__(kThreads) sub_lengths_kernel(const uint8_t* __
     for (int i = threadIdx.x; i < ENTRO_MAX_SYMBOLS; i += kThreads) s_len[i] = cb->len[i];
     __syncthreads();
     const uint32_t lane = threadIdx.x & 31;
-    const uint32_t sub = chunk_symbols / kSubBlocks;
     for (uint32_t c = blockIdx.x * kWarps + (threadIdx.x >> 5); c < n_chunks; c += gridDim.x * kWarps) {
-        uint64_t first = (uint64_t)c * chunk_symbols + (uint64_t)lane * sub;
-        uint64_t chunk_end = min((uint64_t)(c + 1) * chunk_symbols, n);
-        uint64_t last = min(first + sub, chunk_end);
+        const uint64_t first = (uint64_t)c * chunk_symbols;
+        const uint32_t m = (uint32_t)min((uint64_t)chunk_symbols, n - first);
         uint32_t bits = 0, bad = 0;
-        for (uint64_t i = first; i < last; ++i) {
-            uint32_t l = s_len[q[i]];
+        for_each_symbol(q, first, m, lane, [&](uint32_t sym) {
+            uint32_t l = s_len[sym];
             bad |= (l == 0);
             bits += l;
-        }
+        });
         if (bad) atomicOr(bad_symbol, 1u);
         sub_len[(uint64_t)c * kSubBlocks + lane] = (uint16_t)bits;
         uint32_t total = bits;
@@ -104,7 +126,6 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const uint8_t* __restric
     }
     __syncthreads();
     const uint32_t lane = threadIdx.x & 31;
-    const uint32_t sub = chunk_symbols / kSubBlocks;
     for (uint32_t c = blockIdx.x * kWarps + (threadIdx.x >> 5); c < n_chunks; c += gridDim.x * kWarps) {
         uint32_t mine = sub_len[(uint64_t)c * kSubBlocks + lane];
         uint32_t incl = mine;
@@ -114,20 +135,18 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const uint8_t* __restric
             if (lane >= (uint32_t)d) incl += t;
         }
         unsigned long long pos = offsets[c] + (incl - mine);   // first bit of this sub-block
-        uint64_t first = (uint64_t)c * chunk_symbols + (uint64_t)lane * sub;
-        uint64_t chunk_end = min((uint64_t)(c + 1) * chunk_symbols, n);
-        uint64_t last = min(first + sub, chunk_end);
-        if (first >= last) continue;
+        const uint64_t first = (uint64_t)c * chunk_symbols;
+        const uint32_t m = (uint32_t)min((uint64_t)chunk_symbols, n - first);
+        if (lane * kGroup >= m) continue;     // empty sub-block
 
         // acc holds `fill` pending bits, left-justified; word is where they go next.
         unsigned long long word = pos >> 5;
         uint32_t fill = (uint32_t)(pos & 31);   // bits of `word` that belong to earlier sub-blocks
         unsigned long long acc = 0;             // bits [63 - fill ...] downwards are ours
         bool first_word = true;
-        for (uint64_t i = first; i < last; ++i) {
-            uint32_t sym = q[i];
+        for_each_symbol(q, first, m, lane, [&](uint32_t sym) {
             uint32_t l = s_len[sym];
-            if (l == 0) continue;               // reported by pass 1
+            if (l == 0) return;                 // reported by pass 1
             acc |= (unsigned long long)s_code[sym] << (64 - fill - l);
             fill += l;
             if (fill >= 32) {
@@ -139,7 +158,7 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const uint8_t* __restric
                 acc <<= 32;
                 fill -= 32;
             }
-        }
+        });
         if (fill) atomicOr(&stream[word], (uint32_t)(acc >> 32));
     }
 }
