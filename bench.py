@@ -127,8 +127,10 @@ def physical_gpu_index(local_rank: int) -> int:
 class DeviceModel:
     """A synthetic model compressed on the device with the library's own offline stages."""
 
-    def __init__(self, wl, E, lut_bits: int):
+    def __init__(self, wl, E, lut_bits: int, keep_q: bool = False):
         self.wl = wl
+        self.q = []              # quantised symbols per tensor (only with keep_q)
+        self.qparams = []
         self.keep = []           # device buffers
         descs = []
         # per-tensor decode tables read from HBM: canonical ranges + the lookup table of the tensor's mode
@@ -150,6 +152,9 @@ class DeviceModel:
             counts = E.entro_histogram(q, wl.bits)
             cb = E.entro_build_codebook(counts.tolist())
             enc = E.entro_encode(q, cb, wl.chunk_symbols, stream_words=E.entro_stream_words(counts.tolist(), cb))
+            self.qparams.append((qp.scale, qp.zero_point))
+            if keep_q:
+                self.q.append(q)
             del w, q
             out = self.out[pos:pos + spec.numel]
             pos += (spec.numel + 15) // 16 * 16
@@ -191,10 +196,8 @@ def time_steps(E, model, steps, warmup, world, sampler_index):
     if world > 1:
         dist.barrier()
     ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2505_02380_b200 import multirank
+    ms = multirank.max_over_ranks(ms, "cuda")
     launches = E.entro_kernel_launch_count() - launches0
     kernel_ms = E.entro_profile_read(steps)
     E.entro_profile_begin(0)
