@@ -25,7 +25,8 @@
 //     no bank conflicts whatever the data.
 //   alphabets <= 16 symbols, eight symbols per lookup: the next K bits index a table of
 //     16-byte entries (eight fp16 values) and a byte table (bits used, 0 = no eight whole
-//     codes in K bits).
+//     codes in K bits); one unreplicated copy of the exponent-indexed table serves the
+//     symbol-by-symbol repair of such windows.
 //   aux   canonical ranges per length, for whatever the tables do not resolve.
 #include <cuda_fp16.h>
 
@@ -40,11 +41,26 @@ constexpr uint32_t kNone = 0xffffffffu;
 constexpr uint32_t kWaitTries = 1u << 16;  // bound on polling a bulk copy (each try may suspend)
 constexpr uint32_t kEscLen = 0x40u;        // length field of a cell the table cannot resolve
 constexpr uint32_t kOverRead = 2064;       // a lane fed garbage may read this far past its chunk's bytes
+// Address of dynamic shared memory in the shared window on sm_100 (the first KiB of the
+// window is the driver's).  The hand-written lookups address the tables as [offset + 1024];
+// the kernel checks the assumption before it does anything else.
+constexpr uint32_t kSmemBase = 1024;
+static_assert(kExpBits == 4, "the hand-written lookups hard-code the 4-bit cell mask and shift");
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// 32-bit word at a shared-window address.
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
 
 // Shared-memory bytes of the lookup tables for a K-bit eight-symbol table.
 __host__ __device__ constexpr uint32_t lut_bytes(int K)
 {
-    return (17u << K) > (uint32_t)kExpEntries * 128u ? (17u << K) : (uint32_t)kExpEntries * 128u;
+    return (17u << K) + 4u * kExpEntries > (uint32_t)kExpEntries * 128u ? (17u << K) + 4u * kExpEntries
+                                                                        : (uint32_t)kExpEntries * 128u;
 }
 
 // ------------------------------------------------------------------ table construction
@@ -142,7 +158,8 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
             out.oct_val[i] = e;
             out.oct_len[i] = ok ? (uint8_t)used : (uint8_t)0;
         }
-    } else {
+    }
+    {
         // cell (e5, mant): windows that start with r ones and a zero, followed by the bits ~mant
         for (uint32_t i = tid; i < (uint32_t)kExpEntries; i += 256) {
             const uint32_t e5 = i >> kExpBits, mant = i & ((1u << kExpBits) - 1u);
@@ -184,15 +201,16 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
 struct Win {
     uint32_t hi, lo;
     uint32_t k;
-    const uint32_t* next;     // shared memory: next word to pull in
+    uint32_t next;            // shared-window address of the next word to pull in
 };
 
+// Window over the bits that start `bit_pos` bits after shared-window address `base`.
 template <bool kInv>
-__device__ __forceinline__ void win_init(Win& r, const uint32_t* words, uint32_t bit_pos)
+__device__ __forceinline__ void win_init(Win& r, uint32_t base, uint32_t bit_pos)
 {
-    const uint32_t* p = words + (bit_pos >> 5);
+    const uint32_t p = base + ((bit_pos >> 5) << 2);
     const uint32_t bit = bit_pos & 31u;
-    uint32_t w0 = p[0], w1 = p[1];
+    uint32_t w0 = lds32(p), w1 = lds32(p + 4);
     if (kInv) {
         w0 = ~w0;
         w1 = ~w1;
@@ -200,7 +218,7 @@ __device__ __forceinline__ void win_init(Win& r, const uint32_t* words, uint32_t
     r.hi = __funnelshift_l(w1, w0, bit);
     r.lo = w1 << bit;
     r.k = bit - 32u;          // 64 - bit valid bits
-    r.next = p + 2;
+    r.next = p + 8;
 }
 
 // Top up to more than 32 valid bits.  With 32 or fewer the low word is empty.
@@ -208,7 +226,8 @@ template <bool kInv>
 __device__ __forceinline__ void win_refill(Win& r)
 {
     if (!(r.k & 0x8000u)) {
-        uint32_t w = *r.next++;
+        uint32_t w = lds32(r.next);
+        r.next += 4;
         if (kInv) w = ~w;
         r.hi |= __funnelshift_l(w, 0u, r.k);      // w >> (32 - k), nothing for k = 0
         r.lo = __funnelshift_l(0u, w, r.k);       // w << k
@@ -232,10 +251,11 @@ __device__ __forceinline__ void win_skip_any(Win& r, uint32_t n)
     r.k += n;
 }
 
-__device__ __forceinline__ uint32_t win_used_bits(const Win& r, const uint32_t* words, uint32_t bit_pos)
+__device__ __forceinline__ int win_valid_bits(uint32_t k) { return 32 - (int)(short)(k & 0xffffu); }
+
+__device__ __forceinline__ uint32_t win_used_bits(const Win& r, uint32_t base, uint32_t bit_pos)
 {
-    const int valid = 32 - (int)(short)(r.k & 0xffffu);
-    return (uint32_t)(r.next - words) * 32u - (uint32_t)valid - bit_pos;
+    return (r.next - base) * 8u - (uint32_t)win_valid_bits(r.k) - bit_pos;
 }
 
 // The same over global memory, word by word, for chunks that are not staged.
@@ -283,52 +303,122 @@ __device__ __noinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32_t 
     return ((uint32_t)aux->val[sym] << 16) | len;
 }
 
-struct SlowOut {
-    Win r;
-    uint32_t e[4];
-};
+// One group of lookups of an 8-bit alphabet, hand-scheduled.  In: the inverted window
+// (hi, lo, k, next) and lane4 = 4 * lane.  The refill is predicated (no branch), the G
+// lookups read the window at the running sum of the entries before them (a funnel shift
+// uses the low five bits, the length sums), and the window is advanced by the final sum
+// in place.  Out: the fp16 values in pairs, and s, the sum of the G entries: the group
+// stands iff (s & 0xffe0) == 0, that is, every cell was resolved (an unresolved one adds
+// 64) and fewer than 32 bits were used.  If it does not stand the caller repairs it with
+// repair_group, which needs only next, k and s: k grew by exactly s, next did not move.
+#define ENTRO_LOOKUP(dst, win)                       \
+    "cvt.rz.f32.u32 f, " win ";\n\t"                  \
+    "mov.b32 a, f;\n\t"                               \
+    "shr.u32 a, a, 12;\n\t"                           \
+    "lop3.b32 a, a, 0xFF80, %7, 0xEA;\n\t"            \
+    "ld.shared.b32 " dst ", [a+1024];\n\t"
+#define ENTRO_REFILL                                 \
+    "and.b32 t, %2, 0x8000;\n\t"                      \
+    "setp.eq.u32 p, t, 0;\n\t"                        \
+    "@p ld.shared.b32 w, [%3];\n\t"                   \
+    "@p add.u32 %3, %3, 4;\n\t"                       \
+    "@p not.b32 w, w;\n\t"                            \
+    "@p shf.l.wrap.b32 t, w, 0, %2;\n\t"              \
+    "@p or.b32 %0, %0, t;\n\t"                        \
+    "@p shf.l.wrap.b32 %1, 0, w, %2;\n\t"             \
+    "@p add.u32 %2, %2, 0xffffffe0;\n\t"
+#define ENTRO_ADVANCE                                \
+    "shf.l.wrap.b32 %0, %1, %0, %6;\n\t"              \
+    "shf.l.wrap.b32 %1, 0, %1, %6;\n\t"               \
+    "add.u32 %2, %2, %6;\n\t"
 
-// A group of `count` (2 or 4) symbols of an 8-bit alphabet that the fast path gave up on:
-// symbol by symbol, any code length.  -> values in the high halves of e[].
-__device__ __noinline__ SlowOut single_slow(const DecodeAux* aux, uint32_t* status, uint32_t lane4, Win r, int count)
+__device__ __forceinline__ void group4(Win& r, uint32_t lane4, uint32_t& pk0, uint32_t& pk1, uint32_t& s)
 {
-    SlowOut o;
-    for (int k = 0; k < 4; ++k) o.e[k] = 0;
-    for (int k = 0; k < count; ++k) {
-        win_refill<true>(r);
-        uint32_t e = exp_lookup(lane4, r.hi);
-        if ((e & 0xffffu) > 32u) e = decode_by_range(aux, ~r.hi, status);
-        win_skip_any(r, e & 0xffffu);
-        o.e[k] = e;
-    }
-    o.r = r;
-    return o;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b32 t, w, a, e0, e1, e2, e3;\n\t"
+        ".reg .f32 f;\n\t" ENTRO_REFILL ENTRO_LOOKUP("e0", "%0")
+        "shf.l.wrap.b32 w, %1, %0, e0;\n\t" ENTRO_LOOKUP("e1", "w")
+        "add.u32 %6, e0, e1;\n\t"
+        "shf.l.wrap.b32 w, %1, %0, %6;\n\t" ENTRO_LOOKUP("e2", "w")
+        "add.u32 %6, %6, e2;\n\t"
+        "shf.l.wrap.b32 w, %1, %0, %6;\n\t" ENTRO_LOOKUP("e3", "w")
+        "add.u32 %6, %6, e3;\n\t"
+        "prmt.b32 %4, e0, e1, 0x7632;\n\t"
+        "prmt.b32 %5, e2, e3, 0x7632;\n\t" ENTRO_ADVANCE "}"
+        : "+r"(r.hi), "+r"(r.lo), "+r"(r.k), "+r"(r.next), "=&r"(pk0), "=&r"(pk1), "=&r"(s)
+        : "r"(lane4));
 }
 
-struct OctOut {
-    Win r;
-    uint4 v;
-};
+__device__ __forceinline__ void group2(Win& r, uint32_t lane4, uint32_t& pk0, uint32_t& s)
+{
+    uint32_t unused;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b32 t, w, a, e0, e1;\n\t"
+        ".reg .f32 f;\n\t" ENTRO_REFILL ENTRO_LOOKUP("e0", "%0")
+        "shf.l.wrap.b32 w, %1, %0, e0;\n\t" ENTRO_LOOKUP("e1", "w")
+        "add.u32 %6, e0, e1;\n\t"
+        "prmt.b32 %4, e0, e1, 0x7632;\n\t"
+        "mov.b32 %5, 0;\n\t" ENTRO_ADVANCE "}"
+        : "+r"(r.hi), "+r"(r.lo), "+r"(r.k), "+r"(r.next), "=&r"(pk0), "=&r"(unused), "=&r"(s)
+        : "r"(lane4));
+}
+#undef ENTRO_LOOKUP
+#undef ENTRO_REFILL
+#undef ENTRO_ADVANCE
+
+// The next symbol by itself, any code length: refill, one exponent-indexed lookup (this
+// lane's copy for 8-bit alphabets, the single copy behind the eight-symbol tables for 4-bit
+// ones), the canonical ranges if the cell is unresolved.  -> value << 16 | length.
+template <int K, bool kOct>
+__device__ __forceinline__ uint32_t next_symbol(Win& r, uint32_t* status, uint32_t lane4)
+{
+    win_refill<!kOct>(r);
+    const uint32_t inv = kOct ? ~r.hi : r.hi;
+    const uint32_t cell = (__float_as_uint(__uint2float_rz(inv)) >> (23 - kExpBits)) & (uint32_t)(kExpEntries - 1);
+    uint32_t e = kOct ? *reinterpret_cast<const uint32_t*>(smem + (17u << K) + cell * 4u)
+                      : *reinterpret_cast<const uint32_t*>(smem + cell * 128u + lane4);
+    if ((e & 0xffffu) > 32u) e = decode_by_range(reinterpret_cast<const DecodeAux*>(smem + lut_bytes(K)), ~inv, status);
+    win_skip_any(r, e & 0xffffu);
+    return e;
+}
+
+// Repair of a group of G symbols that did not stand (kept inline: a call here would park
+// the caller's registers in local memory, which misses the small L1 left beside 228 KB of
+// shared memory).  Rebuilds the window as it was before the group from (k, next, s), then
+// takes the symbols one by one.
+template <int K, int G>
+__device__ __forceinline__ void repair_group(Win& r, uint32_t* status, uint32_t lane4, uint32_t s, uint32_t& pk0,
+                                             uint32_t& pk1)
+{
+    const uint32_t valid = (uint32_t)win_valid_bits(r.k - s);   // 33 .. 64 bits were valid when the group began
+    const uint32_t bit_addr = r.next * 8u - valid;              // where they begin, in bits of the shared window
+    win_init<true>(r, (bit_addr >> 5) << 2, bit_addr & 31u);
+    const uint32_t e0 = next_symbol<K, false>(r, status, lane4);
+    const uint32_t e1 = next_symbol<K, false>(r, status, lane4);
+    pk0 = __byte_perm(e0, e1, 0x7632);
+    if (G == 4) {
+        const uint32_t e2 = next_symbol<K, false>(r, status, lane4);
+        const uint32_t e3 = next_symbol<K, false>(r, status, lane4);
+        pk1 = __byte_perm(e2, e3, 0x7632);
+    }
+}
 
 // Eight symbols of a 4-bit alphabet whose codes do not fit the table's window.
-__device__ __noinline__ OctOut oct_slow(const DecodeAux* aux, uint32_t* status, Win r)
+template <int K>
+__device__ __forceinline__ uint4 repair_oct(Win& r, uint32_t* status)
 {
     uint32_t h[8];
-    for (int k = 0; k < 8; ++k) {
-        win_refill<false>(r);
-        uint32_t e = decode_by_range(aux, r.hi, status);
-        win_skip_any(r, e & 0xffu);
-        h[k] = e >> 16;
-    }
-    OctOut o;
-    o.r = r;
-    o.v = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
-    return o;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) h[k] = next_symbol<K, true>(r, status, 0u);
+    return make_uint4(__byte_perm(h[0], h[1], 0x7632), __byte_perm(h[2], h[3], 0x7632), __byte_perm(h[4], h[5], 0x7632),
+                      __byte_perm(h[6], h[7], 0x7632));
 }
 
 // ------------------------------------------------------------------ bulk copy + mbarrier
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
@@ -363,31 +453,36 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 
 // ------------------------------------------------------------------ one chunk
 
+// Fixed places in shared memory: [tables][aux][tensor][rings ...].
+template <int K>
+__device__ __forceinline__ DecodeAux* aux_ptr() { return reinterpret_cast<DecodeAux*>(smem + lut_bytes(K)); }
+template <int K>
+__device__ __forceinline__ DevTensor* tensor_ptr()
+{
+    return reinterpret_cast<DevTensor*>(smem + lut_bytes(K) + sizeof(DecodeAux));
+}
+
+// What a warp carries from chunk to chunk (kept small: it lives in registers across the
+// decode loop).
 struct WarpCtx {
-    const DecodeAux* aux;      // shared
-    uint32_t* status;          // global
-    unsigned char* stage;      // shared: this warp's ring for compressed bytes
-    uint32_t stage_bytes;
-    uint32_t bar;              // shared address of this warp's two mbarriers
-    uint32_t tickets;          // bulk copies issued so far
-    bool dead;                 // a bulk copy never completed: stop staging
+    uint32_t stage_addr;       // shared-window address of this warp's ring for compressed bytes
+    uint32_t bar;              // shared-window address of this warp's two mbarriers
+    uint32_t idx_addr;         // shared-window address of this warp's two index slots
+    uint32_t state;            // bulk copies issued so far; bit 31: a copy never completed, stop staging
+    __device__ __forceinline__ bool dead() const { return (state >> 31) != 0u; }
 };
 
-// Chunk whose index entries have been requested from global memory.
-struct Pending {
-    uint32_t c;                // chunk within the tensor, or kNone
-    uint64_t off;              // even lanes: offsets[c], odd lanes: offsets[c + 1]
-    uint32_t bits;             // this lane's sub-block length
-};
+// An index slot holds one chunk's index entries, fetched asynchronously two chunks ahead:
+// the 32 sub-block lengths (64 bytes), then offsets[c] and offsets[c + 1].
+constexpr uint32_t kSlotBytes = 80;
 
 enum : uint32_t { kStaged = 0, kGeneral = 1, kSkip = 2 };
 
-// Chunk ready to decode.  meta packs what the staging needs: ring offset / 16 (12 bits),
-// bytes / 16 (12 bits), ticket modulo 4 (2 bits), kind (2 bits), copy issued (1 bit).
+// Chunk whose bytes have been asked for.  meta packs what the staging needs: ring offset /
+// 16 (12 bits), bytes / 16 (12 bits), ticket modulo 4 (2 bits), kind (2 bits), copy issued
+// (1 bit).  Everything else is re-read from the chunk's index slot when it is decoded.
 struct Ready {
     uint32_t c;                // or kNone
-    uint32_t pos;              // staged: this lane's first bit within the staged bytes; general: bits before it in the chunk
-    uint32_t my_bits;
     uint32_t meta;
     __device__ __forceinline__ uint32_t at() const { return (meta & 0xfffu) << 4; }
     __device__ __forceinline__ uint32_t bytes() const { return ((meta >> 12) & 0xfffu) << 4; }
@@ -400,76 +495,84 @@ __device__ __forceinline__ uint32_t ready_meta(uint32_t at, uint32_t bytes, uint
     return (at >> 4) | ((bytes >> 4) << 12) | ((ticket & 3u) << 24) | (kind << 26);
 }
 
-__device__ __forceinline__ Pending fetch_index(const DevTensor& T, uint32_t c, uint32_t lane)
+__device__ __forceinline__ unsigned long long lds64(uint32_t addr)
 {
-    Pending p;
-    p.c = c;
-    p.off = 0;
-    p.bits = 0;
-    if (c != kNone) {
-        p.off = T.offsets[c + (lane & 1u)];
-        p.bits = T.sub_len[(uint64_t)c * kSubBlocks + lane];
-    }
-    return p;
+    unsigned long long v;
+    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(addr));
+    return v;
 }
 
-__device__ __forceinline__ void issue_copy(WarpCtx& cx, const DevTensor& T, Ready& r, uint64_t byte0, uint32_t lane)
+// Ask for chunk c's index entries to be copied into the slot at shared address `slot`
+// (lanes 0..15 two sub-block lengths each, lanes 16 and 17 one offset each).  Nothing is
+// held in registers while the copies are in flight.
+__device__ __forceinline__ void fetch_index(const DevTensor& T, uint32_t c, uint32_t slot, uint32_t lane)
+{
+    if (c != kNone) {
+        if (lane < 16u) {
+            const char* src = reinterpret_cast<const char*>(T.sub_len + (uint64_t)c * kSubBlocks) + lane * 4u;
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(slot + lane * 4u), "l"(src) : "memory");
+        } else if (lane < 18u) {
+            const uint64_t* src = T.offsets + c + (lane - 16u);
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(slot + 64u + (lane - 16u) * 8u), "l"(src)
+                         : "memory");
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+__device__ __forceinline__ void issue_copy(const WarpCtx& cx, const DevTensor& T, Ready& r, uint64_t byte0, uint32_t lane)
 {
     if (lane == 0)
-        bulk_load(smem_addr(cx.stage + r.at()), reinterpret_cast<const char*>(T.stream) + byte0, r.bytes(),
+        bulk_load(cx.stage_addr + r.at(), reinterpret_cast<const char*>(T.stream) + byte0, r.bytes(),
                   cx.bar + 8u * (r.ticket() & 1u));
     r.meta |= 1u << 28;
 }
 
-// Turn a fetched index entry into a decodable chunk: lane start positions by prefix sum,
-// consistency checks, a place in the ring next to `prev` (the chunk decoded before this
-// one, possibly still undecoded), and the bulk copy if that place is free already.
-__device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, const Pending& p, const Ready& prev,
-                                         uint32_t lane)
+// Bytes of the stream that decoding a chunk touches: from the 16-byte boundary below its
+// first bit to 13 bytes past its last (a window looks ahead), rounded up to 16.
+__device__ __forceinline__ void chunk_bytes(uint64_t off0, uint64_t off1, uint64_t& byte0, uint64_t& byte1)
+{
+    byte0 = (off0 >> 3) & ~15ull;
+    byte1 = ((off1 >> 3) + 13 + 15) & ~15ull;
+}
+
+// Chunk c's offsets have arrived in `slot`: check them, find a place in the ring next to
+// `prev` (the chunk decoded before this one, still undecoded), and start the bulk copy if
+// that place is free already.  All lanes compute the same values.
+__device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32_t stage_bytes, uint32_t* status,
+                                         uint32_t c, uint32_t slot, const Ready& prev, uint32_t lane)
 {
     Ready r;
-    r.c = p.c;
-    r.pos = 0;
-    r.my_bits = p.bits;
+    r.c = c;
     r.meta = ready_meta(0, 0, 0, kSkip);
-    if (p.c == kNone) return r;
-    const uint64_t off0 = __shfl_sync(0xffffffffu, p.off, 0);
-    const uint64_t off1 = __shfl_sync(0xffffffffu, p.off, 1);
-    uint32_t incl = p.bits;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= (uint32_t)d) incl += t;
-    }
-    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
-    const uint32_t excl = incl - p.bits;
-    // bytes the chunk's decode touches: from the 16-byte boundary below its first bit to
-    // 13 bytes past its last (a window looks ahead), rounded up to 16
-    const uint64_t byte0 = (off0 >> 3) & ~15ull;
-    const uint64_t byte1 = ((off1 >> 3) + 13 + 15) & ~15ull;
-    if (off1 < off0 || off1 - off0 != (uint64_t)total || byte1 > T.stream_words * 4) {
-        if (lane == 0) atomicOr(cx.status, kStatCorrupt);
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncwarp();
+    if (c == kNone) return r;
+    const uint64_t off0 = lds64(slot + 64u), off1 = lds64(slot + 72u);
+    uint64_t byte0, byte1;
+    chunk_bytes(off0, off1, byte0, byte1);
+    if (off1 < off0 || off1 - off0 > 32ull * 65535ull || byte1 > T.stream_words * 4) {
+        if (lane == 0) atomicOr(status, kStatCorrupt);
         return r;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    const bool full = (uint64_t)(p.c + 1) * T.chunk_symbols <= T.n;
-    const uint64_t bytes = byte1 - byte0;
-    if (!full || (sub & 15u) || bytes > cx.stage_bytes || cx.dead) {
+    const bool full = (uint64_t)(c + 1) * T.chunk_symbols <= T.n;
+    const uint32_t bytes = (uint32_t)(byte1 - byte0);
+    if (!full || (sub & 7u) || bytes > stage_bytes || cx.dead()) {
         r.meta = ready_meta(0, 0, 0, kGeneral);
-        r.pos = excl;
         return r;
     }
-    r.pos = (uint32_t)(off0 - byte0 * 8) + excl;
     // ring placement: behind the previous chunk's bytes, else at the start if that does not
     // overlap them, else at the start once the previous chunk has been decoded
     uint32_t at = 0;
     bool now = true;
     if (prev.c != kNone && prev.kind() == kStaged) {
         const uint32_t end = prev.at() + prev.bytes();
-        if (end + (uint32_t)bytes <= cx.stage_bytes) at = end;
-        else if ((uint32_t)bytes > prev.at()) now = false;
+        if (end + bytes <= stage_bytes) at = end;
+        else if (bytes > prev.at()) now = false;
     }
-    r.meta = ready_meta(at, (uint32_t)bytes, cx.tickets++, kStaged);
+    r.meta = ready_meta(at, bytes, cx.state, kStaged);
+    cx.state++;
     if (now) issue_copy(cx, T, r, byte0, lane);
     return r;
 }
@@ -513,100 +616,129 @@ __device__ __noinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t
     if (used != my_bits) atomicOr(status, kStatCorrupt);
 }
 
-// 8-bit alphabets: G lookups per refill.  The lookups of a group read the window at the
-// running sum of the lengths before them; the group stands if that sum ends below 32 bits
-// (the refill guarantees 33), which also rules out an unresolved cell (length 64).
-// out_lane: this lane's first group; consecutive groups of a lane are 32 groups apart.
-template <int G>
-__device__ __forceinline__ void rows_single(Win& r, const WarpCtx& cx, uint32_t lane4, uint16_t* out_lane, uint32_t sub)
+// 8-bit alphabets: G lookups per window refill (group4 / group2 above).
+// dst: this lane's first group; consecutive groups of a lane are 32 groups apart.
+template <int K, int G>
+__device__ __forceinline__ void rows_single(Win& r, uint32_t* status, uint32_t lane4, uint4* dst, uint32_t sub)
 {
-    for (uint32_t t0 = 0; t0 < sub; t0 += 16) {
+    for (uint32_t t0 = 0; t0 < sub; t0 += 8, dst += kSubBlocks) {
+        uint32_t pk[4];
+        if (G == 4) {
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            uint32_t pk[4];
-#pragma unroll
-            for (int g = 0; g < 8 / G; ++g) {
-                win_refill<true>(r);
-                uint32_t e[4];
-                e[0] = exp_lookup(lane4, r.hi);
-                uint32_t s = e[0];
-#pragma unroll
-                for (int k = 1; k < G; ++k) {
-                    e[k] = exp_lookup(lane4, __funnelshift_l(r.lo, r.hi, s));   // shift = low 5 bits of s
-                    s += e[k];
-                }
-                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) {
-                    SlowOut o = single_slow(cx.aux, cx.status, lane4, r, G);
-                    r = o.r;
-#pragma unroll
-                    for (int k = 0; k < G; ++k) e[k] = o.e[k];
-                } else {
-                    win_skip(r, s);
-                }
-#pragma unroll
-                for (int k = 0; k < G; k += 2) pk[(g * G + k) / 2] = __byte_perm(e[k], e[k + 1], 0x7632);
+            for (int g = 0; g < 2; ++g) {
+                uint32_t s;
+                group4(r, lane4, pk[2 * g], pk[2 * g + 1], s);
+                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_group<K, 4>(r, status, lane4, s, pk[2 * g], pk[2 * g + 1]);
             }
-            __stcs(reinterpret_cast<uint4*>(out_lane + (size_t)(t0 + 8 * half) * kSubBlocks),
-                   make_uint4(pk[0], pk[1], pk[2], pk[3]));
+        } else {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                uint32_t s;
+                group2(r, lane4, pk[g], s);
+                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) {
+                    uint32_t none;
+                    repair_group<K, 2>(r, status, lane4, s, pk[g], none);
+                }
+            }
         }
+        __stcs(dst, make_uint4(pk[0], pk[1], pk[2], pk[3]));
     }
 }
 
 // 4-bit alphabets: eight symbols per lookup.
 template <int K>
-__device__ __forceinline__ void rows_oct(Win& r, const WarpCtx& cx, uint16_t* out_lane, uint32_t sub)
+__device__ __forceinline__ void rows_oct(Win& r, uint32_t* status, uint4* dst, uint32_t sub)
 {
-    for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
+    for (uint32_t t0 = 0; t0 < sub; t0 += 8, dst += kSubBlocks) {
         win_refill<false>(r);
         const uint32_t idx = r.hi >> (32 - K);
         uint4 v = *reinterpret_cast<const uint4*>(smem + idx * 16u);
         const uint32_t n = *(smem + (16u << K) + idx);
-        if (__builtin_expect(n == 0u, 0)) {
-            OctOut o = oct_slow(cx.aux, cx.status, r);
-            r = o.r;
-            v = o.v;
-        } else {
-            win_skip(r, n);
-        }
-        __stcs(reinterpret_cast<uint4*>(out_lane + (size_t)t0 * kSubBlocks), v);
+        if (__builtin_expect(n == 0u, 0)) v = repair_oct<K>(r, status);
+        else win_skip(r, n);
+        __stcs(dst, v);
     }
 }
 
+// What decode_start leaves for decode_finish: where this lane begins and must end.
+struct Lane {
+    uint32_t start, end;       // staged: shared-window bit addresses; general: bits before this lane's, and its count
+    uint32_t kind;
+};
+
+// First half of decoding chunk r (its index slot is about to be reused): lane positions by
+// a warp prefix sum over the sub-block lengths, checked against the offsets.
 template <int K>
-__device__ __forceinline__ void decode_ready(WarpCtx& cx, const DevTensor& T, Ready& r, uint32_t lane)
+__device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status, const Ready& r, uint32_t slot,
+                                             uint32_t lane)
 {
-    uint32_t kind = r.kind();
-    if (kind == kSkip) return;
-    if (kind == kStaged) {
+    Lane L;
+    L.start = L.end = 0;
+    L.kind = r.c == kNone ? (uint32_t)kSkip : r.kind();
+    if (L.kind == kSkip) return L;
+    const uint32_t pair = lds32(slot + (lane >> 1) * 4u);
+    const uint32_t bits = (lane & 1u) ? pair >> 16 : pair & 0xffffu;
+    uint32_t incl = bits;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= (uint32_t)d) incl += t;
+    }
+    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+    const uint64_t off0 = lds64(slot + 64u), off1 = lds64(slot + 72u);
+    if (off1 - off0 != (uint64_t)total) {       // the recorded lengths do not add up to the chunk
+        if (lane == 0) atomicOr(status, kStatCorrupt);
+        L.kind = kSkip;
+        return L;
+    }
+    const uint32_t excl = incl - bits;
+    if (L.kind == kGeneral) {
+        L.start = excl;
+        L.end = bits;
+    } else {
+        const uint32_t byte0_bits = (uint32_t)off0 & ~127u;    // bit offset of the copied bytes' start, modulo 2^32
+        L.start = (cx.stage_addr + r.at()) * 8u + ((uint32_t)off0 - byte0_bits) + excl;
+        L.end = L.start + bits;
+    }
+    return L;
+}
+
+template <int K>
+__device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Ready& r, Lane L, uint32_t lane)
+{
+    if (L.kind == kSkip) return;
+    const DevTensor& T = *tensor_ptr<K>();
+    if (L.kind == kStaged) {
         if (!r.issued()) issue_copy(cx, T, r, (T.offsets[r.c] >> 3) & ~15ull, lane);
         bool ok = mbar_wait(cx.bar + 8u * (r.ticket() & 1u), (r.ticket() >> 1) & 1u);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) {
-            if (lane == 0) atomicOr(cx.status, kStatTimeout);
-            cx.dead = true;
-            // fall back to global memory; this lane's bits before it: pos minus the chunk's first bit
-            const uint32_t first = __shfl_sync(0xffffffffu, r.pos, 0);
-            kind = kGeneral;
-            r.pos -= first;
+            if (lane == 0) atomicOr(status, kStatTimeout);
+            cx.state |= 1u << 31;
+            // fall back to global memory: bits of the chunk before this lane's, and this lane's count
+            const uint32_t first = __shfl_sync(0xffffffffu, L.start, 0);
+            L.kind = kGeneral;
+            L.end -= L.start;
+            L.start -= first;
         }
     }
-    if (kind == kGeneral) {
-        decode_chunk_general(cx.aux, cx.status, T, r.c, r.pos, r.my_bits, lane);
+    if (L.kind == kGeneral) {
+        decode_chunk_general(aux_ptr<K>(), status, T, r.c, L.start, L.end, lane);
         return;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    const uint32_t* words = reinterpret_cast<const uint32_t*>(cx.stage + r.at());
-    uint16_t* out_lane = T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u;
+    uint4* dst = reinterpret_cast<uint4*>(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
     Win w;
-    if (cx.aux->oct) {
-        win_init<false>(w, words, r.pos);
-        rows_oct<K>(w, cx, out_lane, sub);
+    if (aux_ptr<K>()->oct) {
+        win_init<false>(w, (L.start >> 5) << 2, L.start & 31u);
+        rows_oct<K>(w, status, dst, sub);
     } else {
-        win_init<true>(w, words, r.pos);
-        if (cx.aux->group == 4u) rows_single<4>(w, cx, lane * 4u, out_lane, sub);
-        else rows_single<2>(w, cx, lane * 4u, out_lane, sub);
+        win_init<true>(w, (L.start >> 5) << 2, L.start & 31u);
+        if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lane * 4u, dst, sub);
+        else rows_single<K, 2>(w, status, lane * 4u, dst, sub);
     }
-    if (win_used_bits(w, words, r.pos) != r.my_bits) atomicOr(cx.status, kStatCorrupt);
+    // the lane must stand exactly at the end of its sub-block
+    if (w.next * 8u - (uint32_t)win_valid_bits(w.k) != L.end) atomicOr(status, kStatCorrupt);
     __syncwarp();   // all lanes are done with these bytes before the ring reuses them
 }
 
@@ -621,26 +753,27 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                                                          uint32_t chunks_per_item, uint32_t stage_bytes,
                                                          uint32_t* __restrict__ control)
 {
-    // layout: [tables][aux][tensor][per-warp rings][over-read pad][mbarriers][item + claim slots]
-    DecodeAux* s_aux = reinterpret_cast<DecodeAux*>(smem + lut_bytes(K));
-    DevTensor* s_tensor = reinterpret_cast<DevTensor*>(s_aux + 1);
-    unsigned char* p = reinterpret_cast<unsigned char*>(s_tensor + 1);
-    p = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(p) + 127) & ~(uintptr_t)127);
+    // layout: [tables][aux][tensor][per-warp rings][over-read pad][mbarriers][index slots][item + claim slots]
+    if (smem_addr(smem) != kSmemBase) {   // the lookups' address arithmetic would be wrong: refuse to run
+        if (threadIdx.x == 0) atomicOr(control + 1, kStatInternal);
+        return;
+    }
+    DecodeAux* s_aux = aux_ptr<K>();
+    DevTensor* s_tensor = tensor_ptr<K>();
     const uint32_t warps = blockDim.x >> 5;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned char* stages = p;
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(stages + (size_t)warps * stage_bytes + kOverRead);
-    volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(bars + 2 * warps);   // [2]
-    uint32_t* s_claim = const_cast<uint32_t*>(s_item) + 2;                                // [2]
+    constexpr uint32_t kRings = (lut_bytes(K) + (uint32_t)sizeof(DecodeAux) + (uint32_t)sizeof(DevTensor) + 127u) & ~127u;
+    const uint32_t after = kRings + warps * stage_bytes + kOverRead;          // offset in smem, a multiple of 16
+    const uint32_t slots = after + warps * 16u;
+    volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(smem + slots + warps * 2u * kSlotBytes);   // [2]
+    uint32_t* s_claim = const_cast<uint32_t*>(s_item) + 2;                                                     // [2]
+    uint32_t* status = control + 1;
 
     WarpCtx cx;
-    cx.aux = s_aux;
-    cx.status = control + 1;
-    cx.stage = stages + (size_t)warp * stage_bytes;
-    cx.stage_bytes = stage_bytes;
-    cx.bar = smem_addr(bars + 2 * warp);
-    cx.tickets = 0;
-    cx.dead = false;
+    cx.stage_addr = kSmemBase + kRings + warp * stage_bytes;
+    cx.bar = kSmemBase + after + warp * 16u;
+    cx.idx_addr = kSmemBase + slots + warp * 2u * kSlotBytes;
+    cx.state = 0;
 
     if (lane == 0) {
         mbar_init(cx.bar, 1);
@@ -688,6 +821,8 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                 const uint4* g2 = reinterpret_cast<const uint4*>(tt->oct_len);
                 uint4* s2 = reinterpret_cast<uint4*>(smem + (16u << K));
                 for (uint32_t i = threadIdx.x; i < (1u << K) / 16; i += blockDim.x) s2[i] = __ldg(g2 + i);
+                uint32_t* s3 = reinterpret_cast<uint32_t*>(smem + (17u << K));
+                for (uint32_t i = threadIdx.x; i < (uint32_t)kExpEntries; i += blockDim.x) s3[i] = __ldg(tt->exp_lut + i);
             } else {
                 // 32 copies, cell-major: word (cell * 32 + lane) belongs to lane's bank
                 uint32_t* s1 = reinterpret_cast<uint32_t*>(smem);
@@ -698,32 +833,41 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
         }
         const DevTensor& T = *s_tensor;
         const uint32_t first = (item - __ldg(item_start + cur)) * chunks_per_item;
-        const uint32_t count = min(chunks_per_item, T.n_chunks - first);
 
-        // the warps share out the item's chunks; each runs: fetch index (i + 2), copy (i + 1), decode (i)
+        // The warps share out the item's chunks.  Each warp, per turn: start the bulk copy of
+        // chunk i + 1 (its offsets arrived a turn ago), work out the lanes' positions in chunk
+        // i, ask for the index entries of chunk i + 2 in the slot that frees, decode chunk i.
         auto claim = [&]() -> uint32_t {
             uint32_t k = 0;
             if (lane == 0) k = atomicAdd(&s_claim[slot], 1u);
             k = __shfl_sync(0xffffffffu, k, 0);
-            return k < count ? first + k : kNone;
+            return k < min(chunks_per_item, T.n_chunks - first) ? first + k : kNone;
         };
         Ready r0;
         r0.c = kNone;
-        r0.pos = r0.my_bits = 0;
         r0.meta = ready_meta(0, 0, 0, kSkip);
-        Pending p2 = fetch_index(T, claim(), lane);
+        uint32_t sp = cx.idx_addr;                  // slot of the chunk fetched last
+        uint32_t c2 = claim();
+        fetch_index(T, c2, sp, lane);
         while (true) {
-            Ready r1 = prepare(cx, T, p2, r0, lane);
-            p2 = fetch_index(T, r1.c == kNone ? kNone : claim(), lane);
-            if (r0.c != kNone) decode_ready<K>(cx, T, r0, lane);
+            Ready r1 = prepare(cx, T, stage_bytes, status, c2, sp, r0, lane);
+            const uint32_t other = cx.idx_addr + (sp == cx.idx_addr ? kSlotBytes : 0u);
+            const Lane L = decode_start<K>(cx, status, r0, other, lane);
+            __syncwarp();                           // every lane has read the slot before it is refilled
+            c2 = r1.c == kNone ? kNone : claim();
+            fetch_index(T, c2, other, lane);
+            decode_finish<K>(cx, status, r0, L, lane);
             if (r1.c == kNone) break;
             r0 = r1;
+            sp = other;
         }
+        asm volatile("cp.async.wait_all;" ::: "memory");
         __syncthreads();   // tables may be replaced; s_item / s_claim [slot ^ 1] are now visible
         slot ^= 1u;
     }
     // A warp that gave up on a bulk copy lets it land (bounded) before its buffer goes away.
-    if (cx.dead && cx.tickets) (void)mbar_wait(cx.bar + 8u * ((cx.tickets - 1) & 1u), ((cx.tickets - 1) >> 1) & 1u);
+    const uint32_t issued = cx.state & 0x7fffffffu;
+    if (cx.dead() && issued) (void)mbar_wait(cx.bar + 8u * ((issued - 1) & 1u), ((issued - 1) >> 1) & 1u);
 }
 
 struct Shape {
@@ -735,7 +879,7 @@ struct Shape {
 Shape shape_for(const DecodeConfig& cfg, int max_smem)
 {
     size_t fixed = lut_bytes(cfg.lut_bits) + sizeof(DecodeAux) + sizeof(DevTensor) + 128 + kOverRead;
-    size_t per_warp_fixed = 16;   // two mbarriers
+    size_t per_warp_fixed = 16 + 2 * kSlotBytes;   // two mbarriers, two index slots
     size_t tail = 16;
     size_t budget = (size_t)max_smem / cfg.ctas_per_sm;
     if (cfg.ctas_per_sm > 1) budget -= 1024;   // per-CTA reservation of the driver

@@ -16,6 +16,7 @@ constexpr int kExpEntries = 32 << kExpBits;
 // Device status bits (OR-ed by kernels, read by entro_last_device_status).
 constexpr uint32_t kStatCorrupt = 1u;         // index / stream / codebook disagree
 constexpr uint32_t kStatTimeout = 2u;         // a bounded wait on a bulk copy ran out
+constexpr uint32_t kStatInternal = 4u;        // the kernel found its own assumptions about the device violated
 
 // One tensor as the decode kernels see it.
 struct DevTensor {

@@ -116,6 +116,7 @@ extern "C" entro_status entro_last_device_status(void* cuda_stream)
     ENTRO_CUDA(cudaMemcpyAsync(&st, ws->control + 1, sizeof(st), cudaMemcpyDeviceToHost, s));
     ENTRO_CUDA(cudaMemsetAsync(ws->control + 1, 0, sizeof(uint32_t), s));
     ENTRO_CUDA(cudaStreamSynchronize(s));
+    if (st & kStatInternal) return ENTRO_ERR_UNSUPPORTED;   // the device does not lay out shared memory as the kernel expects
     return st ? ENTRO_ERR_CORRUPT_STREAM : ENTRO_OK;
 }
 
