@@ -292,7 +292,7 @@ __device__ __forceinline__ uint32_t exp_lookup(uint32_t lane4, uint32_t inv_wind
 
 // One symbol from a full 32-bit window (true stream bits) by the canonical ranges; a pattern
 // that is no codeword is flagged and dropped as a single bit.  -> value << 16 | length.
-__device__ __noinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32_t window, uint32_t* status)
+__device__ __forceinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32_t window, uint32_t* status)
 {
     uint32_t len;
     uint32_t sym = range_decode(*aux, window, aux->max_len, len);
@@ -579,7 +579,7 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32
 
 // Any symbol count per lane, words fetched straight from global memory, scalar stores: the
 // ragged last chunk of a tensor, odd chunk sizes, chunks larger than the ring.
-__device__ __noinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t* status, const DevTensor& T, uint32_t c,
+__device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t* status, const DevTensor& T, uint32_t c,
                                                   uint32_t excl, uint32_t my_bits, uint32_t lane)
 {
     const uint64_t chunk_first = (uint64_t)c * T.chunk_symbols;
