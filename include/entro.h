@@ -194,6 +194,40 @@ entro_status entro_decode_dequant_batched_host(const entro_tensor_desc *descs_ho
                                                const entro_host_io *io_host, int ntensors,
                                                void *cuda_stream);
 
+/* The matrix-vector side of one tensor of entro_decode_dequant_gemv.  Host struct; the
+ * pointers inside are device pointers. */
+typedef struct {
+    uint32_t rows, cols;        /* W is [rows, cols] row-major, rows * cols = the tensor's n */
+    const void *x_fp16_dev;     /* cols fp16 values, 16-byte aligned */
+    void *y_fp16_dev;           /* rows fp16 results */
+} entro_gemv_io;
+
+/*
+ * Decode + dequantise + batch-1 matrix-vector product in one pass, without ever writing the
+ * fp16 weights: y[o] = fp16_rne( sum_i w_hat[o, i] * x[i] ), w_hat = fp16(s * (q - z)) as in
+ * entro_decode_dequant, products and sums in fp32.  This is the token-generation use of
+ * compressed weights: the paper attributes its generation speed-up to "reduced memory
+ * transfers during the memory-bandwidth-limited decoding phase" (Section 4, Table 3); here
+ * only the compressed stream crosses HBM.  descs_host[i].out_fp16_dev is not used and may be
+ * NULL.  All ntensors products are independent and run in one launch.  The order of the
+ * fp32 additions is not fixed (rows that span chunks are summed with atomics), so results
+ * can differ from run to run in the last bits before the final rounding.
+ * Limits: cols a multiple of 256 and at most 16384, chunk_symbols a multiple of 256
+ * (ENTRO_ERR_UNSUPPORTED otherwise).  Asynchronous; malformed input is reported through
+ * entro_last_device_status as for the decode calls.
+ */
+entro_status entro_decode_dequant_gemv(const entro_tensor_desc *descs_host, const entro_gemv_io *io_host,
+                                       int ntensors, void *cuda_stream);
+
+/*
+ * Plain fp16 matrix-vector product y = fp16_rne(W x), W [rows, cols] row-major fp16 on the
+ * device, fp32 products and sums: the step that follows an unfused decode, provided so that
+ * "decode, then multiply" can be timed against the fused call.  cols a multiple of 8; w and
+ * x 16-byte aligned.  Asynchronous.
+ */
+entro_status entro_gemv_fp16(const void *w_fp16_dev, uint32_t rows, uint32_t cols, const void *x_fp16_dev,
+                             void *y_fp16_dev, void *cuda_stream);
+
 /*
  * entro_decode_dequant_batched for callers that cannot allocate device memory.  (The paper
  * has no counterpart; this entry point exists for the sake of the host application.)

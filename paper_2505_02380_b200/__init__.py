@@ -68,6 +68,10 @@ class TensorDesc(C.Structure):
                 ("zero_point", C.c_int32), ("cb", Codebook), ("out_fp16_dev", C.c_void_p)]
 
 
+class GemvIO(C.Structure):
+    _fields_ = [("rows", C.c_uint32), ("cols", C.c_uint32), ("x_fp16_dev", C.c_void_p), ("y_fp16_dev", C.c_void_p)]
+
+
 class HostIO(C.Structure):
     _fields_ = [("stream_host", C.c_void_p), ("index_host", C.c_void_p), ("out_fp16_host", C.c_void_p)]
 
@@ -97,6 +101,8 @@ def lib():
         L.entro_decode_dequant.argtypes = [vp, u64, vp, u64, u32, C.POINTER(Codebook), C.c_float, C.c_int32, vp, vp]
         L.entro_decode_dequant_batched.argtypes = [C.POINTER(TensorDesc), i32, vp]
         L.entro_decode_dequant_batched_host.argtypes = [C.POINTER(TensorDesc), C.POINTER(HostIO), i32, vp]
+        L.entro_decode_dequant_gemv.argtypes = [C.POINTER(TensorDesc), C.POINTER(GemvIO), i32, vp]
+        L.entro_gemv_fp16.argtypes = [vp, u32, u32, vp, vp, vp]
         L.entro_decode_dequant_static.argtypes = [C.POINTER(TensorDesc), i32, vp, vp]
         L.entro_last_device_status.argtypes = [vp]
         L.entro_set_decode_config.argtypes = [i32, i32, i32, i32]
@@ -117,7 +123,7 @@ def lib():
 EXPORTS = ["entro_quantize_tensor", "entro_histogram", "entro_build_codebook", "entro_stream_words",
            "entro_encode_bound_words", "entro_index_bytes", "entro_encode", "entro_decode_dequant",
            "entro_decode_dequant_batched", "entro_decode_dequant_batched_host", "entro_decode_dequant_static",
-           "entro_last_device_status",
+           "entro_decode_dequant_gemv", "entro_gemv_fp16", "entro_last_device_status",
            "entro_set_decode_config", "entro_profile_begin", "entro_profile_read", "entro_kernel_launch_count",
            "entro_status_string"]
 
@@ -259,6 +265,49 @@ def entro_decode_dequant_batched_host(descs, io, stream: Optional[torch.cuda.Str
     """descs, io: ctypes arrays of TensorDesc / HostIO of equal length.  Synchronises."""
     _check(lib().entro_decode_dequant_batched_host(descs, io, len(descs), _stream(stream)),
            "entro_decode_dequant_batched_host")
+
+
+def make_desc_no_out(stream_words: torch.Tensor, index: torch.Tensor, n: int, chunk_symbols: int, cb: Codebook,
+                     scale: float, zero_point: int) -> TensorDesc:
+    """A descriptor for the fused matrix-vector call, which writes no fp16 weights."""
+    d = TensorDesc()
+    d.stream_dev = _dev(stream_words, torch.int32)
+    d.stream_words = stream_words.numel()
+    d.index_dev = _dev(index, torch.uint8)
+    d.n = n
+    d.chunk_symbols = chunk_symbols
+    d.scale = scale
+    d.zero_point = zero_point
+    d.cb = cb
+    d.out_fp16_dev = None
+    return d
+
+
+def entro_decode_dequant_gemv(descs, xs: Sequence[torch.Tensor], shapes: Sequence, ys: Optional[List[torch.Tensor]] = None,
+                              stream: Optional[torch.cuda.Stream] = None) -> List[torch.Tensor]:
+    """descs[i]: compressed W_i of shape shapes[i] = (rows, cols); xs[i]: fp16 vector of cols values.
+    -> fp16 vectors y_i = W_i x_i.  Asynchronous."""
+    if isinstance(descs, list):
+        descs = desc_array(descs)
+    n = len(descs)
+    if ys is None:
+        ys = [torch.empty(shapes[i][0], dtype=torch.float16, device=xs[i].device) for i in range(n)]
+    io = (GemvIO * n)()
+    for i in range(n):
+        io[i] = GemvIO(int(shapes[i][0]), int(shapes[i][1]), _dev(xs[i], torch.float16), _dev(ys[i], torch.float16))
+    _check(lib().entro_decode_dequant_gemv(descs, io, n, _stream(stream)), "entro_decode_dequant_gemv")
+    return ys
+
+
+def entro_gemv_fp16(w: torch.Tensor, x: torch.Tensor, y: Optional[torch.Tensor] = None,
+                    stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """y = W x for an fp16 matrix W [rows, cols] on the device (fp32 accumulation).  Asynchronous."""
+    rows, cols = w.shape
+    if y is None:
+        y = torch.empty(rows, dtype=torch.float16, device=w.device)
+    _check(lib().entro_gemv_fp16(_dev(w, torch.float16), rows, cols, _dev(x, torch.float16), _dev(y, torch.float16),
+                                 _stream(stream)), "entro_gemv_fp16")
+    return y
 
 
 def entro_decode_dequant_static(descs, status: Optional[torch.Tensor] = None,

@@ -462,6 +462,17 @@ __device__ __forceinline__ DevTensor* tensor_ptr()
     return reinterpret_cast<DevTensor*>(smem + lut_bytes(K) + sizeof(DecodeAux));
 }
 
+// The matrix-vector kernel keeps two more things behind the tensor: its GemvTensor and x.
+template <int K>
+constexpr uint32_t kGemvDesc = lut_bytes(K) + (uint32_t)sizeof(DecodeAux) + (uint32_t)sizeof(DevTensor);
+template <int K>
+constexpr uint32_t kGemvX = kGemvDesc<K> + (uint32_t)sizeof(GemvTensor);
+template <int K>
+__device__ __forceinline__ GemvTensor* gemv_ptr() { return reinterpret_cast<GemvTensor*>(smem + kGemvDesc<K>); }
+// Offset of the first ring.
+template <int K, bool kGemv>
+constexpr uint32_t kRingsAt = ((kGemv ? kGemvX<K> + 2u * kGemvMaxCols : kGemvDesc<K>) + 127u) & ~127u;
+
 // What a warp carries from chunk to chunk (kept small: it lives in registers across the
 // decode loop).
 struct WarpCtx {
@@ -577,10 +588,12 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32
     return r;
 }
 
-// Any symbol count per lane, words fetched straight from global memory, scalar stores: the
-// ragged last chunk of a tensor, odd chunk sizes, chunks larger than the ring.
-__device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t* status, const DevTensor& T, uint32_t c,
-                                                  uint32_t excl, uint32_t my_bits, uint32_t lane)
+// Any symbol count per lane, words fetched straight from global memory, one value at a
+// time: the ragged last chunk of a tensor, odd chunk sizes, chunks larger than the ring.
+// With G set the values are not stored but multiplied into the matrix-vector product.
+__device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t* status, const DevTensor& T,
+                                                     const GemvTensor* G, uint32_t c, uint32_t excl, uint32_t my_bits,
+                                                     uint32_t lane)
 {
     const uint64_t chunk_first = (uint64_t)c * T.chunk_symbols;
     const uint32_t m = (uint32_t)min((uint64_t)T.chunk_symbols, T.n - chunk_first);   // symbols in the chunk
@@ -600,6 +613,7 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
     // this lane's symbols: groups lane, lane + 32, ... of 8 consecutive symbols
     for (uint32_t g = lane; g * 8u < m; g += kSubBlocks) {
         const uint32_t end = min(g * 8u + 8u, m);
+        float acc = 0.f;
         for (uint32_t i = g * 8u; i < end; ++i) {
             gwin_refill(r);
             uint32_t e = kEscLen;
@@ -609,19 +623,91 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
             r.hi = __funnelshift_lc(r.lo, r.hi, n);
             r.lo = __funnelshift_lc(0u, r.lo, n);
             r.nb -= (int)n;
-            out[i] = (uint16_t)(e >> 16);
+            if (G) {
+                const uint32_t col = (uint32_t)((chunk_first + i) % G->cols);
+                acc = fmaf(__half2float(__ushort_as_half((uint16_t)(e >> 16))),
+                           __half2float(__ushort_as_half(__ldg(G->x + col))), acc);
+            } else {
+                out[i] = (uint16_t)(e >> 16);
+            }
         }
+        // a group of 8 lies inside one row (cols is a multiple of 8)
+        if (G) atomicAdd(G->y32 + (chunk_first + g * 8u) / G->cols, acc);
     }
     const uint64_t used = ((uint64_t)r.next << 5) - (uint64_t)r.nb - bit;
     if (used != my_bits) atomicOr(status, kStatCorrupt);
 }
 
-// 8-bit alphabets: G lookups per window refill (group4 / group2 above).
-// dst: this lane's first group; consecutive groups of a lane are 32 groups apart.
-template <int K, int G>
-__device__ __forceinline__ void rows_single(Win& r, uint32_t* status, uint32_t lane4, uint4* dst, uint32_t sub)
+// ------------------------------------------------------------------ what happens to decoded values
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
 {
-    for (uint32_t t0 = 0; t0 < sub; t0 += 8, dst += kSubBlocks) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// Plain decode: the 8 values of this lane's next group go to the output tensor.  A lane's
+// consecutive groups are 32 groups apart, so one call per lane writes 512 contiguous bytes.
+struct EmitStore {
+    uint4* dst;
+    __device__ __forceinline__ void operator()(uint4 v)
+    {
+        __stcs(dst, v);
+        dst += kSubBlocks;
+    }
+    __device__ __forceinline__ void finish() {}
+};
+
+// Fused matrix-vector product: the 8 values are weights of one row of W (stored [rows, cols],
+// cols a multiple of 256, so the 32 lanes of a step stay inside one row) and meet the 8
+// matching entries of x, staged in shared memory as fp16; products and sums in fp32.  When
+// the row ends the warp adds its lanes up and adds the result to the row's fp32 accumulator.
+struct EmitDot {
+    uint32_t xaddr;       // shared-window address of x[col .. col + 8) for this lane's next group
+    uint32_t xlane;       // the same at the start of a row
+    uint32_t left;        // steps left in the current row
+    uint32_t rs;          // steps per row (cols / 256)
+    float acc;
+    float* yrow;          // fp32 accumulator of the current row
+    uint32_t lane;
+
+    __device__ __forceinline__ void flush()
+    {
+        float v = acc;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+        if (lane == 0) atomicAdd(yrow, v);
+        acc = 0.f;
+        ++yrow;
+        left = rs;
+        xaddr = xlane;
+    }
+    __device__ __forceinline__ void operator()(uint4 w)
+    {
+        const uint4 x = lds128(xaddr);
+        const uint32_t wv[4] = {w.x, w.y, w.z, w.w}, xv[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&wv[i]));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&xv[i]));
+            acc = fmaf(a.x, b.x, acc);
+            acc = fmaf(a.y, b.y, acc);
+        }
+        xaddr += 512u;
+        if (--left == 0u) flush();
+    }
+    __device__ __forceinline__ void finish()
+    {
+        if (left != rs) flush();     // the chunk ended inside a row
+    }
+};
+
+// 8-bit alphabets: G lookups per window refill (group4 / group2 above).
+template <int K, int G, class Emit>
+__device__ __forceinline__ void rows_single(Win& r, uint32_t* status, uint32_t lane4, Emit& emit, uint32_t sub)
+{
+    for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
         uint32_t pk[4];
         if (G == 4) {
 #pragma unroll
@@ -641,22 +727,22 @@ __device__ __forceinline__ void rows_single(Win& r, uint32_t* status, uint32_t l
                 }
             }
         }
-        __stcs(dst, make_uint4(pk[0], pk[1], pk[2], pk[3]));
+        emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
     }
 }
 
 // 4-bit alphabets: eight symbols per lookup.
-template <int K>
-__device__ __forceinline__ void rows_oct(Win& r, uint32_t* status, uint4* dst, uint32_t sub)
+template <int K, class Emit>
+__device__ __forceinline__ void rows_oct(Win& r, uint32_t* status, Emit& emit, uint32_t sub)
 {
-    for (uint32_t t0 = 0; t0 < sub; t0 += 8, dst += kSubBlocks) {
+    for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
         win_refill<false>(r);
         const uint32_t idx = r.hi >> (32 - K);
         uint4 v = *reinterpret_cast<const uint4*>(smem + idx * 16u);
         const uint32_t n = *(smem + (16u << K) + idx);
         if (__builtin_expect(n == 0u, 0)) v = repair_oct<K>(r, status);
         else win_skip(r, n);
-        __stcs(dst, v);
+        emit(v);
     }
 }
 
@@ -703,11 +789,12 @@ __device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status
     return L;
 }
 
-template <int K>
+template <int K, bool kGemv>
 __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Ready& r, Lane L, uint32_t lane)
 {
     if (L.kind == kSkip) return;
     const DevTensor& T = *tensor_ptr<K>();
+    const GemvTensor* G = kGemv ? gemv_ptr<K>() : nullptr;
     if (L.kind == kStaged) {
         if (!r.issued()) issue_copy(cx, T, r, (T.offsets[r.c] >> 3) & ~15ull, lane);
         bool ok = mbar_wait(cx.bar + 8u * (r.ticket() & 1u), (r.ticket() >> 1) & 1u);
@@ -723,19 +810,37 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         }
     }
     if (L.kind == kGeneral) {
-        decode_chunk_general(aux_ptr<K>(), status, T, r.c, L.start, L.end, lane);
+        decode_chunk_general(aux_ptr<K>(), status, T, G, r.c, L.start, L.end, lane);
         return;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    uint4* dst = reinterpret_cast<uint4*>(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
     Win w;
-    if (aux_ptr<K>()->oct) {
-        win_init<false>(w, (L.start >> 5) << 2, L.start & 31u);
-        rows_oct<K>(w, status, dst, sub);
+    const bool oct = aux_ptr<K>()->oct != 0;
+    if (oct) win_init<false>(w, (L.start >> 5) << 2, L.start & 31u);
+    else win_init<true>(w, (L.start >> 5) << 2, L.start & 31u);
+    if (kGemv) {
+        // the chunk starts gs0 steps of 256 weights into the matrix; a row is rs steps long
+        const uint32_t rs = G->cols >> 8;
+        const uint32_t gs0 = (uint32_t)(((uint64_t)r.c * T.chunk_symbols) >> 8);
+        const uint32_t row0 = gs0 / rs, k0 = gs0 - row0 * rs;
+        EmitDot em;
+        em.lane = lane;
+        em.rs = rs;
+        em.left = rs - k0;
+        em.xlane = kSmemBase + kGemvX<K> + lane * 16u;
+        em.xaddr = em.xlane + k0 * 512u;
+        em.acc = 0.f;
+        em.yrow = G->y32 + row0;
+        if (oct) rows_oct<K>(w, status, em, sub);
+        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lane * 4u, em, sub);
+        else rows_single<K, 2>(w, status, lane * 4u, em, sub);
+        em.finish();
     } else {
-        win_init<true>(w, (L.start >> 5) << 2, L.start & 31u);
-        if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lane * 4u, dst, sub);
-        else rows_single<K, 2>(w, status, lane * 4u, dst, sub);
+        EmitStore em;
+        em.dst = reinterpret_cast<uint4*>(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
+        if (oct) rows_oct<K>(w, status, em, sub);
+        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lane * 4u, em, sub);
+        else rows_single<K, 2>(w, status, lane * 4u, em, sub);
     }
     // the lane must stand exactly at the end of its sub-block
     if (w.next * 8u - (uint32_t)win_valid_bits(w.k) != L.end) atomicOr(status, kStatCorrupt);
@@ -746,14 +851,17 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
 
 // item_start[t] = first work item of tensor t, item_start[ntensors] = number of items; an
 // item is up to chunks_per_item consecutive chunks of one tensor.
-template <int K>
+// With kGemv the decoded weights are not stored: gemv[t] describes the matrix-vector product
+// they enter (the fused decode + dequantise + GEMV of a batch-1 token step).
+template <int K, bool kGemv>
 __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __restrict__ tensors, int ntensors,
                                                          const uint32_t* __restrict__ item_start,
                                                          const TensorTables* __restrict__ tables,
                                                          uint32_t chunks_per_item, uint32_t stage_bytes,
-                                                         uint32_t* __restrict__ control)
+                                                         uint32_t* __restrict__ control,
+                                                         const GemvTensor* __restrict__ gemv)
 {
-    // layout: [tables][aux][tensor][per-warp rings][over-read pad][mbarriers][index slots][item + claim slots]
+    // layout: [tables][aux][tensor]([gemv descriptor][x])[per-warp rings][over-read pad][mbarriers][index slots][item + claim slots]
     if (smem_addr(smem) != kSmemBase) {   // the lookups' address arithmetic would be wrong: refuse to run
         if (threadIdx.x == 0) atomicOr(control + 1, kStatInternal);
         return;
@@ -762,7 +870,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     DevTensor* s_tensor = tensor_ptr<K>();
     const uint32_t warps = blockDim.x >> 5;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr uint32_t kRings = (lut_bytes(K) + (uint32_t)sizeof(DecodeAux) + (uint32_t)sizeof(DevTensor) + 127u) & ~127u;
+    constexpr uint32_t kRings = kRingsAt<K, kGemv>;
     const uint32_t after = kRings + warps * stage_bytes + kOverRead;          // offset in smem, a multiple of 16
     const uint32_t slots = after + warps * 16u;
     volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(smem + slots + warps * 2u * kSlotBytes);   // [2]
@@ -814,6 +922,15 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             const uint4* gt = reinterpret_cast<const uint4*>(tensors + cur);
             uint4* st = reinterpret_cast<uint4*>(s_tensor);
             for (uint32_t i = threadIdx.x; i < sizeof(DevTensor) / 16; i += blockDim.x) st[i] = __ldg(gt + i);
+            if (kGemv) {
+                const uint4* gg = reinterpret_cast<const uint4*>(gemv + cur);
+                uint4* sg = reinterpret_cast<uint4*>(gemv_ptr<K>());
+                if (threadIdx.x < sizeof(GemvTensor) / 16) sg[threadIdx.x] = __ldg(gg + threadIdx.x);
+                const uint4* gx = reinterpret_cast<const uint4*>(gemv[cur].x);      // cols is a multiple of 256
+                uint4* sx = reinterpret_cast<uint4*>(smem + kGemvX<K>);
+                const uint32_t n16 = gemv[cur].cols / 8u;
+                for (uint32_t i = threadIdx.x; i < n16; i += blockDim.x) sx[i] = __ldg(gx + i);
+            }
             if (__ldg(&tt->aux.oct)) {
                 const uint4* g1 = tt->oct_val;
                 uint4* s1 = reinterpret_cast<uint4*>(smem);
@@ -856,7 +973,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             __syncwarp();                           // every lane has read the slot before it is refilled
             c2 = r1.c == kNone ? kNone : claim();
             fetch_index(T, c2, other, lane);
-            decode_finish<K>(cx, status, r0, L, lane);
+            decode_finish<K, kGemv>(cx, status, r0, L, lane);
             if (r1.c == kNone) break;
             r0 = r1;
             sp = other;
@@ -876,9 +993,10 @@ struct Shape {
 };
 
 // Shared memory of one CTA for a launch shape; stage_bytes == 0 if it cannot fit.
-Shape shape_for(const DecodeConfig& cfg, int max_smem)
+Shape shape_for(const DecodeConfig& cfg, int max_smem, bool gemv = false)
 {
     size_t fixed = lut_bytes(cfg.lut_bits) + sizeof(DecodeAux) + sizeof(DevTensor) + 128 + kOverRead;
+    if (gemv) fixed += sizeof(GemvTensor) + 2 * kGemvMaxCols;
     size_t per_warp_fixed = 16 + 2 * kSlotBytes;   // two mbarriers, two index slots
     size_t tail = 16;
     size_t budget = (size_t)max_smem / cfg.ctas_per_sm;
@@ -893,48 +1011,57 @@ Shape shape_for(const DecodeConfig& cfg, int max_smem)
     return s;
 }
 
-template <int K>
+template <int K, bool kGemv>
 entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
                            const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
-                           cudaStream_t s)
+                           const GemvTensor* gemv, cudaStream_t s)
 {
-    Shape sh = shape_for(cfg, ws->max_smem_optin);
+    Shape sh = shape_for(cfg, ws->max_smem_optin, kGemv);
     if (sh.stage_bytes == 0) return ENTRO_ERR_UNSUPPORTED;
     static int configured_smem[64] = {0};
     if ((int)sh.smem > configured_smem[ws->device]) {
-        ENTRO_CUDA(cudaFuncSetAttribute(decode_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh.smem));
+        ENTRO_CUDA(cudaFuncSetAttribute(decode_kernel<K, kGemv>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sh.smem));
         configured_smem[ws->device] = (int)sh.smem;
     }
     uint32_t grid = (uint32_t)ws->sm_count * cfg.ctas_per_sm;
     if (grid > total_items) grid = total_items;
     const bool timed = ws->prof_used < ws->prof_cap;
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_start[ws->prof_used], s));
-    decode_kernel<K><<<grid, cfg.warps_per_cta * 32, sh.smem, s>>>(tensors, ntensors, item_start, tables,
-                                                                   (uint32_t)cfg.chunks_per_item, sh.stage_bytes,
-                                                                   ws->control);
+    decode_kernel<K, kGemv><<<grid, cfg.warps_per_cta * 32, sh.smem, s>>>(
+        tensors, ntensors, item_start, tables, (uint32_t)cfg.chunks_per_item, sh.stage_bytes, ws->control, gemv);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_stop[ws->prof_used++], s));
     return ENTRO_OK;
 }
 
+// gemv == nullptr: plain decode.
 entro_status launch_decode_any(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
                                const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
-                               cudaStream_t s)
+                               cudaStream_t s, const GemvTensor* gemv = nullptr)
 {
+    if (gemv) {
+        switch (cfg.lut_bits) {
+            case 10: return launch_decode<10, true>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
+            case 11: return launch_decode<11, true>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
+            case 12: return launch_decode<12, true>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
+        }
+        return ENTRO_ERR_UNSUPPORTED;
+    }
     switch (cfg.lut_bits) {
-        case 10: return launch_decode<10>(ws, cfg, tensors, ntensors, item_start, total_items, tables, s);
-        case 11: return launch_decode<11>(ws, cfg, tensors, ntensors, item_start, total_items, tables, s);
-        case 12: return launch_decode<12>(ws, cfg, tensors, ntensors, item_start, total_items, tables, s);
+        case 10: return launch_decode<10, false>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
+        case 11: return launch_decode<11, false>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
+        case 12: return launch_decode<12, false>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
     }
     return ENTRO_ERR_UNSUPPORTED;
 }
 
-entro_status validate_desc(const entro_tensor_desc& d)
+entro_status validate_desc(const entro_tensor_desc& d, bool need_out = true)
 {
     if (d.n == 0) return ENTRO_OK;
-    if (!d.stream_dev || !d.index_dev || !d.out_fp16_dev) return ENTRO_ERR_INVALID_ARG;
-    if (!aligned(d.stream_dev, 16) || !aligned(d.index_dev, 8) || !aligned(d.out_fp16_dev, 16))
+    if (!d.stream_dev || !d.index_dev || (need_out && !d.out_fp16_dev)) return ENTRO_ERR_INVALID_ARG;
+    if (!aligned(d.stream_dev, 16) || !aligned(d.index_dev, 8) || (need_out && !aligned(d.out_fp16_dev, 16)))
         return ENTRO_ERR_INVALID_ARG;
     if (d.chunk_symbols < kSubBlocks || d.chunk_symbols % kSubBlocks || d.chunk_symbols > ENTRO_MAX_CHUNK_SYMBOLS)
         return ENTRO_ERR_INVALID_ARG;
@@ -1080,6 +1207,143 @@ extern "C" entro_status entro_decode_dequant_batched_host(const entro_tensor_des
         ENTRO_CUDA(cudaMemcpyAsync(io[i].out_fp16_host, d.out_fp16_dev, d.n * 2, cudaMemcpyDeviceToHost, s));
     }
     ENTRO_CUDA(cudaStreamSynchronize(s));
+    return ENTRO_OK;
+}
+
+// ------------------------------------------------------------------ matrix-vector products
+
+namespace entro {
+namespace {
+
+// y = fp16(y32) for every tensor of a fused call.
+__global__ void __launch_bounds__(256) gemv_finalize_kernel(const GemvTensor* __restrict__ g, int ntensors)
+{
+    for (int t = blockIdx.y; t < ntensors; t += gridDim.y) {
+        const GemvTensor G = g[t];
+        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < G.rows; i += gridDim.x * blockDim.x)
+            G.y[i] = __half_as_ushort(__float2half_rn(G.y32[i]));
+    }
+}
+
+// Plain fp16 matrix-vector product (the step that follows an unfused decode): one warp per
+// row, 16-byte loads, fp32 products and sums, x read through the read-only path.
+__global__ void __launch_bounds__(256) gemv_fp16_kernel(const uint16_t* __restrict__ w, uint32_t rows, uint32_t cols,
+                                                        const uint16_t* __restrict__ x, uint16_t* __restrict__ y)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
+    for (uint32_t r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < rows; r += warps) {
+        const uint4* wr = reinterpret_cast<const uint4*>(w + (uint64_t)r * cols);
+        const uint4* xr = reinterpret_cast<const uint4*>(x);
+        float acc = 0.f;
+        for (uint32_t i = lane; i < cols / 8u; i += 32u) {
+            const uint4 a = __ldcs(wr + i), b = __ldg(xr + i);
+            const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&av[k]));
+                const float2 q = __half22float2(*reinterpret_cast<const __half2*>(&bv[k]));
+                acc = fmaf(p.x, q.x, acc);
+                acc = fmaf(p.y, q.y, acc);
+            }
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+        if (lane == 0) y[r] = __half_as_ushort(__float2half_rn(acc));
+    }
+}
+
+}  // namespace
+}  // namespace entro
+
+extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs_host, const entro_gemv_io* io_host,
+                                                  int ntensors, void* cuda_stream)
+{
+    if (ntensors < 0 || (ntensors > 0 && (!descs_host || !io_host))) return ENTRO_ERR_INVALID_ARG;
+    if (ntensors == 0) return ENTRO_OK;
+    uint64_t total_rows = 0;
+    for (int i = 0; i < ntensors; ++i) {
+        const entro_tensor_desc& d = descs_host[i];
+        const entro_gemv_io& g = io_host[i];
+        if (d.n == 0) return ENTRO_ERR_INVALID_ARG;
+        entro_status st = validate_desc(d, false);
+        if (st != ENTRO_OK) return st;
+        if (!g.x_fp16_dev || !g.y_fp16_dev || !aligned(g.x_fp16_dev, 16) || !aligned(g.y_fp16_dev, 2))
+            return ENTRO_ERR_INVALID_ARG;
+        if (g.rows == 0 || g.cols == 0 || (uint64_t)g.rows * g.cols != d.n) return ENTRO_ERR_INVALID_ARG;
+        if (g.cols % 256u || g.cols > kGemvMaxCols || d.chunk_symbols % 256u) return ENTRO_ERR_UNSUPPORTED;
+        total_rows += g.rows;
+    }
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    Guard guard;
+    Workspace* ws = workspace();
+    if (!ws) return ENTRO_ERR_CUDA;
+    const DecodeConfig cfg = decode_config();
+
+    // workspace: [DevTensor x n][item_start][GemvTensor x n] (uploaded) [tables x n][y32]
+    const size_t tensors_bytes = (size_t)ntensors * sizeof(DevTensor);
+    const size_t items_bytes = (((size_t)ntensors + 1) * 4 + 15) & ~(size_t)15;
+    const size_t gemv_bytes = (size_t)ntensors * sizeof(GemvTensor);
+    const size_t upload_bytes = tensors_bytes + items_bytes + gemv_bytes;
+    const size_t tables_bytes = (size_t)ntensors * sizeof(TensorTables);
+    const size_t y32_bytes = (total_rows * 4 + 15) & ~(size_t)15;
+    if (!reserve_pinned(ws, upload_bytes)) return ENTRO_ERR_CUDA;
+    if (!reserve_device(ws, upload_bytes + tables_bytes + y32_bytes)) return ENTRO_ERR_CUDA;
+    char* base = static_cast<char*>(ws->dev);
+    char* hbase = static_cast<char*>(ws->pinned);
+    DevTensor* ht = reinterpret_cast<DevTensor*>(hbase);
+    uint32_t* hitems = reinterpret_cast<uint32_t*>(hbase + tensors_bytes);
+    GemvTensor* hg = reinterpret_cast<GemvTensor*>(hbase + tensors_bytes + items_bytes);
+    float* y32 = reinterpret_cast<float*>(base + upload_bytes + tables_bytes);
+    uint64_t items = 0, row0 = 0;
+    for (int i = 0; i < ntensors; ++i) {
+        hitems[i] = (uint32_t)items;
+        items += fill_dev_tensor(descs_host[i], cfg, ht[i]);
+        if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
+        hg[i].x = static_cast<const uint16_t*>(io_host[i].x_fp16_dev);
+        hg[i].y32 = y32 + row0;
+        hg[i].y = static_cast<uint16_t*>(io_host[i].y_fp16_dev);
+        hg[i].rows = io_host[i].rows;
+        hg[i].cols = io_host[i].cols;
+        row0 += io_host[i].rows;
+    }
+    hitems[ntensors] = (uint32_t)items;
+    DevTensor* dt = reinterpret_cast<DevTensor*>(base);
+    uint32_t* ditems = reinterpret_cast<uint32_t*>(base + tensors_bytes);
+    GemvTensor* dg = reinterpret_cast<GemvTensor*>(base + tensors_bytes + items_bytes);
+    TensorTables* dtables = reinterpret_cast<TensorTables*>(base + upload_bytes);
+    ENTRO_CUDA(cudaMemcpyAsync(dt, ht, upload_bytes, cudaMemcpyHostToDevice, s));
+    mark_pinned_in_use(ws, s);
+    ENTRO_CUDA(cudaMemsetAsync(y32, 0, y32_bytes, s));
+    build_tables_kernel<<<ntensors, 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
+    count_launch();
+    ENTRO_CUDA(cudaGetLastError());
+    entro_status st = launch_decode_any(ws, cfg, dt, ntensors, ditems, (uint32_t)items, dtables, s, dg);
+    if (st != ENTRO_OK) return st;
+    dim3 grid(16, (unsigned)(ntensors < 64 ? ntensors : 64));
+    gemv_finalize_kernel<<<grid, 256, 0, s>>>(dg, ntensors);
+    count_launch();
+    ENTRO_CUDA(cudaGetLastError());
+    return ENTRO_OK;
+}
+
+extern "C" entro_status entro_gemv_fp16(const void* w_fp16_dev, uint32_t rows, uint32_t cols, const void* x_fp16_dev,
+                                        void* y_fp16_dev, void* cuda_stream)
+{
+    if (!w_fp16_dev || !x_fp16_dev || !y_fp16_dev || rows == 0 || cols == 0) return ENTRO_ERR_INVALID_ARG;
+    if (cols % 8u || !aligned(w_fp16_dev, 16) || !aligned(x_fp16_dev, 16) || !aligned(y_fp16_dev, 2))
+        return ENTRO_ERR_INVALID_ARG;
+    int dev = 0, sms = 0;
+    ENTRO_CUDA(cudaGetDevice(&dev));
+    ENTRO_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    unsigned blocks = (rows + 7u) / 8u;
+    const unsigned cap = (unsigned)sms * 8u;
+    if (blocks > cap) blocks = cap;
+    gemv_fp16_kernel<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>(
+        static_cast<const uint16_t*>(w_fp16_dev), rows, cols, static_cast<const uint16_t*>(x_fp16_dev),
+        static_cast<uint16_t*>(y_fp16_dev));
+    count_launch();
+    ENTRO_CUDA(cudaGetLastError());
     return ENTRO_OK;
 }
 

@@ -36,6 +36,16 @@ struct DevTensor {
 };
 static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vectors");
 
+// The matrix-vector side of one tensor for the fused decode + GEMV kernel.
+struct GemvTensor {
+    const uint16_t* x;    // cols fp16 values
+    float* y32;           // rows fp32 accumulators (workspace), zero before the kernel
+    uint16_t* y;          // rows fp16 results
+    uint32_t rows, cols;
+};
+static_assert(sizeof(GemvTensor) == 32, "GemvTensor is read as two 16-byte vectors");
+constexpr uint32_t kGemvMaxCols = 16384;      // x is staged in shared memory as fp16
+
 // Per-tensor canonical-code description beside the lookup tables.
 struct DecodeAux {
     unsigned long long limit[ENTRO_MAX_CODE_LEN + 1];  // left-justified end of the codes of length <= l

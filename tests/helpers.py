@@ -40,4 +40,5 @@ def expected_out(c: oracle.Compressed) -> np.ndarray:
 
 
 def assert_status_ok():
-    assert E.entro_last_device_status() == E.OK
+    st = E.entro_last_device_status()
+    assert st == E.OK, E.status_string(st)
