@@ -235,6 +235,76 @@ def time_e2e(E, model, steps, warmup):
     return ms, h2d, d2h
 
 
+def measure_gemv(E, max_layers, reps=5):
+    """Config 5: mistral-7B-shaped 4-bit layer stack, batch-1 fp16 GEMV per projection.  Fused
+    (decode + dequant + GEMV, one call per layer) against unfused (decode the layer to fp16,
+    then seven plain fp16 GEMVs)."""
+    wl = workloads.mistral_layer_stack(max_layers=max_layers)
+    layers = {}
+    for spec in wl.tensors:
+        layers.setdefault(spec.name.split(".")[1], []).append(spec)
+    keep, per_layer, comp_bytes, n_weights = [], [], 0, 0
+    biggest = max(sum(t.numel for t in specs) for specs in layers.values())
+    scratch = torch.empty(biggest, dtype=torch.float16, device="cuda")
+    for name, specs in layers.items():
+        descs_f, descs_u, xs, ys, shapes, views = [], [], [], [], [], []
+        pos = 0
+        for k, spec in enumerate(specs):
+            w = workloads.make_tensor(spec, "cuda").view(-1)
+            q, qp = E.entro_quantize_tensor(w, wl.bits)
+            counts = E.entro_histogram(q, wl.bits)
+            cb = E.entro_build_codebook(counts.tolist())
+            enc = E.entro_encode(q, cb, wl.chunk_symbols, stream_words=E.entro_stream_words(counts.tolist(), cb))
+            del w, q
+            keep.append(enc)
+            out = scratch[pos:pos + spec.numel]
+            pos += spec.numel
+            descs_f.append(E.make_desc_no_out(enc.stream, enc.index, spec.numel, wl.chunk_symbols, cb, qp.scale,
+                                              qp.zero_point))
+            descs_u.append(E.make_desc(enc.stream, enc.index, spec.numel, wl.chunk_symbols, cb, qp.scale,
+                                       qp.zero_point, out))
+            xs.append(workloads.make_vector(spec.cols, 1000 + k).cuda())
+            ys.append(torch.empty(spec.rows, dtype=torch.float16, device="cuda"))
+            shapes.append((spec.rows, spec.cols))
+            views.append(out.view(spec.rows, spec.cols))
+            comp_bytes += (enc.total_bits + 7) // 8 + enc.index.numel() + 2 * (spec.rows + spec.cols)
+            n_weights += spec.numel
+        per_layer.append((E.desc_array(descs_f), E.desc_array(descs_u), xs, ys, shapes, views))
+
+    def fused():
+        for df, du, xs, ys, shapes, views in per_layer:
+            E.entro_decode_dequant_gemv(df, xs, shapes, ys)
+
+    def unfused():
+        for df, du, xs, ys, shapes, views in per_layer:
+            E.entro_decode_dequant_batched(du)
+            for v, x, y in zip(views, xs, ys):
+                E.entro_gemv_fp16(v, x, y)
+
+    out = {}
+    for name, fn in (("fused", fused), ("unfused", unfused)):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(reps):
+            fn()
+        ev1.record()
+        torch.cuda.synchronize()
+        assert E.entro_last_device_status() == E.OK
+        out[name] = ev0.elapsed_time(ev1) / reps
+    nl = len(per_layer)
+    return {"workload": wl.name, "layers": nl, "weights": n_weights,
+            "fused_ms_per_layer": out["fused"] / nl, "unfused_ms_per_layer": out["unfused"] / nl,
+            "speedup_fused_vs_unfused": out["unfused"] / out["fused"],
+            "weights_per_s": n_weights / (out["fused"] * 1e-3),
+            "effective_GBs_compressed_in_plus_xy": comp_bytes / (out["fused"] * 1e-3) / 1e9,
+            "fp16_equivalent_GBs": 2.0 * n_weights / (out["fused"] * 1e-3) / 1e9,
+            "note": "fused: one launch per layer over its 7 projections; unfused: decode to fp16 then 7 fp16 GEMVs; "
+                    "the fused pass is bound by decode issue rate, not by HBM (0.14 B/weight read)"}
+
+
 # ----------------------------------------------------------------------------- CPU oracle legs
 
 def oracle_sample(wl, max_symbols):
@@ -353,6 +423,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-gemv", action="store_true", help="skip the fused decode+GEMV section (config 5)")
     ap.add_argument("--lut-bits", type=int, default=0)
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
@@ -393,6 +464,11 @@ def main():
                 **{k: r2[k] for k in ("value", "ms_per_step", "weights_per_s", "bytes_per_step", "bits_per_weight",
                                        "max_code_len", "roofline", "clocks")}}
 
+    gemv = None
+    if not args.no_gemv and rank == 0 and world == 1:
+        torch.cuda.empty_cache()
+        gemv = measure_gemv(E, args.max_layers)
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": main_res["value"], "unit": "GB/s", "n_gpus": world, "steps": args.steps,
@@ -416,6 +492,8 @@ def main():
             line["cpu_baseline"] = main_res["cpu_baseline"]
         if also:
             line["also"] = also
+        if gemv:
+            line["gemv"] = gemv
         line["paper_context"] = ("paper: 6.66 s (uint8) / 1.66 s (uint4) to decode phi3-mini-4k on a Jetson P3450, "
                                  "4 CPU threads, integer output (Table 3) -- other hardware, context only")
         print(json.dumps(line))

@@ -1071,6 +1071,21 @@ entro_status validate_desc(const entro_tensor_desc& d, bool need_out = true)
     return ENTRO_OK;
 }
 
+// Work items small enough that a launch with few chunks (one layer, one tensor) still gives
+// every CTA several of them: at most the configured size, at least one chunk per warp.
+DecodeConfig item_size_for(DecodeConfig cfg, const entro_tensor_desc* descs, int ntensors, int sm_count)
+{
+    uint64_t chunks = 0;
+    for (int i = 0; i < ntensors; ++i)
+        if (descs[i].n) chunks += num_chunks(descs[i].n, descs[i].chunk_symbols);
+    const uint64_t ctas = (uint64_t)sm_count * cfg.ctas_per_sm;
+    uint64_t want = (chunks + ctas * 4 - 1) / (ctas * 4);
+    want = (want + cfg.warps_per_cta - 1) / cfg.warps_per_cta * cfg.warps_per_cta;
+    if (want < (uint64_t)cfg.warps_per_cta) want = cfg.warps_per_cta;
+    if (want < (uint64_t)cfg.chunks_per_item) cfg.chunks_per_item = (int)want;
+    return cfg;
+}
+
 // Device-side form of a descriptor; returns the tensor's number of work items.
 uint64_t fill_dev_tensor(const entro_tensor_desc& d, const DecodeConfig& cfg, DevTensor& t)
 {
@@ -1096,7 +1111,7 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, const DecodeConfig& cfg, De
 // Upload descriptors, build the tables and run the persistent decode kernel.
 entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs, int ntensors, cudaStream_t s)
 {
-    const DecodeConfig cfg = decode_config();
+    const DecodeConfig cfg = item_size_for(decode_config(), descs, ntensors, ws->sm_count);
     int live = 0;
     for (int i = 0; i < ntensors; ++i) {
         entro_status st = validate_desc(descs[i]);
@@ -1278,7 +1293,7 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
     Guard guard;
     Workspace* ws = workspace();
     if (!ws) return ENTRO_ERR_CUDA;
-    const DecodeConfig cfg = decode_config();
+    const DecodeConfig cfg = item_size_for(decode_config(), descs_host, ntensors, ws->sm_count);
 
     // workspace: [DevTensor x n][item_start][GemvTensor x n] (uploaded) [tables x n][y32]
     const size_t tensors_bytes = (size_t)ntensors * sizeof(DevTensor);
@@ -1437,7 +1452,7 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
         if (status_dev) ENTRO_CUDA(cudaMemsetAsync(status_dev, 0, sizeof(uint32_t), s));
         return ENTRO_OK;
     }
-    const DecodeConfig cfg = decode_config();
+    const DecodeConfig cfg = item_size_for(decode_config(), descs_host, ntensors, sd->sm_count);
 
     StaticUpload up;
     uint64_t items = 0;
