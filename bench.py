@@ -33,6 +33,11 @@ import workloads
 
 METRIC = "Huffman decode+dequant GB/s (compressed in + fp16 out)"
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes per weight of the decode kernel (dram__bytes_read.sum + dram__bytes_write.sum of one
+# ncu capture on the 1-layer truncation, 480,260,096 weights; traffic grows in proportion to the
+# weights, so a full launch is this figure times its weights).  See profiles/.  Set an entry to
+# None when the kernel changes until the counters have been taken again.
+NCU_DRAM_BYTES_PER_WEIGHT = {8: 1100.4e6 / 480260096, 4: 966.95e6 / 480260096}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -398,7 +403,10 @@ def measure(E, wl, args, world, local_rank, rank, peak, with_e2e, with_cpu):
         "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak[0],
                      "unit": "GB/s", "frac": achieved / peak[0], "peak_source": peak[1],
                      "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS, "kernel_ms": k_ms,
-                     "kernel_ms_min": float(np.min(kernel_ms)) if kernel_ms else None, "traffic": None},
+                     "kernel_ms_min": float(np.min(kernel_ms)) if kernel_ms else None,
+                     "traffic": (NCU_DRAM_BYTES_PER_WEIGHT.get(wl.bits) * model.n
+                                 if NCU_DRAM_BYTES_PER_WEIGHT.get(wl.bits) else None),
+                     "traffic_note": "bytes per launch: ncu DRAM read+write on the 1-layer case, scaled by weights"},
         "model": model,
     }
     if with_e2e and rank == 0 or (with_e2e and world > 1):
