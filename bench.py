@@ -53,6 +53,8 @@ def measured_peak():
 
 
 def pick_workload(name: str, max_layers):
+    if name.endswith("-gauss"):
+        return workloads.with_matrix_kind(pick_workload(name[:-6], max_layers), "gauss")
     if name == "mistral8":
         return workloads.mistral_7b(bits=8, max_layers=max_layers)
     if name == "mistral4":
@@ -425,7 +427,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--workload", default="mistral8",
-                    choices=["mistral8", "mistral4", "smollm8", "phi3_4", "single"])
+                    choices=["mistral8", "mistral4", "smollm8", "phi3_4", "single", "mistral8-gauss", "mistral4-gauss"])
     ap.add_argument("--also", default="mistral4", help="second workload reported under 'also' ('' = none)")
     ap.add_argument("--max-layers", type=int, default=None, help="truncate the model (for profiling runs)")
     ap.add_argument("--e2e-steps", type=int, default=2)

@@ -16,13 +16,15 @@
 // Tables per tensor (built by build_tables_kernel, copied into shared memory per CTA):
 //   alphabets > 16 symbols, one symbol per lookup.  Canonical codes grow longer towards the
 //     all-ones end of the code space, so the table is indexed like a floating-point number:
-//     by the count of leading one bits of the window and the kExpBits bits after the first
-//     zero.  Converting the inverted window to float yields exactly that index (exponent |
-//     top mantissa bits) in one instruction, and 32 << kExpBits cells resolve every code
-//     whose length is at most leading ones + 1 + kExpBits - on bell-shaped histograms all
-//     of them, where a direct table of the same size would miss the tail.  The shared-
-//     memory copy is replicated 32 times, cell-major, so lane l only ever touches bank l:
-//     no bank conflicts whatever the data.
+//     by the count of leading one bits of the window and the m bits after the first zero.
+//     Converting the inverted window to float yields exactly that index (exponent | top
+//     mantissa bits) in one instruction, and 32 << m cells resolve every code whose length
+//     is at most leading ones + 1 + m - on bell-shaped histograms all of them, where a
+//     direct table of the same size would miss the tail.  m = 4 when that already covers
+//     the code (peaked, heavy-tailed histograms): the shared-memory copy is then replicated
+//     32 times, cell-major, so lane l only ever touches bank l and no lookup conflicts,
+//     whatever the data.  Flatter histograms get m = 5 and 16 copies (lanes l and l + 16
+//     share one: at most two wavefronts per lookup).
 //   alphabets <= 16 symbols, eight symbols per lookup: the next K bits index a table of
 //     16-byte entries (eight fp16 values) and a byte table (bits used, 0 = no eight whole
 //     codes in K bits); one unreplicated copy of the exponent-indexed table serves the
@@ -45,7 +47,7 @@ constexpr uint32_t kOverRead = 2064;       // a lane fed garbage may read this f
 // window is the driver's).  The hand-written lookups address the tables as [offset + 1024];
 // the kernel checks the assumption before it does anything else.
 constexpr uint32_t kSmemBase = 1024;
-static_assert(kExpBits == 4, "the hand-written lookups hard-code the 4-bit cell mask and shift");
+static_assert(kExpBitsMax == 5, "the lookups shift by 12 and mask: right for 4 and 5 mantissa bits only");
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 // 32-bit word at a shared-window address.
@@ -59,8 +61,7 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
 // Shared-memory bytes of the lookup tables for a K-bit eight-symbol table.
 __host__ __device__ constexpr uint32_t lut_bytes(int K)
 {
-    return (17u << K) + 4u * kExpEntries > (uint32_t)kExpEntries * 128u ? (17u << K) + 4u * kExpEntries
-                                                                        : (uint32_t)kExpEntries * 128u;
+    return (17u << K) + 4u * kExpEntriesMax > 65536u ? (17u << K) + 4u * kExpEntriesMax : 65536u;
 }
 
 // ------------------------------------------------------------------ table construction
@@ -86,6 +87,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     __shared__ DecodeAux aux;
     __shared__ uint32_t count[ENTRO_MAX_CODE_LEN + 1];
     __shared__ uint8_t len[ENTRO_MAX_SYMBOLS];
+    __shared__ float unresolved4;   // probability mass (by 2^-length) of codes a 4-bit-mantissa table leaves open
     const int t = blockIdx.x;
     const int tid = threadIdx.x;
     const DevTensor& T = tensors[t];
@@ -100,7 +102,8 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     if (tid == 0) {
         unsigned long long code = 0;   // reaches 2^32 after the last length of a complete code
         uint32_t off = 0, max_len = 0;
-        float mean_len = 0.f;          // sum over codes of len * 2^-len: the code's own estimate of its mean length
+        // bits per symbol of this tensor's stream, from the index (a wrong index can only pick a slower mode)
+        const float mean_len = (float)T.offsets[T.n_chunks] / (float)T.n;
         aux.limit[0] = 0;
         aux.first_code[0] = 0;
         aux.offset[0] = 0;
@@ -112,20 +115,28 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
             off += count[k];
             aux.limit[k] = code << (32 - k);
             if (count[k]) max_len = k;
-            mean_len += (float)count[k] * (float)k * exp2f(-(float)k);
         }
         aux.max_len = max_len;
-        aux.oct = T.nsym <= 16 ? 1u : 0u;
-        // four lookups per window refill while their lengths almost always sum to <= 32 bits
+        // eight symbols per lookup pay off while eight codes usually fit the table's window
+        aux.oct = (T.nsym <= 16 && mean_len * 8.f <= (float)lut_bits - 1.5f) ? 1u : 0u;
+        // four lookups per window refill while their lengths almost always sum to < 32 bits
         aux.group = mean_len <= 4.75f ? 4u : 2u;
-        aux.pad = 0;
+        aux.expm = 4u;
+        unresolved4 = 0.f;
     }
     __syncthreads();
     if (l) {
         uint32_t rank = 0;
         for (int k = 0; k < tid; ++k) rank += (len[k] == l);
         aux.sorted[aux.offset[l] + rank] = (uint8_t)tid;
+        // would a table with 4 mantissa bits resolve this symbol's code?  It has r leading ones.
+        const uint32_t left = (aux.first_code[l] + rank) << (32u - l);
+        uint32_t r = (uint32_t)__clz((int)~left);
+        if (r > l) r = l;
+        if (l > r + 5u) atomicAdd(&unresolved4, exp2f(-(float)l));
     }
+    __syncthreads();
+    if (tid == 0 && unresolved4 > 6e-5f) aux.expm = 5u;
     const float d = (float)(tid - T.zero_point);
     aux.val[tid] = __half_as_ushort(__float2half_rn(__fmul_rn(T.scale, d)));
     __syncthreads();
@@ -161,11 +172,12 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     }
     {
         // cell (e5, mant): windows that start with r ones and a zero, followed by the bits ~mant
-        for (uint32_t i = tid; i < (uint32_t)kExpEntries; i += 256) {
+        const uint32_t kExpBits = aux.expm;
+        for (uint32_t i = tid; i < (32u << kExpBits); i += 256) {
             const uint32_t e5 = i >> kExpBits, mant = i & ((1u << kExpBits) - 1u);
             const uint32_t r = (30u - e5) & 31u;
             const uint32_t avail = 31u - r;                               // window bits after the zero
-            const uint32_t mb = avail < (uint32_t)kExpBits ? avail : (uint32_t)kExpBits;
+            const uint32_t mb = avail < kExpBits ? avail : kExpBits;
             uint32_t entry = kEscLen;
             if ((mant & ((1u << (kExpBits - mb)) - 1u)) == 0u) {          // else no window maps here
                 const uint32_t mt = mant >> (kExpBits - mb);
@@ -281,12 +293,25 @@ __device__ __forceinline__ void gwin_refill(GlobalWin& r)
 
 // ------------------------------------------------------------------ lookups
 
+// How a lane addresses its copy of the exponent-indexed table (which starts at the
+// beginning of shared memory, cell-major): byte offset = ((float bits >> 12) & mask) | lane.
+// m = 4: 32 copies, cells 128 bytes apart; m = 5: 16 copies, 64 bytes apart.
+struct LutKey {
+    uint32_t mask, lane;
+};
+__device__ __forceinline__ LutKey lut_key(uint32_t expm, uint32_t lane)
+{
+    LutKey k;
+    k.mask = expm == 4u ? 0xff80u : 0xffc0u;
+    k.lane = (expm == 4u ? lane : (lane & 15u)) * 4u;
+    return k;
+}
+
 // Cell of the exponent-indexed table for an inverted window, in this lane's copy.
-// lane4 = 4 * lane.  The table starts at the beginning of shared memory.
-__device__ __forceinline__ uint32_t exp_lookup(uint32_t lane4, uint32_t inv_window)
+__device__ __forceinline__ uint32_t exp_lookup(LutKey key, uint32_t inv_window)
 {
     const uint32_t fb = __float_as_uint(__uint2float_rz(inv_window));
-    const uint32_t a = ((fb >> (16 - kExpBits)) & (((32u << kExpBits) - 1u) << 7)) | lane4;
+    const uint32_t a = ((fb >> 12) & key.mask) | key.lane;
     return *reinterpret_cast<const uint32_t*>(smem + a);
 }
 
@@ -304,7 +329,7 @@ __device__ __forceinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32
 }
 
 // One group of lookups of an 8-bit alphabet, hand-scheduled.  In: the inverted window
-// (hi, lo, k, next) and lane4 = 4 * lane.  The refill is predicated (no branch), the G
+// (hi, lo, k, next) and the lane's table key.  The refill is predicated (no branch), the G
 // lookups read the window at the running sum of the entries before them (a funnel shift
 // uses the low five bits, the length sums), and the window is advanced by the final sum
 // in place.  Out: the fp16 values in pairs, and s, the sum of the G entries: the group
@@ -315,7 +340,7 @@ __device__ __forceinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32
     "cvt.rz.f32.u32 f, " win ";\n\t"                  \
     "mov.b32 a, f;\n\t"                               \
     "shr.u32 a, a, 12;\n\t"                           \
-    "lop3.b32 a, a, 0xFF80, %7, 0xEA;\n\t"            \
+    "lop3.b32 a, a, %8, %7, 0xEA;\n\t"                \
     "ld.shared.b32 " dst ", [a+1024];\n\t"
 #define ENTRO_REFILL                                 \
     "and.b32 t, %2, 0x8000;\n\t"                      \
@@ -332,7 +357,7 @@ __device__ __forceinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32
     "shf.l.wrap.b32 %1, 0, %1, %6;\n\t"               \
     "add.u32 %2, %2, %6;\n\t"
 
-__device__ __forceinline__ void group4(Win& r, uint32_t lane4, uint32_t& pk0, uint32_t& pk1, uint32_t& s)
+__device__ __forceinline__ void group4(Win& r, LutKey key, uint32_t& pk0, uint32_t& pk1, uint32_t& s)
 {
     asm volatile(
         "{\n\t"
@@ -348,10 +373,10 @@ __device__ __forceinline__ void group4(Win& r, uint32_t lane4, uint32_t& pk0, ui
         "prmt.b32 %4, e0, e1, 0x7632;\n\t"
         "prmt.b32 %5, e2, e3, 0x7632;\n\t" ENTRO_ADVANCE "}"
         : "+r"(r.hi), "+r"(r.lo), "+r"(r.k), "+r"(r.next), "=&r"(pk0), "=&r"(pk1), "=&r"(s)
-        : "r"(lane4));
+        : "r"(key.lane), "r"(key.mask));
 }
 
-__device__ __forceinline__ void group2(Win& r, uint32_t lane4, uint32_t& pk0, uint32_t& s)
+__device__ __forceinline__ void group2(Win& r, LutKey key, uint32_t& pk0, uint32_t& s)
 {
     uint32_t unused;
     asm volatile(
@@ -364,7 +389,7 @@ __device__ __forceinline__ void group2(Win& r, uint32_t lane4, uint32_t& pk0, ui
         "prmt.b32 %4, e0, e1, 0x7632;\n\t"
         "mov.b32 %5, 0;\n\t" ENTRO_ADVANCE "}"
         : "+r"(r.hi), "+r"(r.lo), "+r"(r.k), "+r"(r.next), "=&r"(pk0), "=&r"(unused), "=&r"(s)
-        : "r"(lane4));
+        : "r"(key.lane), "r"(key.mask));
 }
 #undef ENTRO_LOOKUP
 #undef ENTRO_REFILL
@@ -374,13 +399,18 @@ __device__ __forceinline__ void group2(Win& r, uint32_t lane4, uint32_t& pk0, ui
 // lane's copy for 8-bit alphabets, the single copy behind the eight-symbol tables for 4-bit
 // ones), the canonical ranges if the cell is unresolved.  -> value << 16 | length.
 template <int K, bool kOct>
-__device__ __forceinline__ uint32_t next_symbol(Win& r, uint32_t* status, uint32_t lane4)
+__device__ __forceinline__ uint32_t next_symbol(Win& r, uint32_t* status, LutKey key)
 {
     win_refill<!kOct>(r);
     const uint32_t inv = kOct ? ~r.hi : r.hi;
-    const uint32_t cell = (__float_as_uint(__uint2float_rz(inv)) >> (23 - kExpBits)) & (uint32_t)(kExpEntries - 1);
-    uint32_t e = kOct ? *reinterpret_cast<const uint32_t*>(smem + (17u << K) + cell * 4u)
-                      : *reinterpret_cast<const uint32_t*>(smem + cell * 128u + lane4);
+    uint32_t e;
+    if (kOct) {
+        const uint32_t m = reinterpret_cast<const DecodeAux*>(smem + lut_bytes(K))->expm;
+        const uint32_t cell = (__float_as_uint(__uint2float_rz(inv)) >> (23u - m)) & ((32u << m) - 1u);
+        e = *reinterpret_cast<const uint32_t*>(smem + (17u << K) + cell * 4u);
+    } else {
+        e = exp_lookup(key, inv);
+    }
     if ((e & 0xffffu) > 32u) e = decode_by_range(reinterpret_cast<const DecodeAux*>(smem + lut_bytes(K)), ~inv, status);
     win_skip_any(r, e & 0xffffu);
     return e;
@@ -391,18 +421,18 @@ __device__ __forceinline__ uint32_t next_symbol(Win& r, uint32_t* status, uint32
 // shared memory).  Rebuilds the window as it was before the group from (k, next, s), then
 // takes the symbols one by one.
 template <int K, int G>
-__device__ __forceinline__ void repair_group(Win& r, uint32_t* status, uint32_t lane4, uint32_t s, uint32_t& pk0,
+__device__ __forceinline__ void repair_group(Win& r, uint32_t* status, LutKey key, uint32_t s, uint32_t& pk0,
                                              uint32_t& pk1)
 {
     const uint32_t valid = (uint32_t)win_valid_bits(r.k - s);   // 33 .. 64 bits were valid when the group began
     const uint32_t bit_addr = r.next * 8u - valid;              // where they begin, in bits of the shared window
     win_init<true>(r, (bit_addr >> 5) << 2, bit_addr & 31u);
-    const uint32_t e0 = next_symbol<K, false>(r, status, lane4);
-    const uint32_t e1 = next_symbol<K, false>(r, status, lane4);
+    const uint32_t e0 = next_symbol<K, false>(r, status, key);
+    const uint32_t e1 = next_symbol<K, false>(r, status, key);
     pk0 = __byte_perm(e0, e1, 0x7632);
     if (G == 4) {
-        const uint32_t e2 = next_symbol<K, false>(r, status, lane4);
-        const uint32_t e3 = next_symbol<K, false>(r, status, lane4);
+        const uint32_t e2 = next_symbol<K, false>(r, status, key);
+        const uint32_t e3 = next_symbol<K, false>(r, status, key);
         pk1 = __byte_perm(e2, e3, 0x7632);
     }
 }
@@ -413,7 +443,7 @@ __device__ __forceinline__ uint4 repair_oct(Win& r, uint32_t* status)
 {
     uint32_t h[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) h[k] = next_symbol<K, true>(r, status, 0u);
+    for (int k = 0; k < 8; ++k) h[k] = next_symbol<K, true>(r, status, LutKey{0u, 0u});
     return make_uint4(__byte_perm(h[0], h[1], 0x7632), __byte_perm(h[2], h[3], 0x7632), __byte_perm(h[4], h[5], 0x7632),
                       __byte_perm(h[6], h[7], 0x7632));
 }
@@ -617,7 +647,7 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
         for (uint32_t i = g * 8u; i < end; ++i) {
             gwin_refill(r);
             uint32_t e = kEscLen;
-            if (!oct) e = exp_lookup(lane * 4u, ~r.hi);
+            if (!oct) e = exp_lookup(lut_key(aux->expm, lane), ~r.hi);
             if ((e & 0xffffu) > 32u) e = decode_by_range(aux, r.hi, status);
             const uint32_t n = e & 0xffffu;
             r.hi = __funnelshift_lc(r.lo, r.hi, n);
@@ -705,7 +735,7 @@ struct EmitDot {
 
 // 8-bit alphabets: G lookups per window refill (group4 / group2 above).
 template <int K, int G, class Emit>
-__device__ __forceinline__ void rows_single(Win& r, uint32_t* status, uint32_t lane4, Emit& emit, uint32_t sub)
+__device__ __forceinline__ void rows_single(Win& r, uint32_t* status, LutKey key, Emit& emit, uint32_t sub)
 {
     for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
         uint32_t pk[4];
@@ -713,17 +743,17 @@ __device__ __forceinline__ void rows_single(Win& r, uint32_t* status, uint32_t l
 #pragma unroll
             for (int g = 0; g < 2; ++g) {
                 uint32_t s;
-                group4(r, lane4, pk[2 * g], pk[2 * g + 1], s);
-                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_group<K, 4>(r, status, lane4, s, pk[2 * g], pk[2 * g + 1]);
+                group4(r, key, pk[2 * g], pk[2 * g + 1], s);
+                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_group<K, 4>(r, status, key, s, pk[2 * g], pk[2 * g + 1]);
             }
         } else {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 uint32_t s;
-                group2(r, lane4, pk[g], s);
+                group2(r, key, pk[g], s);
                 if (__builtin_expect((s & 0xffe0u) != 0u, 0)) {
                     uint32_t none;
-                    repair_group<K, 2>(r, status, lane4, s, pk[g], none);
+                    repair_group<K, 2>(r, status, key, s, pk[g], none);
                 }
             }
         }
@@ -832,15 +862,15 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         em.acc = 0.f;
         em.yrow = G->y32 + row0;
         if (oct) rows_oct<K>(w, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lane * 4u, em, sub);
-        else rows_single<K, 2>(w, status, lane * 4u, em, sub);
+        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
         em.finish();
     } else {
         EmitStore em;
         em.dst = reinterpret_cast<uint4*>(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
         if (oct) rows_oct<K>(w, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lane * 4u, em, sub);
-        else rows_single<K, 2>(w, status, lane * 4u, em, sub);
+        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
     }
     // the lane must stand exactly at the end of its sub-block
     if (w.next * 8u - (uint32_t)win_valid_bits(w.k) != L.end) atomicOr(status, kStatCorrupt);
@@ -939,12 +969,14 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                 uint4* s2 = reinterpret_cast<uint4*>(smem + (16u << K));
                 for (uint32_t i = threadIdx.x; i < (1u << K) / 16; i += blockDim.x) s2[i] = __ldg(g2 + i);
                 uint32_t* s3 = reinterpret_cast<uint32_t*>(smem + (17u << K));
-                for (uint32_t i = threadIdx.x; i < (uint32_t)kExpEntries; i += blockDim.x) s3[i] = __ldg(tt->exp_lut + i);
+                for (uint32_t i = threadIdx.x; i < (uint32_t)kExpEntriesMax; i += blockDim.x) s3[i] = __ldg(tt->exp_lut + i);
             } else {
-                // 32 copies, cell-major: word (cell * 32 + lane) belongs to lane's bank
+                // cell-major copies: 32 of them (word cell * 32 + lane sits in lane's bank) or 16
                 uint32_t* s1 = reinterpret_cast<uint32_t*>(smem);
-                for (uint32_t cell = warp; cell < (uint32_t)kExpEntries; cell += warps)
-                    s1[cell * 32u + lane] = __ldg(tt->exp_lut + cell);
+                const uint32_t m = __ldg(&tt->aux.expm);
+                const uint32_t copies = m == 4u ? 32u : 16u;
+                for (uint32_t cell = warp; cell < (32u << m); cell += warps)
+                    s1[cell * copies + (lane & (copies - 1u))] = __ldg(tt->exp_lut + cell);
             }
             __syncthreads();
         }

@@ -10,8 +10,8 @@ namespace entro {
 
 constexpr int kSubBlocks = ENTRO_SUB_BLOCKS;
 constexpr int kMaxLutBits = 12;               // widest window of the eight-symbol table
-constexpr int kExpBits = 4;                   // mantissa bits of the exponent-indexed table
-constexpr int kExpEntries = 32 << kExpBits;
+constexpr int kExpBitsMax = 5;                // mantissa bits of the exponent-indexed table: 4 or 5 per tensor
+constexpr int kExpEntriesMax = 32 << kExpBitsMax;
 
 // Device status bits (OR-ed by kernels, read by entro_last_device_status).
 constexpr uint32_t kStatCorrupt = 1u;         // index / stream / codebook disagree
@@ -56,7 +56,7 @@ struct DecodeAux {
     uint32_t max_len;
     uint32_t oct;      // 1: eight symbols per lookup (alphabets of <= 16 symbols)
     uint32_t group;    // one-symbol lookups per window refill: 4 or 2
-    uint32_t pad;
+    uint32_t expm;     // mantissa bits of this tensor's exponent-indexed table
 };
 static_assert(sizeof(DecodeAux) % 16 == 0, "DecodeAux is copied as 16-byte vectors");
 
@@ -64,7 +64,7 @@ static_assert(sizeof(DecodeAux) % 16 == 0, "DecodeAux is copied as 16-byte vecto
 struct TensorTables {
     uint4 oct_val[1u << kMaxLutBits];      // eight fp16 values per window (oct mode)
     uint8_t oct_len[1u << kMaxLutBits];    // bits they use, 0 = not eight whole codes
-    uint32_t exp_lut[kExpEntries];         // value << 16 | length, or length 64 (one-symbol mode)
+    uint32_t exp_lut[kExpEntriesMax];      // value << 16 | length, or length 64; 32 << aux.expm cells in use
     DecodeAux aux;
 };
 static_assert(sizeof(TensorTables) % 16 == 0, "TensorTables is copied as 16-byte vectors");

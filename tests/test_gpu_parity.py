@@ -111,6 +111,28 @@ def test_decode_of_oracle_streams_small_and_ragged(bits, chunk):
     assert_status_ok()
 
 
+@pytest.mark.parametrize("bits,chunk", [(8, 4096), (4, 8192)])
+def test_decode_flat_histograms(bits, chunk):
+    """Inputs without heavy tails spread the symbols over many levels: the 8-bit path then uses
+    the wider exponent-indexed table and groups of two, the 4-bit path one symbol per lookup.
+    A uniform histogram (every code the same length) is resolved by no table cell at all and
+    runs entirely on the symbol-by-symbol repair."""
+    for n in (chunk - 1, 9 * chunk, 33 * chunk + 77):
+        w_np, _ = _values(n, 0.02, 4242 + n % 100 + bits, "gauss")
+        c = oracle.compress(w_np, bits, chunk)
+        assert np.array_equal(gpu_decode_from_oracle_stream(c, n, chunk), expected_out(c)), (bits, n)
+    nsym = 1 << bits
+    q = np.random.default_rng(bits).integers(0, nsym, 20 * chunk + 5).astype(np.uint8)
+    ln = oracle.huffman_lengths(np.bincount(q, minlength=nsym).tolist())
+    cd = oracle.canonical_codes(ln)
+    enc = oracle.encode(q, ln, cd, chunk)
+    out = E.entro_decode_dequant(to_dev_stream(enc.stream), to_dev_index(enc), q.size, chunk,
+                                 E.Codebook.from_lengths(ln.tolist(), cd.tolist()), 0.03125, nsym // 2)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.dequant(q, 0.03125, nsym // 2))
+    assert_status_ok()
+
+
 def test_decode_config1_single_tensor():
     """1024 x 1024, sigma 0.02, seed 0, asymmetric uint8, 4096-symbol chunks."""
     wl = workloads.single_tensor()
