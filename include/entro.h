@@ -268,7 +268,9 @@ entro_status entro_last_device_status(void *cuda_stream);
 /*
  * Launch shape of the decode kernel; every argument may be 0 to keep its current value.
  *   lut_bits: window of the eight-symbol table used for alphabets of <= 16 symbols (10 .. 12)
- *   warps_per_cta: 4 .. 32;  ctas_per_sm: 1 .. 8;  chunks_per_item: chunks a CTA claims at once
+ *   warps_per_cta: 4 .. 32;  ctas_per_sm: 1 .. 8;  chunks_per_item: largest number of 4096-symbol
+ *   chunks a CTA claims at once (the library shrinks it for small launches, for the last
+ *   part of a large one, and in proportion for larger chunks)
  * ENTRO_ERR_INVALID_ARG (nothing changed) if a value is out of range or the shape does
  * not fit in shared memory.
  */

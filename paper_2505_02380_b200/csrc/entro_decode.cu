@@ -880,14 +880,14 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
 // ------------------------------------------------------------------ persistent kernel
 
 // item_start[t] = first work item of tensor t, item_start[ntensors] = number of items; an
-// item is up to chunks_per_item consecutive chunks of one tensor.
+// item is up to tensors[t].item_chunks consecutive chunks of one tensor.
 // With kGemv the decoded weights are not stored: gemv[t] describes the matrix-vector product
 // they enter (the fused decode + dequantise + GEMV of a batch-1 token step).
 template <int K, bool kGemv>
 __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __restrict__ tensors, int ntensors,
                                                          const uint32_t* __restrict__ item_start,
                                                          const TensorTables* __restrict__ tables,
-                                                         uint32_t chunks_per_item, uint32_t stage_bytes,
+                                                         uint32_t stage_bytes,
                                                          uint32_t* __restrict__ control,
                                                          const GemvTensor* __restrict__ gemv)
 {
@@ -981,6 +981,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             __syncthreads();
         }
         const DevTensor& T = *s_tensor;
+        const uint32_t chunks_per_item = T.item_chunks;
         const uint32_t first = (item - __ldg(item_start + cur)) * chunks_per_item;
 
         // The warps share out the item's chunks.  Each warp, per turn: start the bulk copy of
@@ -1061,7 +1062,7 @@ entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTens
     const bool timed = ws->prof_used < ws->prof_cap;
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_start[ws->prof_used], s));
     decode_kernel<K, kGemv><<<grid, cfg.warps_per_cta * 32, sh.smem, s>>>(
-        tensors, ntensors, item_start, tables, (uint32_t)cfg.chunks_per_item, sh.stage_bytes, ws->control, gemv);
+        tensors, ntensors, item_start, tables, sh.stage_bytes, ws->control, gemv);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_stop[ws->prof_used++], s));
@@ -1103,23 +1104,38 @@ entro_status validate_desc(const entro_tensor_desc& d, bool need_out = true)
     return ENTRO_OK;
 }
 
-// Work items small enough that a launch with few chunks (one layer, one tensor) still gives
-// every CTA several of them: at most the configured size, at least one chunk per warp.
-DecodeConfig item_size_for(DecodeConfig cfg, const entro_tensor_desc* descs, int ntensors, int sm_count)
+// How a launch's chunks are cut into work items.  Large items keep the per-item costs (a
+// CTA-wide barrier, table reload, pipeline refill) small; the items at the end of the list
+// are an eighth of that size so that the CTAs finish together; and a launch with few chunks
+// (one layer, one tensor) gets items small enough that every CTA still has several.
+struct ItemPlan {
+    uint64_t total = 0;        // chunks in the launch
+    uint64_t seen = 0;         // chunks of the tensors planned so far
+    uint32_t base = 0, tail = 0;
+    bool graded = false;
+};
+
+ItemPlan plan_items(const DecodeConfig& cfg, const entro_tensor_desc* descs, int ntensors, int sm_count)
 {
-    uint64_t chunks = 0;
+    ItemPlan p;
+    int live = 0;
     for (int i = 0; i < ntensors; ++i)
-        if (descs[i].n) chunks += num_chunks(descs[i].n, descs[i].chunk_symbols);
+        if (descs[i].n) {
+            p.total += num_chunks(descs[i].n, descs[i].chunk_symbols);
+            ++live;
+        }
     const uint64_t ctas = (uint64_t)sm_count * cfg.ctas_per_sm;
-    uint64_t want = (chunks + ctas * 4 - 1) / (ctas * 4);
+    uint64_t want = (p.total + ctas * 4 - 1) / (ctas * 4);
     want = (want + cfg.warps_per_cta - 1) / cfg.warps_per_cta * cfg.warps_per_cta;
     if (want < (uint64_t)cfg.warps_per_cta) want = cfg.warps_per_cta;
-    if (want < (uint64_t)cfg.chunks_per_item) cfg.chunks_per_item = (int)want;
-    return cfg;
+    p.base = want < (uint64_t)cfg.chunks_per_item ? (uint32_t)want : (uint32_t)cfg.chunks_per_item;
+    p.tail = p.base / 8 < (uint32_t)cfg.warps_per_cta ? (uint32_t)cfg.warps_per_cta : p.base / 8;
+    p.graded = live >= 8 && p.base == (uint32_t)cfg.chunks_per_item;
+    return p;
 }
 
 // Device-side form of a descriptor; returns the tensor's number of work items.
-uint64_t fill_dev_tensor(const entro_tensor_desc& d, const DecodeConfig& cfg, DevTensor& t)
+uint64_t fill_dev_tensor(const entro_tensor_desc& d, ItemPlan& plan, DevTensor& t)
 {
     const uint64_t nc = num_chunks(d.n, d.chunk_symbols);
     t.stream = d.stream_dev;
@@ -1133,9 +1149,16 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, const DecodeConfig& cfg, De
     t.nsym = (uint32_t)d.cb.nsym;
     t.scale = d.scale;
     t.zero_point = d.zero_point;
-    t.pad[0] = t.pad[1] = t.pad[2] = 0;
+    // the last 12 % of the launch's chunks go out in small items; sizes are meant for
+    // 4096-symbol chunks and scale down for larger ones, so that an item is as much work
+    uint32_t per_item = (plan.graded && (plan.seen + nc) * 100 > plan.total * 88) ? plan.tail : plan.base;
+    if (d.chunk_symbols > 4096u) per_item = (uint32_t)((uint64_t)per_item * 4096u / d.chunk_symbols);
+    if (per_item < 32u) per_item = 32u;
+    t.item_chunks = per_item;
+    plan.seen += nc;
+    t.pad[0] = t.pad[1] = 0;
     for (int j = 0; j < ENTRO_MAX_SYMBOLS; ++j) t.len[j] = j < d.cb.nsym ? d.cb.len[j] : 0;
-    return (nc + cfg.chunks_per_item - 1) / cfg.chunks_per_item;
+    return (nc + t.item_chunks - 1) / t.item_chunks;
 }
 
 }  // namespace
@@ -1143,7 +1166,8 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, const DecodeConfig& cfg, De
 // Upload descriptors, build the tables and run the persistent decode kernel.
 entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs, int ntensors, cudaStream_t s)
 {
-    const DecodeConfig cfg = item_size_for(decode_config(), descs, ntensors, ws->sm_count);
+    const DecodeConfig cfg = decode_config();
+    ItemPlan plan = plan_items(cfg, descs, ntensors, ws->sm_count);
     int live = 0;
     for (int i = 0; i < ntensors; ++i) {
         entro_status st = validate_desc(descs[i]);
@@ -1166,7 +1190,7 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     for (int i = 0; i < ntensors; ++i) {
         if (!descs[i].n) continue;
         hitems[k] = (uint32_t)items;
-        items += fill_dev_tensor(descs[i], cfg, ht[k]);
+        items += fill_dev_tensor(descs[i], plan, ht[k]);
         if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
         ++k;
     }
@@ -1325,7 +1349,8 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
     Guard guard;
     Workspace* ws = workspace();
     if (!ws) return ENTRO_ERR_CUDA;
-    const DecodeConfig cfg = item_size_for(decode_config(), descs_host, ntensors, ws->sm_count);
+    const DecodeConfig cfg = decode_config();
+    ItemPlan plan = plan_items(cfg, descs_host, ntensors, ws->sm_count);
 
     // workspace: [DevTensor x n][item_start][GemvTensor x n] (uploaded) [tables x n][y32]
     const size_t tensors_bytes = (size_t)ntensors * sizeof(DevTensor);
@@ -1345,7 +1370,7 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
     uint64_t items = 0, row0 = 0;
     for (int i = 0; i < ntensors; ++i) {
         hitems[i] = (uint32_t)items;
-        items += fill_dev_tensor(descs_host[i], cfg, ht[i]);
+        items += fill_dev_tensor(descs_host[i], plan, ht[i]);
         if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
         hg[i].x = static_cast<const uint16_t*>(io_host[i].x_fp16_dev);
         hg[i].y32 = y32 + row0;
@@ -1484,7 +1509,8 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
         if (status_dev) ENTRO_CUDA(cudaMemsetAsync(status_dev, 0, sizeof(uint32_t), s));
         return ENTRO_OK;
     }
-    const DecodeConfig cfg = item_size_for(decode_config(), descs_host, ntensors, sd->sm_count);
+    const DecodeConfig cfg = decode_config();
+    ItemPlan plan = plan_items(cfg, descs_host, ntensors, sd->sm_count);
 
     StaticUpload up;
     uint64_t items = 0;
@@ -1492,7 +1518,7 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
     for (int i = 0; i < ntensors; ++i) {
         if (!descs_host[i].n) continue;
         up.item_start[k] = (uint32_t)items;
-        items += fill_dev_tensor(descs_host[i], cfg, up.tensors[k]);
+        items += fill_dev_tensor(descs_host[i], plan, up.tensors[k]);
         if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
         ++k;
     }

@@ -31,7 +31,8 @@ struct DevTensor {
     uint32_t nsym;
     float scale;
     int32_t zero_point;
-    uint32_t pad[3];
+    uint32_t item_chunks;         // chunks per work item of this tensor
+    uint32_t pad[2];
     uint8_t len[ENTRO_MAX_SYMBOLS];
 };
 static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vectors");
@@ -73,7 +74,7 @@ struct DecodeConfig {
     int lut_bits = 12;
     int warps_per_cta = 32;
     int ctas_per_sm = 1;
-    int chunks_per_item = 512;
+    int chunks_per_item = 1024;
 };
 
 // Per-device workspace owned by the library.
