@@ -265,11 +265,6 @@ __device__ __forceinline__ void win_skip_any(Win& r, uint32_t n)
 
 __device__ __forceinline__ int win_valid_bits(uint32_t k) { return 32 - (int)(short)(k & 0xffffu); }
 
-__device__ __forceinline__ uint32_t win_used_bits(const Win& r, uint32_t base, uint32_t bit_pos)
-{
-    return (r.next - base) * 8u - (uint32_t)win_valid_bits(r.k) - bit_pos;
-}
-
 // The same over global memory, word by word, for chunks that are not staged.
 struct GlobalWin {
     uint32_t hi, lo;
@@ -378,7 +373,7 @@ __device__ __forceinline__ void group4(Win& r, LutKey key, uint32_t& pk0, uint32
 
 __device__ __forceinline__ void group2(Win& r, LutKey key, uint32_t& pk0, uint32_t& s)
 {
-    uint32_t unused;
+    __attribute__((unused)) uint32_t unused;   // operand slot of the second pair, which a group of two does not have
     asm volatile(
         "{\n\t"
         ".reg .pred p;\n\t"
@@ -871,6 +866,7 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         if (oct) rows_oct<K>(w, status, em, sub);
         else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
         else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        em.finish();
     }
     // the lane must stand exactly at the end of its sub-block
     if (w.next * 8u - (uint32_t)win_valid_bits(w.k) != L.end) atomicOr(status, kStatCorrupt);
