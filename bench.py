@@ -138,6 +138,7 @@ class DeviceModel:
         self.wl = wl
         self.q = []              # quantised symbols per tensor (only with keep_q)
         self.qparams = []
+        self.cbs = []
         self.keep = []           # device buffers
         descs = []
         # per-tensor decode tables read from HBM: canonical ranges + the lookup table of the tensor's mode
@@ -160,6 +161,7 @@ class DeviceModel:
             cb = E.entro_build_codebook(counts.tolist())
             enc = E.entro_encode(q, cb, wl.chunk_symbols, stream_words=E.entro_stream_words(counts.tolist(), cb))
             self.qparams.append((qp.scale, qp.zero_point))
+            self.cbs.append(cb)
             if keep_q:
                 self.q.append(q)
             del w, q
@@ -210,6 +212,32 @@ def time_steps(E, model, steps, warmup, world, sampler_index):
     E.entro_profile_begin(0)
     assert E.entro_last_device_status() == E.OK
     return ms, launches, kernel_ms, clocks
+
+
+def time_symbols(E, model, steps=10):
+    """The same model decoded to integer symbols (the paper's decoder output): one byte per
+    symbol at 8 bits, two symbols per byte at 4 bits.  -> kernel ms, GB/s (compressed in + bytes out)."""
+    packed = model.wl.bits == 4
+    nbytes = [(t.numel + 1) // 2 if packed else t.numel for t in model.wl.tensors]
+    buf = torch.empty(sum((b + 15) // 16 * 16 for b in nbytes), dtype=torch.uint8, device="cuda")
+    descs, pos = [], 0
+    for spec, enc, cb, nb in zip(model.wl.tensors, model.keep, model.cbs, nbytes):
+        descs.append(E.make_desc_bytes(enc.stream, enc.index, spec.numel, model.wl.chunk_symbols, cb, buf[pos:pos + nb]))
+        pos += (nb + 15) // 16 * 16
+    descs = E.desc_array(descs)
+    for _ in range(3):
+        E.entro_decode_symbols_batched(descs, packed)
+    torch.cuda.synchronize()
+    E.entro_profile_begin(steps)
+    for _ in range(steps):
+        E.entro_decode_symbols_batched(descs, packed)
+    torch.cuda.synchronize()
+    ms = float(np.mean(E.entro_profile_read(steps)))
+    E.entro_profile_begin(0)
+    assert E.entro_last_device_status() == E.OK
+    bytes_moved = model.stream_bytes + model.index_bytes + model.table_bytes + sum(nbytes)
+    return {"kernel_ms": ms, "GBs": bytes_moved / (ms * 1e-3) / 1e9, "weights_per_s": model.n / (ms * 1e-3),
+            "output": "two 4-bit symbols per byte" if packed else "one symbol per byte"}
 
 
 def time_e2e(E, model, steps, warmup):
@@ -415,6 +443,8 @@ def measure(E, wl, args, world, local_rank, rank, peak, with_e2e, with_cpu):
         e_ms, h2d, d2h = time_e2e(E, model, max(1, min(args.e2e_steps, args.steps)), 1)
         res["e2e"] = {"value": world * model.algorithmic_bytes / (e_ms * 1e-3) / 1e9, "unit": "GB/s",
                       "ms_per_step": e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    if rank == 0 and world == 1:
+        res["symbols_out"] = time_symbols(E, model)
     if with_cpu and rank == 0 and world == 1:
         res["cpu_baseline"] = cpu_baseline(wl)
     return res
@@ -472,7 +502,7 @@ def main():
         r2.pop("model")
         also = {"workload": wl2.name + " full-model decode", "bits": wl2.bits, "chunk_symbols": wl2.chunk_symbols,
                 **{k: r2[k] for k in ("value", "ms_per_step", "weights_per_s", "bytes_per_step", "bits_per_weight",
-                                       "max_code_len", "roofline", "clocks")}}
+                                       "max_code_len", "roofline", "clocks", "symbols_out") if k in r2}}
 
     gemv = None
     if not args.no_gemv and rank == 0 and world == 1:
@@ -500,6 +530,8 @@ def main():
             line["e2e"] = main_res["e2e"]
         if "cpu_baseline" in main_res:
             line["cpu_baseline"] = main_res["cpu_baseline"]
+        if "symbols_out" in main_res:
+            line["symbols_out"] = main_res["symbols_out"]
         if also:
             line["also"] = also
         if gemv:

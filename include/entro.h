@@ -177,6 +177,19 @@ entro_status entro_decode_dequant(const uint32_t *stream_dev, uint64_t stream_wo
 entro_status entro_decode_dequant_batched(const entro_tensor_desc *descs_host, int ntensors,
                                           void *cuda_stream);
 
+/*
+ * Parallel decode to integers, the form in which the paper's decoder hands the weights to
+ * its inference engine (Section 4: the engine works on the packed low-bit values).  Same
+ * descriptors as entro_decode_dequant_batched; scale and zero_point are not used, and
+ * out_fp16_dev points to bytes instead of fp16 values (16-byte aligned):
+ *   packed = 0: n bytes, one symbol per byte;
+ *   packed = 1: ceil(n / 2) bytes, symbol 2i in the low nibble of byte i and symbol 2i + 1
+ *               in the high one (alphabets of at most 16 symbols; chunk_symbols even).
+ * Asynchronous; errors as for the decode calls.
+ */
+entro_status entro_decode_symbols_batched(const entro_tensor_desc *descs_host, int ntensors, int packed,
+                                          void *cuda_stream);
+
 /* Host-resident input and output for one tensor of entro_decode_dequant_batched_host. */
 typedef struct {
     const uint32_t *stream_host;  /* stream_words words (pinned memory for full speed) */

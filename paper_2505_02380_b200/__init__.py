@@ -101,6 +101,7 @@ def lib():
         L.entro_decode_dequant.argtypes = [vp, u64, vp, u64, u32, C.POINTER(Codebook), C.c_float, C.c_int32, vp, vp]
         L.entro_decode_dequant_batched.argtypes = [C.POINTER(TensorDesc), i32, vp]
         L.entro_decode_dequant_batched_host.argtypes = [C.POINTER(TensorDesc), C.POINTER(HostIO), i32, vp]
+        L.entro_decode_symbols_batched.argtypes = [C.POINTER(TensorDesc), i32, i32, vp]
         L.entro_decode_dequant_gemv.argtypes = [C.POINTER(TensorDesc), C.POINTER(GemvIO), i32, vp]
         L.entro_gemv_fp16.argtypes = [vp, u32, u32, vp, vp, vp]
         L.entro_decode_dequant_static.argtypes = [C.POINTER(TensorDesc), i32, vp, vp]
@@ -123,7 +124,7 @@ def lib():
 EXPORTS = ["entro_quantize_tensor", "entro_histogram", "entro_build_codebook", "entro_stream_words",
            "entro_encode_bound_words", "entro_index_bytes", "entro_encode", "entro_decode_dequant",
            "entro_decode_dequant_batched", "entro_decode_dequant_batched_host", "entro_decode_dequant_static",
-           "entro_decode_dequant_gemv", "entro_gemv_fp16", "entro_last_device_status",
+           "entro_decode_dequant_gemv", "entro_gemv_fp16", "entro_decode_symbols_batched", "entro_last_device_status",
            "entro_set_decode_config", "entro_profile_begin", "entro_profile_read", "entro_kernel_launch_count",
            "entro_status_string"]
 
@@ -259,6 +260,22 @@ def entro_decode_dequant_batched(descs, stream: Optional[torch.cuda.Stream] = No
     if isinstance(descs, list):
         descs = desc_array(descs)
     _check(lib().entro_decode_dequant_batched(descs, len(descs), _stream(stream)), "entro_decode_dequant_batched")
+
+
+def make_desc_bytes(stream_words: torch.Tensor, index: torch.Tensor, n: int, chunk_symbols: int, cb: Codebook,
+                    out: torch.Tensor) -> TensorDesc:
+    """A descriptor for entro_decode_symbols_batched: out is a uint8 device tensor."""
+    d = make_desc_no_out(stream_words, index, n, chunk_symbols, cb, 1.0, 0)
+    d.out_fp16_dev = _dev(out, torch.uint8)
+    return d
+
+
+def entro_decode_symbols_batched(descs, packed: bool = False, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Decode to integer symbols (one per byte, or two 4-bit symbols per byte).  Asynchronous."""
+    if isinstance(descs, list):
+        descs = desc_array(descs)
+    _check(lib().entro_decode_symbols_batched(descs, len(descs), 1 if packed else 0, _stream(stream)),
+           "entro_decode_symbols_batched")
 
 
 def entro_decode_dequant_batched_host(descs, io, stream: Optional[torch.cuda.Stream] = None) -> None:

@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     __syncthreads();
     if (tid == 0 && unresolved4 > 6e-5f) aux.expm = 5u;
     const float d = (float)(tid - T.zero_point);
-    aux.val[tid] = __half_as_ushort(__float2half_rn(__fmul_rn(T.scale, d)));
+    aux.val[tid] = T.raw_symbols ? (uint16_t)tid : __half_as_ushort(__float2half_rn(__fmul_rn(T.scale, d)));
     __syncthreads();
     {
         uint32_t used = aux.offset[ENTRO_MAX_CODE_LEN] + count[ENTRO_MAX_CODE_LEN];
@@ -617,8 +617,8 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32
 // time: the ragged last chunk of a tensor, odd chunk sizes, chunks larger than the ring.
 // With G set the values are not stored but multiplied into the matrix-vector product.
 __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t* status, const DevTensor& T,
-                                                     const GemvTensor* G, uint32_t c, uint32_t excl, uint32_t my_bits,
-                                                     uint32_t lane)
+                                                     const GemvTensor* G, int sink, uint32_t c, uint32_t excl,
+                                                     uint32_t my_bits, uint32_t lane)
 {
     const uint64_t chunk_first = (uint64_t)c * T.chunk_symbols;
     const uint32_t m = (uint32_t)min((uint64_t)T.chunk_symbols, T.n - chunk_first);   // symbols in the chunk
@@ -639,6 +639,7 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
     for (uint32_t g = lane; g * 8u < m; g += kSubBlocks) {
         const uint32_t end = min(g * 8u + 8u, m);
         float acc = 0.f;
+        uint32_t low = 0;                       // the even symbol of a nibble pair
         for (uint32_t i = g * 8u; i < end; ++i) {
             gwin_refill(r);
             uint32_t e = kEscLen;
@@ -652,6 +653,13 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
                 const uint32_t col = (uint32_t)((chunk_first + i) % G->cols);
                 acc = fmaf(__half2float(__ushort_as_half((uint16_t)(e >> 16))),
                            __half2float(__ushort_as_half(__ldg(G->x + col))), acc);
+            } else if (sink == kSinkBytes) {
+                reinterpret_cast<uint8_t*>(T.out)[chunk_first + i] = (uint8_t)(e >> 16);
+            } else if (sink == kSinkNibbles) {
+                // pairs never straddle a group of 8 and chunks hold an even number of symbols
+                if (i & 1u) reinterpret_cast<uint8_t*>(T.out)[(chunk_first + i) >> 1] = (uint8_t)(low | ((e >> 16) << 4));
+                else if (i + 1u == m) reinterpret_cast<uint8_t*>(T.out)[(chunk_first + i) >> 1] = (uint8_t)(e >> 16);
+                else low = (e >> 16) & 15u;
             } else {
                 out[i] = (uint16_t)(e >> 16);
             }
@@ -682,6 +690,29 @@ struct EmitStore {
         dst += kSubBlocks;
     }
     __device__ __forceinline__ void finish() {}
+};
+
+// Integer output (the form the paper's decoder produces): the tables hold the symbols
+// themselves in their 16-bit value fields; a group of 8 leaves as 8 bytes ...
+struct EmitBytes {
+    uint2* dst;
+    __device__ __forceinline__ void operator()(uint4 v)
+    {
+        __stcs(dst, make_uint2(__byte_perm(v.x, v.y, 0x6420), __byte_perm(v.z, v.w, 0x6420)));
+        dst += kSubBlocks;
+    }
+};
+
+// ... or, for 4-bit symbols, as 4 bytes of two nibbles each, the earlier symbol low.
+struct EmitNibbles {
+    uint32_t* dst;
+    __device__ __forceinline__ void operator()(uint4 v)
+    {
+        const uint32_t a = __byte_perm(v.x, v.y, 0x6420), b = __byte_perm(v.z, v.w, 0x6420);   // s0..s3, s4..s7
+        const uint32_t ta = a | (a >> 4), tb = b | (b >> 4);                                   // bytes 0 and 2 hold the pairs
+        __stcs(dst, __byte_perm(ta, tb, 0x6420));
+        dst += kSubBlocks;
+    }
 };
 
 // Fused matrix-vector product: the 8 values are weights of one row of W (stored [rows, cols],
@@ -814,9 +845,10 @@ __device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status
     return L;
 }
 
-template <int K, bool kGemv>
+template <int K, int kSink>
 __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Ready& r, Lane L, uint32_t lane)
 {
+    constexpr bool kGemv = kSink == kSinkGemv;
     if (L.kind == kSkip) return;
     const DevTensor& T = *tensor_ptr<K>();
     const GemvTensor* G = kGemv ? gemv_ptr<K>() : nullptr;
@@ -835,7 +867,7 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         }
     }
     if (L.kind == kGeneral) {
-        decode_chunk_general(aux_ptr<K>(), status, T, G, r.c, L.start, L.end, lane);
+        decode_chunk_general(aux_ptr<K>(), status, T, G, kSink, r.c, L.start, L.end, lane);
         return;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
@@ -860,6 +892,19 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
         else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
         em.finish();
+    } else if (kSink == kSinkBytes) {
+        EmitBytes em;
+        em.dst = reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(T.out) + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
+        if (oct) rows_oct<K>(w, status, em, sub);
+        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+    } else if (kSink == kSinkNibbles) {
+        EmitNibbles em;
+        em.dst = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(T.out) + (((uint64_t)r.c * T.chunk_symbols) >> 1) +
+                                             lane * 4u);
+        if (oct) rows_oct<K>(w, status, em, sub);
+        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
     } else {
         EmitStore em;
         em.dst = reinterpret_cast<uint4*>(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
@@ -877,9 +922,10 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
 
 // item_start[t] = first work item of tensor t, item_start[ntensors] = number of items; an
 // item is up to tensors[t].item_chunks consecutive chunks of one tensor.
-// With kGemv the decoded weights are not stored: gemv[t] describes the matrix-vector product
-// they enter (the fused decode + dequantise + GEMV of a batch-1 token step).
-template <int K, bool kGemv>
+// kSink says where the decoded values go.  With kSinkGemv they are not stored: gemv[t]
+// describes the matrix-vector product they enter (the fused decode + dequantise + GEMV of a
+// batch-1 token step).
+template <int K, int kSink>
 __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __restrict__ tensors, int ntensors,
                                                          const uint32_t* __restrict__ item_start,
                                                          const TensorTables* __restrict__ tables,
@@ -887,6 +933,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                                                          uint32_t* __restrict__ control,
                                                          const GemvTensor* __restrict__ gemv)
 {
+    constexpr bool kGemv = kSink == kSinkGemv;
     // layout: [tables][aux][tensor]([gemv descriptor][x])[per-warp rings][over-read pad][mbarriers][index slots][item + claim slots]
     if (smem_addr(smem) != kSmemBase) {   // the lookups' address arithmetic would be wrong: refuse to run
         if (threadIdx.x == 0) atomicOr(control + 1, kStatInternal);
@@ -1002,7 +1049,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             __syncwarp();                           // every lane has read the slot before it is refilled
             c2 = r1.c == kNone ? kNone : claim();
             fetch_index(T, c2, other, lane);
-            decode_finish<K, kGemv>(cx, status, r0, L, lane);
+            decode_finish<K, kSink>(cx, status, r0, L, lane);
             if (r1.c == kNone) break;
             r0 = r1;
             sp = other;
@@ -1040,16 +1087,16 @@ Shape shape_for(const DecodeConfig& cfg, int max_smem, bool gemv = false)
     return s;
 }
 
-template <int K, bool kGemv>
+template <int K, int kSink>
 entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
                            const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
                            const GemvTensor* gemv, cudaStream_t s)
 {
-    Shape sh = shape_for(cfg, ws->max_smem_optin, kGemv);
+    Shape sh = shape_for(cfg, ws->max_smem_optin, kSink == kSinkGemv);
     if (sh.stage_bytes == 0) return ENTRO_ERR_UNSUPPORTED;
     static int configured_smem[64] = {0};
     if ((int)sh.smem > configured_smem[ws->device]) {
-        ENTRO_CUDA(cudaFuncSetAttribute(decode_kernel<K, kGemv>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        ENTRO_CUDA(cudaFuncSetAttribute(decode_kernel<K, kSink>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sh.smem));
         configured_smem[ws->device] = (int)sh.smem;
     }
@@ -1057,7 +1104,7 @@ entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTens
     if (grid > total_items) grid = total_items;
     const bool timed = ws->prof_used < ws->prof_cap;
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_start[ws->prof_used], s));
-    decode_kernel<K, kGemv><<<grid, cfg.warps_per_cta * 32, sh.smem, s>>>(
+    decode_kernel<K, kSink><<<grid, cfg.warps_per_cta * 32, sh.smem, s>>>(
         tensors, ntensors, item_start, tables, sh.stage_bytes, ws->control, gemv);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
@@ -1065,23 +1112,28 @@ entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTens
     return ENTRO_OK;
 }
 
-// gemv == nullptr: plain decode.
+template <int kSink>
+entro_status launch_decode_sink(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
+                                const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
+                                const GemvTensor* gemv, cudaStream_t s)
+{
+    switch (cfg.lut_bits) {
+        case 10: return launch_decode<10, kSink>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
+        case 11: return launch_decode<11, kSink>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
+        case 12: return launch_decode<12, kSink>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
+    }
+    return ENTRO_ERR_UNSUPPORTED;
+}
+
 entro_status launch_decode_any(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
                                const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
-                               cudaStream_t s, const GemvTensor* gemv = nullptr)
+                               cudaStream_t s, const GemvTensor* gemv = nullptr, int sink = kSinkFp16)
 {
-    if (gemv) {
-        switch (cfg.lut_bits) {
-            case 10: return launch_decode<10, true>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
-            case 11: return launch_decode<11, true>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
-            case 12: return launch_decode<12, true>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
-        }
-        return ENTRO_ERR_UNSUPPORTED;
-    }
-    switch (cfg.lut_bits) {
-        case 10: return launch_decode<10, false>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
-        case 11: return launch_decode<11, false>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
-        case 12: return launch_decode<12, false>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
+    if (gemv) return launch_decode_sink<kSinkGemv>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
+    switch (sink) {
+        case kSinkFp16: return launch_decode_sink<kSinkFp16>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
+        case kSinkBytes: return launch_decode_sink<kSinkBytes>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
+        case kSinkNibbles: return launch_decode_sink<kSinkNibbles>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
     }
     return ENTRO_ERR_UNSUPPORTED;
 }
@@ -1152,7 +1204,8 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, ItemPlan& plan, DevTensor& 
     if (per_item < 32u) per_item = 32u;
     t.item_chunks = per_item;
     plan.seen += nc;
-    t.pad[0] = t.pad[1] = 0;
+    t.raw_symbols = 0;
+    t.pad = 0;
     for (int j = 0; j < ENTRO_MAX_SYMBOLS; ++j) t.len[j] = j < d.cb.nsym ? d.cb.len[j] : 0;
     return (nc + t.item_chunks - 1) / t.item_chunks;
 }
@@ -1160,7 +1213,8 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, ItemPlan& plan, DevTensor& 
 }  // namespace
 
 // Upload descriptors, build the tables and run the persistent decode kernel.
-entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs, int ntensors, cudaStream_t s)
+entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs, int ntensors, cudaStream_t s,
+                                   int sink = kSinkFp16)
 {
     const DecodeConfig cfg = decode_config();
     ItemPlan plan = plan_items(cfg, descs, ntensors, ws->sm_count);
@@ -1187,6 +1241,7 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
         if (!descs[i].n) continue;
         hitems[k] = (uint32_t)items;
         items += fill_dev_tensor(descs[i], plan, ht[k]);
+        ht[k].raw_symbols = sink == kSinkFp16 ? 0u : 1u;
         if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
         ++k;
     }
@@ -1201,7 +1256,7 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     build_tables_kernel<<<live, 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
-    return launch_decode_any(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, s);
+    return launch_decode_any(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, s, nullptr, sink);
 }
 
 }  // namespace entro
@@ -1221,6 +1276,23 @@ extern "C" entro_status entro_decode_dequant_batched(const entro_tensor_desc* de
     Workspace* ws = workspace();
     if (!ws) return ENTRO_ERR_CUDA;
     return decode_batched_locked(ws, descs_host, ntensors, (cudaStream_t)cuda_stream);
+}
+
+extern "C" entro_status entro_decode_symbols_batched(const entro_tensor_desc* descs_host, int ntensors, int packed,
+                                                     void* cuda_stream)
+{
+    if (ntensors < 0 || (ntensors > 0 && !descs_host) || (packed != 0 && packed != 1)) return ENTRO_ERR_INVALID_ARG;
+    if (ntensors == 0) return ENTRO_OK;
+    for (int i = 0; i < ntensors; ++i) {
+        entro_status st = validate_desc(descs_host[i]);
+        if (st != ENTRO_OK) return st;
+        if (packed && descs_host[i].n && (descs_host[i].cb.nsym > 16 || (descs_host[i].chunk_symbols & 1u)))
+            return ENTRO_ERR_INVALID_ARG;
+    }
+    Guard g;
+    Workspace* ws = workspace();
+    if (!ws) return ENTRO_ERR_CUDA;
+    return decode_batched_locked(ws, descs_host, ntensors, (cudaStream_t)cuda_stream, packed ? kSinkNibbles : kSinkBytes);
 }
 
 extern "C" entro_status entro_decode_dequant(const uint32_t* stream_dev, uint64_t stream_words, const void* index_dev,

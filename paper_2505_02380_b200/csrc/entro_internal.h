@@ -32,7 +32,8 @@ struct DevTensor {
     float scale;
     int32_t zero_point;
     uint32_t item_chunks;         // chunks per work item of this tensor
-    uint32_t pad[2];
+    uint32_t raw_symbols;         // 1: the tables hold the symbols themselves, not dequantised values
+    uint32_t pad;
     uint8_t len[ENTRO_MAX_SYMBOLS];
 };
 static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vectors");
@@ -75,6 +76,14 @@ struct DecodeConfig {
     int warps_per_cta = 32;
     int ctas_per_sm = 1;
     int chunks_per_item = 1024;
+};
+
+// Where the decode kernel sends the decoded values.
+enum Sink : int {
+    kSinkFp16 = 0,      // dequantised fp16 values to the output tensor
+    kSinkGemv = 1,      // dequantised fp16 values into a matrix-vector product
+    kSinkBytes = 2,     // the symbols, one per byte
+    kSinkNibbles = 3    // the symbols, two per byte, the earlier one in the low nibble
 };
 
 // Per-device workspace owned by the library.

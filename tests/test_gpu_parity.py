@@ -133,6 +133,33 @@ def test_decode_flat_histograms(bits, chunk):
     assert_status_ok()
 
 
+@pytest.mark.parametrize("bits,chunk,packed", [(8, 4096, False), (4, 8192, False), (4, 8192, True), (4, 1024, True),
+                                               (8, 96, False), (4, 64, True)])
+def test_decode_to_integer_symbols(bits, chunk, packed):
+    """The paper's decoder hands integers to the inference engine: one symbol per byte, or two
+    4-bit symbols per byte.  Bit-exact against the oracle's quantised symbols."""
+    keep, descs, outs, refs = [], [], [], []
+    for n in (1, 2, 33, chunk - 1, chunk, 3 * chunk + 517, 40 * chunk + 5, 64 * chunk):
+        w_np, _ = _values(n, 0.02, 31 * n % 1000 + bits)
+        c = oracle.compress(w_np, bits, chunk)
+        s, ix = to_dev_stream(c.enc.stream), to_dev_index(c.enc)
+        out = torch.full(((n + 1) // 2 if packed else n,), 0xEE, dtype=torch.uint8, device="cuda")
+        keep += [s, ix]
+        descs.append(E.make_desc_bytes(s, ix, n, chunk, codebook_from_oracle(c), out))
+        outs.append(out)
+        q = c.q
+        if packed:
+            q2 = np.concatenate([q, np.zeros(n & 1, dtype=np.uint8)])
+            refs.append((q2[0::2] | (q2[1::2] << 4)).astype(np.uint8))
+        else:
+            refs.append(q)
+    E.entro_decode_symbols_batched(descs, packed)
+    torch.cuda.synchronize()
+    assert_status_ok()
+    for out, ref in zip(outs, refs):
+        assert np.array_equal(out.cpu().numpy(), ref)
+
+
 def test_decode_config1_single_tensor():
     """1024 x 1024, sigma 0.02, seed 0, asymmetric uint8, 4096-symbol chunks."""
     wl = workloads.single_tensor()
