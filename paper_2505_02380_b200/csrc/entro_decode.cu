@@ -330,7 +330,7 @@ __device__ __forceinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32
 // in place.  Out: the fp16 values in pairs, and s, the sum of the G entries: the group
 // stands iff (s & 0xffe0) == 0, that is, every cell was resolved (an unresolved one adds
 // 64) and fewer than 32 bits were used.  If it does not stand the caller repairs it with
-// repair_group, which needs only next, k and s: k grew by exactly s, next did not move.
+// rewind_group, which needs only next, k and s: k grew by exactly s, next did not move.
 #define ENTRO_LOOKUP(dst, win)                       \
     "cvt.rz.f32.u32 f, " win ";\n\t"                  \
     "mov.b32 a, f;\n\t"                               \
@@ -411,25 +411,38 @@ __device__ __forceinline__ uint32_t next_symbol(Win& r, uint32_t* status, LutKey
     return e;
 }
 
-// Repair of a group of G symbols that did not stand (kept inline: a call here would park
-// the caller's registers in local memory, which misses the small L1 left beside 228 KB of
-// shared memory).  Rebuilds the window as it was before the group from (k, next, s), then
-// takes the symbols one by one.
-template <int K, int G>
-__device__ __forceinline__ void repair_group(Win& r, uint32_t* status, LutKey key, uint32_t s, uint32_t& pk0,
-                                             uint32_t& pk1)
+// Rebuild the window as it was before a group that did not stand, from what the group
+// left: k grew by exactly s, next did not move after the refill.
+__device__ __forceinline__ void rewind_group(Win& r, uint32_t s)
 {
     const uint32_t valid = (uint32_t)win_valid_bits(r.k - s);   // 33 .. 64 bits were valid when the group began
     const uint32_t bit_addr = r.next * 8u - valid;              // where they begin, in bits of the shared window
     win_init<true>(r, (bit_addr >> 5) << 2, bit_addr & 31u);
+}
+
+// Repair of a group of two symbols that did not stand (kept inline: a call here would park
+// the caller's registers in local memory, which misses the small L1 left beside 228 KB of
+// shared memory): the symbols one by one, any code length.
+template <int K>
+__device__ __forceinline__ void repair_pair(Win& r, uint32_t* status, LutKey key, uint32_t s, uint32_t& pk)
+{
+    rewind_group(r, s);
     const uint32_t e0 = next_symbol<K, false>(r, status, key);
     const uint32_t e1 = next_symbol<K, false>(r, status, key);
-    pk0 = __byte_perm(e0, e1, 0x7632);
-    if (G == 4) {
-        const uint32_t e2 = next_symbol<K, false>(r, status, key);
-        const uint32_t e3 = next_symbol<K, false>(r, status, key);
-        pk1 = __byte_perm(e2, e3, 0x7632);
-    }
+    pk = __byte_perm(e0, e1, 0x7632);
+}
+
+// Repair of a group of four: almost always it merely used 32 bits or more, so two groups of
+// two stand; each of those falls back to repair_pair.
+template <int K>
+__device__ __forceinline__ void repair_quad(Win& r, uint32_t* status, LutKey key, uint32_t s, uint32_t& pk0, uint32_t& pk1)
+{
+    rewind_group(r, s);
+    uint32_t s2;
+    group2(r, key, pk0, s2);
+    if (__builtin_expect((s2 & 0xffe0u) != 0u, 0)) repair_pair<K>(r, status, key, s2, pk0);
+    group2(r, key, pk1, s2);
+    if (__builtin_expect((s2 & 0xffe0u) != 0u, 0)) repair_pair<K>(r, status, key, s2, pk1);
 }
 
 // Eight symbols of a 4-bit alphabet whose codes do not fit the table's window.
@@ -770,17 +783,14 @@ __device__ __forceinline__ void rows_single(Win& r, uint32_t* status, LutKey key
             for (int g = 0; g < 2; ++g) {
                 uint32_t s;
                 group4(r, key, pk[2 * g], pk[2 * g + 1], s);
-                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_group<K, 4>(r, status, key, s, pk[2 * g], pk[2 * g + 1]);
+                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_quad<K>(r, status, key, s, pk[2 * g], pk[2 * g + 1]);
             }
         } else {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 uint32_t s;
                 group2(r, key, pk[g], s);
-                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) {
-                    uint32_t none;
-                    repair_group<K, 2>(r, status, key, s, pk[g], none);
-                }
+                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_pair<K>(r, status, key, s, pk[g]);
             }
         }
         emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
