@@ -79,6 +79,7 @@ def lib():
         L.oracle_dequant.argtypes = [u8p, C.c_uint64, C.c_float, C.c_int, u16p]
         L.oracle_histogram.argtypes = [u8p, C.c_uint64, C.c_int, u64p]
         L.oracle_huffman_lengths.argtypes = [u64p, C.c_int, u8p]
+        L.oracle_length_limited_lengths.argtypes = [u64p, C.c_int, C.c_int, u8p]
         L.oracle_canonical_codes.argtypes = [u8p, C.c_int, u32p]
         L.oracle_num_chunks.restype = C.c_uint64
         L.oracle_num_chunks.argtypes = [C.c_uint64, C.c_uint32]
@@ -187,6 +188,14 @@ def huffman_lengths(counts: Sequence[int]) -> np.ndarray:
     counts = np.ascontiguousarray(counts, dtype=np.uint64)
     ln = np.zeros(counts.size, dtype=np.uint8)
     _check(lib().oracle_huffman_lengths(_ptr(counts, C.c_uint64), counts.size, _ptr(ln, C.c_uint8)))
+    return ln
+
+
+def length_limited_lengths(counts: Sequence[int], max_len: int) -> np.ndarray:
+    """Optimal code lengths with no code longer than max_len (package-merge)."""
+    counts = np.ascontiguousarray(counts, dtype=np.uint64)
+    ln = np.zeros(counts.size, dtype=np.uint8)
+    _check(lib().oracle_length_limited_lengths(_ptr(counts, C.c_uint64), counts.size, int(max_len), _ptr(ln, C.c_uint8)))
     return ln
 
 

@@ -286,6 +286,80 @@ int oracle_huffman_lengths(const uint64_t *counts, int nsym, uint8_t *len)
     return ORACLE_OK;
 }
 
+/* ------------------------------------------------------------------ length-limited lengths */
+
+/*
+ * Optimal prefix-code lengths under a cap: no code longer than max_len, total cost
+ * sum(count * length) minimal among such codes (the package-merge construction of Larmore
+ * and Hirschberg).  This departs from the paper, which uses the unrestricted Huffman code
+ * ("no other prefix code can offer a more efficient representation", Section 3); it is an
+ * optional format variant.  Steps, fixed so that exactly one answer exists:
+ *   - leaves = used symbols, ascending by (count, symbol);
+ *   - for level j = max_len down to 1: the level's list is the leaves merged with the
+ *     packages made at level j + 1 (none at level max_len), ascending by weight; on equal
+ *     weight a leaf comes before a package, leaves in their sorted order, packages in the
+ *     order in which they were made;
+ *   - the packages of level j are the consecutive pairs of its list (first + second,
+ *     third + fourth, ...; an odd last item is dropped);
+ *   - a symbol's length is the number of items among the first 2 * (n - 1) of level 1's
+ *     list that contain it, a package containing what its two halves contain.
+ * One used symbol gets length 1.  Fails if 2^max_len < n.
+ */
+int oracle_length_limited_lengths(const uint64_t *counts, int nsym, int max_len, uint8_t *len)
+{
+    if (!counts || !len || nsym < 1 || nsym > MAX_SYMBOLS || max_len < 1 || max_len > MAX_LEN) return ORACLE_ERR_ARG;
+    int order[MAX_SYMBOLS], n = 0;
+    for (int k = 0; k < nsym; ++k) { len[k] = 0; if (counts[k]) order[n++] = k; }
+    if (n == 0) return ORACLE_OK;
+    if (n == 1) { len[order[0]] = 1; return ORACLE_OK; }
+    if (max_len < 31 && (1u << max_len) < (unsigned)n) return ORACLE_ERR_TOO_LONG;
+    /* insertion sort by (count, symbol): symbols are already ascending, keep them so on ties */
+    for (int i = 1; i < n; ++i) {
+        int s = order[i], j = i - 1;
+        while (j >= 0 && counts[order[j]] > counts[s]) { order[j + 1] = order[j]; --j; }
+        order[j + 1] = s;
+    }
+    /* an item = its weight and, per leaf, how many times it contains that leaf */
+    enum { MAXI = 2 * MAX_SYMBOLS };
+    typedef struct { uint64_t w; uint8_t has[MAX_SYMBOLS]; } item;
+    item *cur = (item *)calloc(MAXI, sizeof(item)), *pk = (item *)calloc(MAXI, sizeof(item));
+    if (!cur || !pk) { free(cur); free(pk); return ORACLE_ERR_ARG; }
+    int npk = 0;
+    int ncur = 0;
+    for (int level = max_len; level >= 1; --level) {
+        /* merge leaves and packages */
+        int a = 0, b = 0;
+        ncur = 0;
+        while (a < n || b < npk) {
+            int take_leaf = b >= npk || (a < n && counts[order[a]] <= pk[b].w);
+            if (take_leaf) {
+                memset(&cur[ncur], 0, sizeof(item));
+                cur[ncur].w = counts[order[a]];
+                cur[ncur].has[a] = 1;
+                ++a;
+            } else {
+                cur[ncur] = pk[b];
+                ++b;
+            }
+            ++ncur;
+        }
+        if (level == 1) break;
+        npk = 0;
+        for (int i = 0; i + 1 < ncur; i += 2) {
+            pk[npk].w = cur[i].w + cur[i + 1].w;
+            for (int k = 0; k < n; ++k) pk[npk].has[k] = (uint8_t)(cur[i].has[k] + cur[i + 1].has[k]);
+            ++npk;
+        }
+    }
+    int need = 2 * (n - 1);
+    if (ncur < need) { free(cur); free(pk); return ORACLE_ERR_TOO_LONG; }
+    for (int i = 0; i < need; ++i)
+        for (int k = 0; k < n; ++k) len[order[k]] = (uint8_t)(len[order[k]] + cur[i].has[k]);
+    free(cur);
+    free(pk);
+    return ORACLE_OK;
+}
+
 /* ------------------------------------------------------------------ canonical codes */
 
 /*

@@ -5,6 +5,7 @@ pair merging (so: a full binary tree, Kraft sum exactly 1, average length within
 of the entropy, no cheaper prefix code exists), coding is lossless, and every segment
 decodes on its own from its known boundary."""
 import functools
+from fractions import Fraction
 import heapq
 import itertools
 import math
@@ -360,3 +361,70 @@ def test_long_codes_round_trip():
     enc = oracle.encode(q, ln, cd, 4096)
     q2, _ = oracle.decode_dequant(enc.stream, enc.offsets, q.size, 4096, ln, 1.0, 0)
     assert np.array_equal(q2, q)
+
+
+# ----------------------------------------------------------------------------- length-limited codes
+
+def _best_limited_cost(counts, max_len):
+    """Brute force: the cheapest Kraft-feasible length vector with every length <= max_len."""
+    used = [c for c in counts if c]
+    best = None
+    for ls in itertools.product(range(1, max_len + 1), repeat=len(used)):
+        if sum(2.0 ** -l for l in ls) <= 1.0 + 1e-12:
+            cost = sum(c * l for c, l in zip(used, ls))
+            best = cost if best is None else min(best, cost)
+    return best
+
+
+def test_length_limited_optimal_against_brute_force():
+    rng = np.random.default_rng(5)
+    for trial in range(60):
+        n = int(rng.integers(2, 7))
+        counts = rng.integers(1, 50, n).tolist() if trial % 3 else (2 ** rng.integers(0, 7, n)).tolist()
+        lo = int(np.ceil(np.log2(n)))
+        for max_len in range(max(lo, 1), 6):
+            ln = oracle.length_limited_lengths(counts, max_len)
+            assert ln.max() <= max_len
+            assert sum(Fraction(1, 2 ** int(l)) for l in ln) == 1          # complete code
+            assert int((np.array(counts) * ln).sum()) == _best_limited_cost(counts, max_len), (counts, max_len)
+
+
+def test_length_limited_reduces_to_huffman_cost_and_obeys_the_cap():
+    rng = np.random.default_rng(6)
+    for nsym in (16, 256):
+        w = workloads.make_values(1 << 18, 0.02, 900 + nsym).numpy()
+        bits = 4 if nsym == 16 else 8
+        q, _ = oracle.quantize_tensor(w, bits)
+        counts = oracle.histogram(q, nsym)
+        huff = oracle.huffman_lengths(counts)
+        cost_h = int((counts * huff.astype(np.uint64)).sum())
+        # a cap at or above the Huffman depth changes nothing about the cost
+        ln = oracle.length_limited_lengths(counts, int(huff.max()))
+        assert int((counts * ln.astype(np.uint64)).sum()) == cost_h
+        prev = None
+        for cap in sorted({int(huff.max()) - 1, 16, 12, 10}, reverse=True):
+            if (1 << cap) < int((counts > 0).sum()):
+                continue
+            ln = oracle.length_limited_lengths(counts, cap)
+            used = ln[counts > 0]
+            assert used.min() >= 1 and used.max() <= cap and not ln[counts == 0].any()
+            assert sum(Fraction(1, 2 ** int(l)) for l in used) == 1
+            cost = int((counts * ln.astype(np.uint64)).sum())
+            assert cost >= cost_h and (prev is None or cost >= prev)       # tighter cap, never cheaper
+            prev = cost
+            oracle.canonical_codes(ln)                                     # a valid canonical code exists
+
+
+def test_length_limited_hand_cases():
+    # cap 2 on four symbols forces the fixed-length code whatever the counts
+    assert oracle.length_limited_lengths([1, 1, 2, 100], 2).tolist() == [2, 2, 2, 2]
+    # Fibonacci counts a..f = 1 1 2 3 5 8 want depths 5 5 4 3 2 1; cap 4, merged by hand under the stated rule:
+    #   level 4: a1 b1 c2 d3 e5 f8                         packages P1=ab(2) P2=cd(5) P3=ef(13)
+    #   level 3: a1 b1 c2 P1 d3 e5 P2 f8 P3                packages Q1=ab(2) Q2=c+P1(4) Q3=de(8) Q4=P2+f(13)
+    #   level 2: a1 b1 c2 Q1 d3 Q2 e5 f8 Q3 Q4             packages R1=ab(2) R2=c+Q1(4) R3=d+Q2(7) R4=ef(13) R5
+    #   level 1: a b c R1 d R2 e R3 f R4 | R5              first 10 items: a b c {ab} d {cab} e {dcab} f {ef}
+    #   a, b appear 4 times, c 3 times, d, e, f twice
+    assert oracle.length_limited_lengths([1, 1, 2, 3, 5, 8], 4).tolist() == [4, 4, 3, 2, 2, 2]
+    assert oracle.length_limited_lengths([0, 9, 0], 5).tolist() == [0, 1, 0]
+    with pytest.raises(oracle.OracleError):
+        oracle.length_limited_lengths([1, 1, 1, 1, 1], 2)                  # five symbols need 3 bits
