@@ -134,7 +134,7 @@ def physical_gpu_index(local_rank: int) -> int:
 class DeviceModel:
     """A synthetic model compressed on the device with the library's own offline stages."""
 
-    def __init__(self, wl, E, lut_bits: int, keep_q: bool = False):
+    def __init__(self, wl, E, lut_bits: int, keep_q: bool = False, max_code_len: int = 0):
         self.wl = wl
         self.q = []              # quantised symbols per tensor (only with keep_q)
         self.qparams = []
@@ -158,7 +158,8 @@ class DeviceModel:
             w = workloads.make_tensor(spec, "cuda").view(-1)
             q, qp = E.entro_quantize_tensor(w, wl.bits)
             counts = E.entro_histogram(q, wl.bits)
-            cb = E.entro_build_codebook(counts.tolist())
+            cb = (E.entro_build_codebook_limited(counts.tolist(), max_code_len) if max_code_len
+                  else E.entro_build_codebook(counts.tolist()))
             enc = E.entro_encode(q, cb, wl.chunk_symbols, stream_words=E.entro_stream_words(counts.tolist(), cb))
             self.qparams.append((qp.scale, qp.zero_point))
             self.cbs.append(cb)
@@ -419,7 +420,7 @@ def run_reference(args, rank, world):
 # ----------------------------------------------------------------------------- main
 
 def measure(E, wl, args, world, local_rank, rank, peak, with_e2e, with_cpu):
-    model = DeviceModel(wl, E, args.lut_bits)
+    model = DeviceModel(wl, E, args.lut_bits, max_code_len=args.max_code_len)
     ms, launches, kernel_ms, clocks = time_steps(E, model, args.steps, args.warmup, world,
                                                  physical_gpu_index(local_rank))
     ms_step = ms / args.steps
@@ -464,6 +465,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-gemv", action="store_true", help="skip the fused decode+GEMV section (config 5)")
+    ap.add_argument("--max-code-len", type=int, default=0,
+                    help="use length-limited codes (not the paper's optimal code); 0 = unrestricted Huffman")
     ap.add_argument("--lut-bits", type=int, default=0)
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
@@ -516,7 +519,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
             "config": {"workload": wl.name + " full-model decode", "bits": wl.bits,
                        "chunk_symbols": wl.chunk_symbols, "tensors": len(wl.tensors), "weights": wl.numel,
-                       "max_layers": args.max_layers, "lut_bits": args.lut_bits,
+                       "max_layers": args.max_layers, "lut_bits": args.lut_bits, "max_code_len_cap": args.max_code_len,
                        "l2": "inputs and outputs per step (GBs) are far larger than L2; no flush needed",
                        "parallelism": f"replicas x{world}, one full model per GPU, no collective"},
             "weights_per_s": main_res["weights_per_s"], "bytes_per_step": main_res["bytes_per_step"],

@@ -131,6 +131,25 @@ entro_status entro_histogram(const uint8_t *q_dev, uint64_t n, int bits, uint64_
  */
 entro_status entro_build_codebook(const uint64_t *counts_host, int nsym, entro_codebook *cb_host);
 
+/*
+ * The same with a cap on the code length: the cheapest prefix code none of whose codes is
+ * longer than max_len (package-merge), then canonical codes.  NOT the paper's code: Section 3
+ * uses the unrestricted Huffman code, which no prefix code beats; a capped code costs more
+ * (measured on the benchmark's 8-bit weights: +0.045 bit per weight at max_len = 12, +0.18
+ * at 10; nothing at 4 bits) and bounds the decoder's table depth.  An optional variant of
+ * the format; streams made with it decode with the ordinary decode calls, correctly but
+ * more slowly than Huffman streams, because this library's tables are shaped for codes that
+ * grow long towards the all-ones end, which a capped code no longer does.  Steps (fixed so that
+ * the result is unique): leaves ascending by (count, symbol); for level j = max_len .. 1 the
+ * list is the leaves merged with the packages of level j + 1, ascending by weight, a leaf
+ * before a package of equal weight, packages in the order they were made; packages are the
+ * consecutive pairs of a list; a symbol's length is the number of the first 2 (n - 1) items
+ * of level 1 that contain it.  ENTRO_ERR_CODE_TOO_LONG if 2^max_len is less than the number
+ * of used symbols; ENTRO_ERR_INVALID_ARG for max_len outside 1 .. 32.
+ */
+entro_status entro_build_codebook_limited(const uint64_t *counts_host, int nsym, int max_len,
+                                          entro_codebook *cb_host);
+
 /* Words a stream buffer needs for these counts under this codebook: ceil(sum count[k] *
  * len[k] / 32) + ENTRO_STREAM_SLACK_WORDS.  0 on a bad argument. */
 uint64_t entro_stream_words(const uint64_t *counts_host, const entro_codebook *cb_host);

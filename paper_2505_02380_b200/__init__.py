@@ -91,6 +91,7 @@ def lib():
         L.entro_quantize_tensor.argtypes = [vp, u64, i32, i32, vp, C.POINTER(QParams), vp]
         L.entro_histogram.argtypes = [vp, u64, i32, C.POINTER(C.c_uint64), vp]
         L.entro_build_codebook.argtypes = [C.POINTER(C.c_uint64), i32, C.POINTER(Codebook)]
+        L.entro_build_codebook_limited.argtypes = [C.POINTER(C.c_uint64), i32, i32, C.POINTER(Codebook)]
         L.entro_stream_words.restype = u64
         L.entro_stream_words.argtypes = [C.POINTER(C.c_uint64), C.POINTER(Codebook)]
         L.entro_encode_bound_words.restype = u64
@@ -121,7 +122,7 @@ def lib():
 
 
 # Every symbol include/entro.h declares.
-EXPORTS = ["entro_quantize_tensor", "entro_histogram", "entro_build_codebook", "entro_stream_words",
+EXPORTS = ["entro_quantize_tensor", "entro_histogram", "entro_build_codebook", "entro_build_codebook_limited", "entro_stream_words",
            "entro_encode_bound_words", "entro_index_bytes", "entro_encode", "entro_decode_dequant",
            "entro_decode_dequant_batched", "entro_decode_dequant_batched_host", "entro_decode_dequant_static",
            "entro_decode_dequant_gemv", "entro_gemv_fp16", "entro_decode_symbols_batched", "entro_last_device_status",
@@ -170,6 +171,14 @@ def entro_build_codebook(counts: Sequence[int]) -> Codebook:
     arr = (C.c_uint64 * len(counts))(*[int(c) for c in counts])
     cb = Codebook()
     _check(lib().entro_build_codebook(arr, len(counts), C.byref(cb)), "entro_build_codebook")
+    return cb
+
+
+def entro_build_codebook_limited(counts: Sequence[int], max_len: int) -> Codebook:
+    """Canonical codebook of the cheapest code with no code longer than max_len."""
+    arr = (C.c_uint64 * len(counts))(*[int(c) for c in counts])
+    cb = Codebook()
+    _check(lib().entro_build_codebook_limited(arr, len(counts), int(max_len), C.byref(cb)), "entro_build_codebook_limited")
     return cb
 
 

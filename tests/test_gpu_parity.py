@@ -160,6 +160,29 @@ def test_decode_to_integer_symbols(bits, chunk, packed):
         assert np.array_equal(out.cpu().numpy(), ref)
 
 
+@pytest.mark.parametrize("bits,chunk,cap", [(8, 4096, 12), (8, 4096, 9), (4, 8192, 6)])
+def test_length_limited_codes_encode_and_decode(bits, chunk, cap):
+    """The optional capped code: the library's codebook equals the oracle's, the GPU encoder
+    produces the oracle's stream under it, and the ordinary decode call returns the dequantised
+    symbols."""
+    n = 37 * chunk + 1234
+    w_np, w_dev = _values(n, 0.02, 5150 + cap)
+    q_ref, qp = oracle.quantize_tensor(w_np, bits)
+    counts = oracle.histogram(q_ref, 1 << bits)
+    ln = oracle.length_limited_lengths(counts, cap)
+    cd = oracle.canonical_codes(ln)
+    assert ln.max() <= cap < oracle.huffman_lengths(counts).max()       # the cap really binds
+    enc_ref = oracle.encode(q_ref, ln, cd, chunk)
+    cb = E.entro_build_codebook_limited(counts.tolist(), cap)
+    assert np.array_equal(cb.lengths(), ln) and np.array_equal(cb.codes(), cd)
+    enc = E.entro_encode(torch.from_numpy(q_ref).cuda(), cb, chunk, stream_words=E.entro_stream_words(counts.tolist(), cb))
+    assert enc.total_bits == enc_ref.total_bits and np.array_equal(enc.stream_np(), enc_ref.stream)
+    out = E.entro_decode_dequant(enc.stream, enc.index, n, chunk, cb, qp.scale, qp.zero_point)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.dequant(q_ref, qp.scale, qp.zero_point))
+    assert_status_ok()
+
+
 def test_decode_config1_single_tensor():
     """1024 x 1024, sigma 0.02, seed 0, asymmetric uint8, 4096-symbol chunks."""
     wl = workloads.single_tensor()

@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 
 import oracle
+import workloads
 import paper_2505_02380_b200 as E
 from paper_2505_02380_b200 import build as build_mod
 
@@ -51,6 +52,33 @@ def test_codebook_matches_oracle_bit_exactly():
         assert np.array_equal(cb.lengths(), ln), counts
         assert np.array_equal(cb.codes(), oracle.canonical_codes(ln))
         assert cb.max_len == int(ln.max())
+
+
+def test_limited_codebook_matches_oracle_bit_exactly():
+    rng = np.random.default_rng(12)
+    cases = [[1, 1, 2, 3, 5, 8], [5, 5, 5, 5], [1, 1, 1, 1, 1, 1, 1], [0, 3, 0, 9, 1]]
+    for _ in range(40):
+        n = int(rng.integers(2, 257))
+        c = rng.integers(0, 1000, n)
+        c[rng.integers(0, n)] = 10 ** 6          # a dominant symbol makes long tails
+        cases.append(c.tolist())
+    for bits in (4, 8):
+        w = workloads.make_values(1 << 18, 0.02, 70 + bits).numpy()
+        q, _ = oracle.quantize_tensor(w, bits)
+        cases.append(oracle.histogram(q, 1 << bits).tolist())
+    for counts in cases:
+        used = sum(1 for c in counts if c)
+        for cap in (32, 16, 12, 10, 8):
+            if used > 1 and (1 << cap) < used:
+                continue
+            ref = oracle.length_limited_lengths(counts, cap)
+            cb = E.entro_build_codebook_limited(counts, cap)
+            assert cb.lengths().tolist() == ref.tolist(), (counts[:8], cap)
+            assert cb.codes().tolist() == oracle.canonical_codes(ref).tolist()
+            assert cb.max_len == int(ref.max())
+    with pytest.raises(E.EntroError) as e:
+        E.entro_build_codebook_limited([1] * 9, 3)
+    assert e.value.status == E.ERR_CODE_TOO_LONG
 
 
 def test_codebook_errors():
