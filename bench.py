@@ -53,6 +53,8 @@ def measured_peak():
 
 
 def pick_workload(name: str, max_layers):
+    if name.endswith("-paperbits"):
+        return workloads.with_paper_bit_rate(pick_workload(name[:-10], max_layers))
     if name.endswith("-gauss"):
         return workloads.with_matrix_kind(pick_workload(name[:-6], max_layers), "gauss")
     if name == "mistral8":
@@ -458,7 +460,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--workload", default="mistral8",
-                    choices=["mistral8", "mistral4", "smollm8", "phi3_4", "single", "mistral8-gauss", "mistral4-gauss"])
+                    choices=["mistral8", "mistral4", "smollm8", "phi3_4", "single", "mistral8-gauss", "mistral4-gauss",
+                             "mistral8-paperbits", "mistral4-paperbits"])
     ap.add_argument("--also", default="mistral4", help="second workload reported under 'also' ('' = none)")
     ap.add_argument("--max-layers", type=int, default=None, help="truncate the model (for profiling runs)")
     ap.add_argument("--e2e-steps", type=int, default=2)

@@ -57,3 +57,14 @@ def test_mistral_shaped_full_model_uint8():
 def test_mistral_shaped_full_model_uint4():
     _check_model(workloads.mistral_7b(bits=4),
                  ["layers.3.v_proj", "layers.20.o_proj", "layers.12.gate_proj", "final_norm"])
+
+
+def test_smollm_shaped_full_model_uint8():
+    """Config 2: 169 matrices + norm gains, unsigned or asymmetric per tensor by the mixed rule."""
+    wl = workloads.smollm_1p7b()
+    _check_model(wl, ["layers.5.k_proj", "layers.23.down_proj", "layers.11.post_attn_norm", "embed_tokens"])
+
+
+def test_phi3_shaped_full_model_uint4():
+    """Config 3: fused qkv / gate_up shapes, 4-bit symbols, 8192-symbol chunks."""
+    _check_model(workloads.phi3_mini_4k(), ["layers.0.qkv_proj", "layers.31.down_proj", "layers.16.o_proj", "final_norm"])
