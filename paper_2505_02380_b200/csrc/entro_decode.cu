@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
         // eight symbols per lookup pay off while eight codes usually fit the table's window
         aux.oct = (T.nsym <= 16 && mean_len * 8.f <= (float)lut_bits - 1.5f) ? 1u : 0u;
         // four lookups per window refill while their lengths almost always sum to < 32 bits
-        aux.group = mean_len <= 4.75f ? 4u : 2u;
+        aux.group = mean_len <= 6.0f ? 4u : 2u;
         aux.expm = 4u;
         unresolved4 = 0.f;
     }
@@ -623,6 +623,10 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32
     r.meta = ready_meta(at, bytes, cx.state, kStaged);
     cx.state++;
     if (now) issue_copy(cx, T, r, byte0, lane);
+    else if (lane == 0)   // no room yet: at least bring the bytes into L2 while the previous chunk is decoded
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const char*>(T.stream) + byte0),
+                     "r"(bytes)
+                     : "memory");
     return r;
 }
 
