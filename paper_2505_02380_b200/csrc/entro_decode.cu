@@ -23,8 +23,9 @@
 //     direct table of the same size would miss the tail.  m = 4 when that already covers
 //     the code (peaked, heavy-tailed histograms): the shared-memory copy is then replicated
 //     32 times, cell-major, so lane l only ever touches bank l and no lookup conflicts,
-//     whatever the data.  Flatter histograms get m = 5 and 16 copies (lanes l and l + 16
-//     share one: at most two wavefronts per lookup).
+//     whatever the data.  Flatter histograms get a larger m, up to 9, in the same 64 KB:
+//     every extra bit halves the number of copies (16 copies: lanes l and l + 16 share one,
+//     at most two wavefronts per lookup; ... ; one copy at m = 9).
 //   alphabets <= 16 symbols, eight symbols per lookup: the next K bits index a table of
 //     16-byte entries (eight fp16 values) and a byte table (bits used, 0 = no eight whole
 //     codes in K bits); one unreplicated copy of the exponent-indexed table serves the
@@ -47,7 +48,8 @@ constexpr uint32_t kOverRead = 2064;       // a lane fed garbage may read this f
 // window is the driver's).  The hand-written lookups address the tables as [offset + 1024];
 // the kernel checks the assumption before it does anything else.
 constexpr uint32_t kSmemBase = 1024;
-static_assert(kExpBitsMax == 5, "the lookups shift by 12 and mask: right for 4 and 5 mantissa bits only");
+static_assert(kExpBitsMin == 4 && kExpBitsMax == 9,
+              "the lookups shift the float bits by 12 whatever m is because cells * copies * 4 bytes = 64 KB");
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 // 32-bit word at a shared-window address.
@@ -61,7 +63,7 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
 // Shared-memory bytes of the lookup tables for a K-bit eight-symbol table.
 __host__ __device__ constexpr uint32_t lut_bytes(int K)
 {
-    return (17u << K) + 4u * kExpEntriesMax > 65536u ? (17u << K) + 4u * kExpEntriesMax : 65536u;
+    return (17u << K) + 4u * kExpEntriesMin > 65536u ? (17u << K) + 4u * kExpEntriesMin : 65536u;
 }
 
 // ------------------------------------------------------------------ table construction
@@ -87,7 +89,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     __shared__ DecodeAux aux;
     __shared__ uint32_t count[ENTRO_MAX_CODE_LEN + 1];
     __shared__ uint8_t len[ENTRO_MAX_SYMBOLS];
-    __shared__ float unresolved4;   // probability mass (by 2^-length) of codes a 4-bit-mantissa table leaves open
+    __shared__ float need_mass[16];   // probability mass (by 2^-length) of the codes that need j bits behind their first zero
     const int t = blockIdx.x;
     const int tid = threadIdx.x;
     const DevTensor& T = tensors[t];
@@ -121,22 +123,35 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
         aux.oct = (T.nsym <= 16 && mean_len * 8.f <= (float)lut_bits - 1.5f) ? 1u : 0u;
         // four lookups per window refill while their lengths almost always sum to < 32 bits
         aux.group = mean_len <= 6.0f ? 4u : 2u;
-        aux.expm = 4u;
-        unresolved4 = 0.f;
+        aux.expm = (uint32_t)kExpBitsMin;
+        for (int j = 0; j < 16; ++j) need_mass[j] = 0.f;
     }
     __syncthreads();
     if (l) {
         uint32_t rank = 0;
         for (int k = 0; k < tid; ++k) rank += (len[k] == l);
         aux.sorted[aux.offset[l] + rank] = (uint8_t)tid;
-        // would a table with 4 mantissa bits resolve this symbol's code?  It has r leading ones.
+        // how many bits behind the first zero does a table need to resolve this symbol's code?
+        // It has r leading ones, so l - r - 1 (none if the code is all ones).
         const uint32_t left = (aux.first_code[l] + rank) << (32u - l);
         uint32_t r = (uint32_t)__clz((int)~left);
         if (r > l) r = l;
-        if (l > r + 5u) atomicAdd(&unresolved4, exp2f(-(float)l));
+        const uint32_t need = l > r + 1u ? l - r - 1u : 0u;
+        atomicAdd(&need_mass[need < 15u ? need : 15u], exp2f(-(float)l));
     }
     __syncthreads();
-    if (tid == 0 && unresolved4 > 6e-5f) aux.expm = 5u;
+    if (tid == 0 && !aux.oct) {
+        // the smallest table that leaves less than 6e-5 of the symbols to the repair path
+        float open = 0.f;
+        uint32_t m = (uint32_t)kExpBitsMax;
+        for (int j = 15; j > kExpBitsMax; --j) open += need_mass[j];
+        while (m > (uint32_t)kExpBitsMin && open + need_mass[m] <= 6e-5f) {
+            open += need_mass[m];
+            --m;
+        }
+        aux.expm = m;
+    }
+    __syncthreads();
     const float d = (float)(tid - T.zero_point);
     aux.val[tid] = T.raw_symbols ? (uint16_t)tid : __half_as_ushort(__float2half_rn(__fmul_rn(T.scale, d)));
     __syncthreads();
@@ -195,7 +210,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
                 }
                 if (ok) entry = ((uint32_t)aux.val[sym] << 16) | sl;
             }
-            out.exp_lut[i] = entry;
+            (aux.oct ? out.exp_small : out.exp_lut())[i] = entry;
         }
     }
     const uint32_t* src = reinterpret_cast<const uint32_t*>(&aux);
@@ -290,15 +305,16 @@ __device__ __forceinline__ void gwin_refill(GlobalWin& r)
 
 // How a lane addresses its copy of the exponent-indexed table (which starts at the
 // beginning of shared memory, cell-major): byte offset = ((float bits >> 12) & mask) | lane.
-// m = 4: 32 copies, cells 128 bytes apart; m = 5: 16 copies, 64 bytes apart.
+// 32 << m cells, 32 >> (m - 4) copies, cells (128 >> (m - 4)) bytes apart: always 64 KB, and the
+// cell index (float bits 27 .. 23 - m) always lands on its byte offset by a shift of 12.
 struct LutKey {
     uint32_t mask, lane;
 };
 __device__ __forceinline__ LutKey lut_key(uint32_t expm, uint32_t lane)
 {
     LutKey k;
-    k.mask = expm == 4u ? 0xff80u : 0xffc0u;
-    k.lane = (expm == 4u ? lane : (lane & 15u)) * 4u;
+    k.mask = ((32u << expm) - 1u) << (11u - expm);
+    k.lane = (lane & ((32u >> (expm - 4u)) - 1u)) * 4u;
     return k;
 }
 
@@ -400,8 +416,7 @@ __device__ __forceinline__ uint32_t next_symbol(Win& r, uint32_t* status, LutKey
     const uint32_t inv = kOct ? ~r.hi : r.hi;
     uint32_t e;
     if (kOct) {
-        const uint32_t m = reinterpret_cast<const DecodeAux*>(smem + lut_bytes(K))->expm;
-        const uint32_t cell = (__float_as_uint(__uint2float_rz(inv)) >> (23u - m)) & ((32u << m) - 1u);
+        const uint32_t cell = (__float_as_uint(__uint2float_rz(inv)) >> (23 - kExpBitsMin)) & (uint32_t)(kExpEntriesMin - 1);
         e = *reinterpret_cast<const uint32_t*>(smem + (17u << K) + cell * 4u);
     } else {
         e = exp_lookup(key, inv);
@@ -1026,14 +1041,13 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                 uint4* s2 = reinterpret_cast<uint4*>(smem + (16u << K));
                 for (uint32_t i = threadIdx.x; i < (1u << K) / 16; i += blockDim.x) s2[i] = __ldg(g2 + i);
                 uint32_t* s3 = reinterpret_cast<uint32_t*>(smem + (17u << K));
-                for (uint32_t i = threadIdx.x; i < (uint32_t)kExpEntriesMax; i += blockDim.x) s3[i] = __ldg(tt->exp_lut + i);
+                for (uint32_t i = threadIdx.x; i < (uint32_t)kExpEntriesMin; i += blockDim.x) s3[i] = __ldg(tt->exp_small + i);
             } else {
-                // cell-major copies: 32 of them (word cell * 32 + lane sits in lane's bank) or 16
+                // cell-major copies, 64 KB in all: word w holds cell w / copies
                 uint32_t* s1 = reinterpret_cast<uint32_t*>(smem);
-                const uint32_t m = __ldg(&tt->aux.expm);
-                const uint32_t copies = m == 4u ? 32u : 16u;
-                for (uint32_t cell = warp; cell < (32u << m); cell += warps)
-                    s1[cell * copies + (lane & (copies - 1u))] = __ldg(tt->exp_lut + cell);
+                const uint32_t shift = 9u - __ldg(&tt->aux.expm);       // log2 of the number of copies
+                for (uint32_t w = threadIdx.x; w < (uint32_t)kExpEntriesMax; w += blockDim.x)
+                    s1[w] = __ldg(tt->exp_lut() + (w >> shift));
             }
             __syncthreads();
         }

@@ -10,8 +10,9 @@ namespace entro {
 
 constexpr int kSubBlocks = ENTRO_SUB_BLOCKS;
 constexpr int kMaxLutBits = 12;               // widest window of the eight-symbol table
-constexpr int kExpBitsMax = 5;                // mantissa bits of the exponent-indexed table: 4 or 5 per tensor
-constexpr int kExpEntriesMax = 32 << kExpBitsMax;
+constexpr int kExpBitsMin = 4, kExpBitsMax = 9;   // mantissa bits of the exponent-indexed table, chosen per tensor
+constexpr int kExpEntriesMax = 32 << kExpBitsMax; // 16384 cells of 4 bytes: the 64 KB the 32 copies of the smallest take
+constexpr int kExpEntriesMin = 32 << kExpBitsMin;
 
 // Device status bits (OR-ed by kernels, read by entro_last_device_status).
 constexpr uint32_t kStatCorrupt = 1u;         // index / stream / codebook disagree
@@ -64,12 +65,17 @@ static_assert(sizeof(DecodeAux) % 16 == 0, "DecodeAux is copied as 16-byte vecto
 
 // Everything the decode kernel loads into shared memory when it switches tensor.
 struct TensorTables {
-    uint4 oct_val[1u << kMaxLutBits];      // eight fp16 values per window (oct mode)
-    uint8_t oct_len[1u << kMaxLutBits];    // bits they use, 0 = not eight whole codes
-    uint32_t exp_lut[kExpEntriesMax];      // value << 16 | length, or length 64; 32 << aux.expm cells in use
+    // oct mode: eight fp16 values per window.  Otherwise the same 64 KB hold the exponent-indexed
+    // table, 32 << aux.expm cells of value << 16 | length (length 64 = unresolved).
+    uint4 oct_val[1u << kMaxLutBits];
+    uint8_t oct_len[1u << kMaxLutBits];    // oct mode: bits the eight codes use, 0 = not eight whole codes
+    uint32_t exp_small[kExpEntriesMin];    // oct mode: 4-bit-mantissa exponent-indexed table for the repair path
     DecodeAux aux;
+    __host__ __device__ uint32_t* exp_lut() { return reinterpret_cast<uint32_t*>(oct_val); }
+    __host__ __device__ const uint32_t* exp_lut() const { return reinterpret_cast<const uint32_t*>(oct_val); }
 };
 static_assert(sizeof(TensorTables) % 16 == 0, "TensorTables is copied as 16-byte vectors");
+static_assert(sizeof(uint4) * (1u << kMaxLutBits) >= 4u * kExpEntriesMax, "the large exponent table shares the oct values' space");
 
 struct DecodeConfig {
     int lut_bits = 12;
