@@ -307,14 +307,15 @@ def measure_gemv(E, max_layers, reps=5):
             views.append(out.view(spec.rows, spec.cols))
             comp_bytes += (enc.total_bits + 7) // 8 + enc.index.numel() + 2 * (spec.rows + spec.cols)
             n_weights += spec.numel
-        per_layer.append((E.desc_array(descs_f), E.desc_array(descs_u), xs, ys, shapes, views))
+        per_layer.append((E.desc_array(descs_f), E.desc_array(descs_u), xs, ys, shapes, views,
+                          E.make_gemv_io(xs, ys, shapes)))
 
     def fused():
-        for df, du, xs, ys, shapes, views in per_layer:
-            E.entro_decode_dequant_gemv(df, xs, shapes, ys)
+        for df, du, xs, ys, shapes, views, io in per_layer:
+            E.entro_decode_dequant_gemv(df, io=io)
 
     def unfused():
-        for df, du, xs, ys, shapes, views in per_layer:
+        for df, du, xs, ys, shapes, views, io in per_layer:
             E.entro_decode_dequant_batched(du)
             for v, x, y in zip(views, xs, ys):
                 E.entro_gemv_fp16(v, x, y)

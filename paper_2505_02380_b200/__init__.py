@@ -309,18 +309,29 @@ def make_desc_no_out(stream_words: torch.Tensor, index: torch.Tensor, n: int, ch
     return d
 
 
-def entro_decode_dequant_gemv(descs, xs: Sequence[torch.Tensor], shapes: Sequence, ys: Optional[List[torch.Tensor]] = None,
-                              stream: Optional[torch.cuda.Stream] = None) -> List[torch.Tensor]:
-    """descs[i]: compressed W_i of shape shapes[i] = (rows, cols); xs[i]: fp16 vector of cols values.
-    -> fp16 vectors y_i = W_i x_i.  Asynchronous."""
-    if isinstance(descs, list):
-        descs = desc_array(descs)
-    n = len(descs)
-    if ys is None:
-        ys = [torch.empty(shapes[i][0], dtype=torch.float16, device=xs[i].device) for i in range(n)]
+def make_gemv_io(xs: Sequence[torch.Tensor], ys: Sequence[torch.Tensor], shapes: Sequence):
+    """The ctypes array entro_decode_dequant_gemv takes, for callers that repeat a call and want
+    to marshal once.  shapes[i] = (rows, cols) of W_i; xs[i] has cols, ys[i] rows fp16 values."""
+    n = len(xs)
     io = (GemvIO * n)()
     for i in range(n):
         io[i] = GemvIO(int(shapes[i][0]), int(shapes[i][1]), _dev(xs[i], torch.float16), _dev(ys[i], torch.float16))
+    return io
+
+
+def entro_decode_dequant_gemv(descs, xs: Optional[Sequence[torch.Tensor]] = None, shapes: Optional[Sequence] = None,
+                              ys: Optional[List[torch.Tensor]] = None, stream: Optional[torch.cuda.Stream] = None,
+                              io=None):
+    """descs[i]: compressed W_i of shape shapes[i] = (rows, cols); xs[i]: fp16 vector of cols values.
+    -> fp16 vectors y_i = W_i x_i (the ys given, or new ones).  Pass io = make_gemv_io(...) instead of
+    xs / shapes / ys to skip the marshalling.  Asynchronous."""
+    if isinstance(descs, list):
+        descs = desc_array(descs)
+    n = len(descs)
+    if io is None:
+        if ys is None:
+            ys = [torch.empty(shapes[i][0], dtype=torch.float16, device=xs[i].device) for i in range(n)]
+        io = make_gemv_io(xs, ys, shapes)
     _check(lib().entro_decode_dequant_gemv(descs, io, n, _stream(stream)), "entro_decode_dequant_gemv")
     return ys
 
