@@ -220,8 +220,10 @@ typedef struct {
 /*
  * End-to-end form with host buffers: for every tensor, copy stream and index from
  * io_host[i] to the device buffers named in descs_host[i], decode + dequantise, and copy
- * the fp16 result back to io_host[i].out_fp16_host.  Copies and kernels are issued on
- * cuda_stream; returns after everything has completed (synchronises).
+ * the fp16 result back to io_host[i].out_fp16_host.  The work is ordered after what
+ * cuda_stream already holds; inside the call, uploads, decodes and downloads of different
+ * groups of tensors overlap on two copy streams of the library's own.  Returns after
+ * everything has completed (synchronises cuda_stream).
  */
 entro_status entro_decode_dequant_batched_host(const entro_tensor_desc *descs_host,
                                                const entro_host_io *io_host, int ntensors,

@@ -1341,38 +1341,80 @@ extern "C" entro_status entro_decode_dequant(const uint32_t* stream_dev, uint64_
     return entro_decode_dequant_batched(&d, 1, cuda_stream);
 }
 
+namespace entro {
+namespace {
+
+bool copy_streams_ready(Workspace* ws)
+{
+    if (ws->copy_in) return true;
+    if (cudaStreamCreateWithFlags(&ws->copy_in, cudaStreamNonBlocking) != cudaSuccess) return false;
+    if (cudaStreamCreateWithFlags(&ws->copy_out, cudaStreamNonBlocking) != cudaSuccess) return false;
+    if (cudaEventCreateWithFlags(&ws->ev_edge, cudaEventDisableTiming) != cudaSuccess) return false;
+    for (int i = 0; i < Workspace::kCopyGroups; ++i) {
+        if (cudaEventCreateWithFlags(&ws->ev_in[i], cudaEventDisableTiming) != cudaSuccess) return false;
+        if (cudaEventCreateWithFlags(&ws->ev_dec[i], cudaEventDisableTiming) != cudaSuccess) return false;
+    }
+    return true;
+}
+
+}  // namespace
+}  // namespace entro
+
+// The tensors are cut into groups; uploads, decodes and downloads of different groups
+// overlap: group g's streams travel host-to-device on one copy stream while group g - 1 is
+// decoded on the caller's stream and group g - 2's fp16 result travels back on another.
 extern "C" entro_status entro_decode_dequant_batched_host(const entro_tensor_desc* descs, const entro_host_io* io,
                                                           int ntensors, void* cuda_stream)
 {
     if (ntensors < 0 || (ntensors > 0 && (!descs || !io))) return ENTRO_ERR_INVALID_ARG;
     if (ntensors == 0) return ENTRO_OK;
     cudaStream_t s = (cudaStream_t)cuda_stream;
+    uint64_t out_bytes = 0;
     for (int i = 0; i < ntensors; ++i) {
         if (!descs[i].n) continue;
         if (!io[i].stream_host || !io[i].index_host || !io[i].out_fp16_host) return ENTRO_ERR_INVALID_ARG;
         entro_status st = validate_desc(descs[i]);
         if (st != ENTRO_OK) return st;
+        out_bytes += descs[i].n * 2;
     }
-    for (int i = 0; i < ntensors; ++i) {
-        const entro_tensor_desc& d = descs[i];
-        if (!d.n) continue;
-        ENTRO_CUDA(cudaMemcpyAsync(const_cast<uint32_t*>(d.stream_dev), io[i].stream_host, d.stream_words * 4,
-                                   cudaMemcpyHostToDevice, s));
-        ENTRO_CUDA(cudaMemcpyAsync(const_cast<void*>(d.index_dev), io[i].index_host,
-                                   entro_index_bytes(d.n, d.chunk_symbols), cudaMemcpyHostToDevice, s));
-    }
-    {
-        Guard g;
-        Workspace* ws = workspace();
-        if (!ws) return ENTRO_ERR_CUDA;
-        entro_status st = decode_batched_locked(ws, descs, ntensors, s);
+    Guard g;
+    Workspace* ws = workspace();
+    if (!ws || !copy_streams_ready(ws)) return ENTRO_ERR_CUDA;
+    // groups of consecutive tensors, about equal in output bytes
+    const uint64_t per_group = out_bytes / Workspace::kCopyGroups + 1;
+    // the copy streams start after what the caller has queued, and the caller's stream ends after them
+    ENTRO_CUDA(cudaEventRecord(ws->ev_edge, s));
+    ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_in, ws->ev_edge, 0));
+    ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_out, ws->ev_edge, 0));
+    int first = 0, group = 0;
+    while (first < ntensors) {
+        int last = first;
+        uint64_t bytes = 0;
+        while (last < ntensors && (bytes < per_group || group == Workspace::kCopyGroups - 1)) bytes += descs[last++].n * 2;
+        for (int i = first; i < last; ++i) {
+            const entro_tensor_desc& d = descs[i];
+            if (!d.n) continue;
+            ENTRO_CUDA(cudaMemcpyAsync(const_cast<uint32_t*>(d.stream_dev), io[i].stream_host, d.stream_words * 4,
+                                       cudaMemcpyHostToDevice, ws->copy_in));
+            ENTRO_CUDA(cudaMemcpyAsync(const_cast<void*>(d.index_dev), io[i].index_host,
+                                       entro_index_bytes(d.n, d.chunk_symbols), cudaMemcpyHostToDevice, ws->copy_in));
+        }
+        ENTRO_CUDA(cudaEventRecord(ws->ev_in[group], ws->copy_in));
+        ENTRO_CUDA(cudaStreamWaitEvent(s, ws->ev_in[group], 0));
+        entro_status st = decode_batched_locked(ws, descs + first, last - first, s);
         if (st != ENTRO_OK) return st;
+        ENTRO_CUDA(cudaEventRecord(ws->ev_dec[group], s));
+        ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_out, ws->ev_dec[group], 0));
+        for (int i = first; i < last; ++i) {
+            const entro_tensor_desc& d = descs[i];
+            if (!d.n) continue;
+            ENTRO_CUDA(cudaMemcpyAsync(io[i].out_fp16_host, d.out_fp16_dev, d.n * 2, cudaMemcpyDeviceToHost, ws->copy_out));
+        }
+        first = last;
+        ++group;
     }
-    for (int i = 0; i < ntensors; ++i) {
-        const entro_tensor_desc& d = descs[i];
-        if (!d.n) continue;
-        ENTRO_CUDA(cudaMemcpyAsync(io[i].out_fp16_host, d.out_fp16_dev, d.n * 2, cudaMemcpyDeviceToHost, s));
-    }
+    ENTRO_CUDA(cudaEventRecord(ws->ev_edge, ws->copy_out));
+    ENTRO_CUDA(cudaStreamWaitEvent(s, ws->ev_edge, 0));
     ENTRO_CUDA(cudaStreamSynchronize(s));
     return ENTRO_OK;
 }

@@ -106,6 +106,10 @@ struct Workspace {
     size_t pinned_bytes = 0;
     cudaEvent_t upload_done = nullptr; // last async read of `pinned` by the device
     bool upload_pending = false;
+    // copy streams and events of the host-buffer entry point (made on first use)
+    static constexpr int kCopyGroups = 48;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_in[kCopyGroups] = {}, ev_dec[kCopyGroups] = {}, ev_edge = nullptr;
     // optional timing of the decode kernel (entro_profile_begin / entro_profile_read)
     cudaEvent_t* prof_start = nullptr;
     cudaEvent_t* prof_stop = nullptr;
