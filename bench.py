@@ -16,6 +16,7 @@ from __future__ import annotations
 
 import argparse
 import ctypes as C
+import dataclasses
 import json
 import os
 import sys
@@ -471,6 +472,8 @@ def main():
     ap.add_argument("--no-gemv", action="store_true", help="skip the fused decode+GEMV section (config 5)")
     ap.add_argument("--max-code-len", type=int, default=0,
                     help="use length-limited codes (not the paper's optimal code); 0 = unrestricted Huffman")
+    ap.add_argument("--chunk-symbols", type=int, default=0,
+                    help="code the main workload with this chunk size instead of its own (a multiple of 256)")
     ap.add_argument("--lut-bits", type=int, default=0)
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
@@ -499,6 +502,8 @@ def main():
     peak = measured_peak()
 
     wl = pick_workload(args.workload, args.max_layers)
+    if args.chunk_symbols:
+        wl = dataclasses.replace(wl, chunk_symbols=args.chunk_symbols)
     main_res = measure(E, wl, args, world, local_rank, rank, peak, not args.no_e2e, not args.no_cpu)
     main_res.pop("model")
     also = None

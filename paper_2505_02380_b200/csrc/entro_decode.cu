@@ -339,72 +339,96 @@ __device__ __forceinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32
     return ((uint32_t)aux->val[sym] << 16) | len;
 }
 
-// One group of lookups of an 8-bit alphabet, hand-scheduled.  In: the inverted window
-// (hi, lo, k, next) and the lane's table key.  The refill is predicated (no branch), the G
-// lookups read the window at the running sum of the entries before them (a funnel shift
-// uses the low five bits, the length sums), and the window is advanced by the final sum
-// in place.  Out: the fp16 values in pairs, and s, the sum of the G entries: the group
-// stands iff (s & 0xffe0) == 0, that is, every cell was resolved (an unresolved one adds
-// 64) and fewer than 32 bits were used.  If it does not stand the caller repairs it with
-// rewind_group, which needs only next, k and s: k grew by exactly s, next did not move.
+// Reader of the grouped lookups of 8-bit alphabets: two consecutive stream words
+// (complemented) in registers and a bit position whose low five bits say where in w0 the
+// next code starts.  Only those five bits and bit 5 (has a word boundary been crossed?) are
+// ever used, so the upper bits of pos may hold anything.
+struct Cur {
+    uint32_t w0, w1;
+    uint32_t pos;
+    uint32_t next;            // shared-window address of the word after w1
+};
+
+__device__ __forceinline__ void cur_init(Cur& c, uint32_t bit_addr)
+{
+    const uint32_t a = (bit_addr >> 5) << 2;
+    c.w0 = ~lds32(a);
+    c.w1 = ~lds32(a + 4);
+    c.next = a + 8;
+    c.pos = bit_addr;
+}
+
+// Shared-window bit address the reader stands at.
+__device__ __forceinline__ uint32_t cur_bit_addr(const Cur& c) { return (c.next - 8u) * 8u + (c.pos & 31u); }
+
+// One group of lookups, hand-scheduled.  The group sees the 32 bits that start at the
+// reader's position (one funnel shift of the two words) and nothing behind them: lookup i
+// reads them shifted left by the lengths of the symbols before it (a funnel shift uses the
+// low five bits of the running sum of the entries), zeros moving in from the right.  Those
+// zeros cannot mislead a lookup whose code ends inside the 32 bits: a cell is resolved only
+// if every window that maps to it begins with the same code, whatever follows.  s is the sum
+// of the G entries: the group stands iff (s & 0xffe0) == 0, that is, every cell was resolved
+// (an unresolved one adds 64) and fewer than 32 bits were used, so all codes did end inside
+// the 32 bits.  Then the position moves on by s and, if that crosses into the next word
+// (bit 5 of the position flips), w1 becomes w0 and one new word is pulled in, predicated.
+// If the group does not stand the caller repairs it from rewind_group, which needs only
+// pos, next and s.
 #define ENTRO_LOOKUP(dst, win)                       \
     "cvt.rz.f32.u32 f, " win ";\n\t"                  \
     "mov.b32 a, f;\n\t"                               \
     "shr.u32 a, a, 12;\n\t"                           \
     "lop3.b32 a, a, %8, %7, 0xEA;\n\t"                \
     "ld.shared.b32 " dst ", [a+1024];\n\t"
-#define ENTRO_REFILL                                 \
-    "and.b32 t, %2, 0x8000;\n\t"                      \
-    "setp.eq.u32 p, t, 0;\n\t"                        \
-    "@p ld.shared.b32 w, [%3];\n\t"                   \
+#define ENTRO_OPEN                                   \
+    "shf.l.wrap.b32 h, %1, %0, %2;\n\t"
+#define ENTRO_MOVE_ON                                \
+    "add.u32 t, %2, %6;\n\t"                          \
+    "xor.b32 a, t, %2;\n\t"                           \
+    "mov.b32 %2, t;\n\t"                              \
+    "and.b32 a, a, 32;\n\t"                           \
+    "setp.ne.u32 p, a, 0;\n\t"                        \
+    "@p mov.b32 %0, %1;\n\t"                          \
+    "@p ld.shared.b32 t, [%3];\n\t"                   \
     "@p add.u32 %3, %3, 4;\n\t"                       \
-    "@p not.b32 w, w;\n\t"                            \
-    "@p shf.l.wrap.b32 t, w, 0, %2;\n\t"              \
-    "@p or.b32 %0, %0, t;\n\t"                        \
-    "@p shf.l.wrap.b32 %1, 0, w, %2;\n\t"             \
-    "@p add.u32 %2, %2, 0xffffffe0;\n\t"
-#define ENTRO_ADVANCE                                \
-    "shf.l.wrap.b32 %0, %1, %0, %6;\n\t"              \
-    "shf.l.wrap.b32 %1, 0, %1, %6;\n\t"               \
-    "add.u32 %2, %2, %6;\n\t"
+    "@p not.b32 %1, t;\n\t"
 
-__device__ __forceinline__ void group4(Win& r, LutKey key, uint32_t& pk0, uint32_t& pk1, uint32_t& s)
+__device__ __forceinline__ void group4(Cur& c, LutKey key, uint32_t& pk0, uint32_t& pk1, uint32_t& s)
 {
     asm volatile(
         "{\n\t"
         ".reg .pred p;\n\t"
-        ".reg .b32 t, w, a, e0, e1, e2, e3;\n\t"
-        ".reg .f32 f;\n\t" ENTRO_REFILL ENTRO_LOOKUP("e0", "%0")
-        "shf.l.wrap.b32 w, %1, %0, e0;\n\t" ENTRO_LOOKUP("e1", "w")
+        ".reg .b32 t, w, a, h, e0, e1, e2, e3;\n\t"
+        ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("e0", "h")
+        "shf.l.wrap.b32 w, 0, h, e0;\n\t" ENTRO_LOOKUP("e1", "w")
         "add.u32 %6, e0, e1;\n\t"
-        "shf.l.wrap.b32 w, %1, %0, %6;\n\t" ENTRO_LOOKUP("e2", "w")
+        "shf.l.wrap.b32 w, 0, h, %6;\n\t" ENTRO_LOOKUP("e2", "w")
         "add.u32 %6, %6, e2;\n\t"
-        "shf.l.wrap.b32 w, %1, %0, %6;\n\t" ENTRO_LOOKUP("e3", "w")
+        "shf.l.wrap.b32 w, 0, h, %6;\n\t" ENTRO_LOOKUP("e3", "w")
         "add.u32 %6, %6, e3;\n\t"
         "prmt.b32 %4, e0, e1, 0x7632;\n\t"
-        "prmt.b32 %5, e2, e3, 0x7632;\n\t" ENTRO_ADVANCE "}"
-        : "+r"(r.hi), "+r"(r.lo), "+r"(r.k), "+r"(r.next), "=&r"(pk0), "=&r"(pk1), "=&r"(s)
+        "prmt.b32 %5, e2, e3, 0x7632;\n\t" ENTRO_MOVE_ON "}"
+        : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk0), "=&r"(pk1), "=&r"(s)
         : "r"(key.lane), "r"(key.mask));
 }
 
-__device__ __forceinline__ void group2(Win& r, LutKey key, uint32_t& pk0, uint32_t& s)
+__device__ __forceinline__ void group2(Cur& c, LutKey key, uint32_t& pk0, uint32_t& s)
 {
     __attribute__((unused)) uint32_t unused;   // operand slot of the second pair, which a group of two does not have
     asm volatile(
         "{\n\t"
         ".reg .pred p;\n\t"
-        ".reg .b32 t, w, a, e0, e1;\n\t"
-        ".reg .f32 f;\n\t" ENTRO_REFILL ENTRO_LOOKUP("e0", "%0")
-        "shf.l.wrap.b32 w, %1, %0, e0;\n\t" ENTRO_LOOKUP("e1", "w")
+        ".reg .b32 t, w, a, h, e0, e1;\n\t"
+        ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("e0", "h")
+        "shf.l.wrap.b32 w, 0, h, e0;\n\t" ENTRO_LOOKUP("e1", "w")
         "add.u32 %6, e0, e1;\n\t"
         "prmt.b32 %4, e0, e1, 0x7632;\n\t"
-        "mov.b32 %5, 0;\n\t" ENTRO_ADVANCE "}"
-        : "+r"(r.hi), "+r"(r.lo), "+r"(r.k), "+r"(r.next), "=&r"(pk0), "=&r"(unused), "=&r"(s)
+        "mov.b32 %5, 0;\n\t" ENTRO_MOVE_ON "}"
+        : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk0), "=&r"(unused), "=&r"(s)
         : "r"(key.lane), "r"(key.mask));
 }
 #undef ENTRO_LOOKUP
-#undef ENTRO_REFILL
-#undef ENTRO_ADVANCE
+#undef ENTRO_OPEN
+#undef ENTRO_MOVE_ON
 
 // The next symbol by itself, any code length: refill, one exponent-indexed lookup (this
 // lane's copy for 8-bit alphabets, the single copy behind the eight-symbol tables for 4-bit
@@ -426,38 +450,41 @@ __device__ __forceinline__ uint32_t next_symbol(Win& r, uint32_t* status, LutKey
     return e;
 }
 
-// Rebuild the window as it was before a group that did not stand, from what the group
-// left: k grew by exactly s, next did not move after the refill.
-__device__ __forceinline__ void rewind_group(Win& r, uint32_t s)
+// Where the reader stood before a group that did not stand: the position moved on by
+// exactly s (modulo 2^16), and the words moved on by one iff bit 5 of the position flipped.
+__device__ __forceinline__ uint32_t rewind_group(const Cur& c, uint32_t s)
 {
-    const uint32_t valid = (uint32_t)win_valid_bits(r.k - s);   // 33 .. 64 bits were valid when the group began
-    const uint32_t bit_addr = r.next * 8u - valid;              // where they begin, in bits of the shared window
-    win_init<true>(r, (bit_addr >> 5) << 2, bit_addr & 31u);
+    const uint32_t before = c.pos - s;
+    const uint32_t crossed = ((before ^ c.pos) >> 5) & 1u;
+    return (c.next - 8u - 4u * crossed) * 8u + (before & 31u);
 }
 
 // Repair of a group of two symbols that did not stand (kept inline: a call here would park
 // the caller's registers in local memory, which misses the small L1 left beside 228 KB of
-// shared memory): the symbols one by one, any code length.
+// shared memory): the symbols one by one, any code length, with the general reader.
 template <int K>
-__device__ __forceinline__ void repair_pair(Win& r, uint32_t* status, LutKey key, uint32_t s, uint32_t& pk)
+__device__ __forceinline__ void repair_pair(Cur& c, uint32_t* status, LutKey key, uint32_t s, uint32_t& pk)
 {
-    rewind_group(r, s);
+    const uint32_t at = rewind_group(c, s);
+    Win r;
+    win_init<true>(r, (at >> 5) << 2, at & 31u);
     const uint32_t e0 = next_symbol<K, false>(r, status, key);
     const uint32_t e1 = next_symbol<K, false>(r, status, key);
     pk = __byte_perm(e0, e1, 0x7632);
+    cur_init(c, r.next * 8u - (uint32_t)win_valid_bits(r.k));
 }
 
 // Repair of a group of four: almost always it merely used 32 bits or more, so two groups of
 // two stand; each of those falls back to repair_pair.
 template <int K>
-__device__ __forceinline__ void repair_quad(Win& r, uint32_t* status, LutKey key, uint32_t s, uint32_t& pk0, uint32_t& pk1)
+__device__ __forceinline__ void repair_quad(Cur& c, uint32_t* status, LutKey key, uint32_t s, uint32_t& pk0, uint32_t& pk1)
 {
-    rewind_group(r, s);
+    cur_init(c, rewind_group(c, s));
     uint32_t s2;
-    group2(r, key, pk0, s2);
-    if (__builtin_expect((s2 & 0xffe0u) != 0u, 0)) repair_pair<K>(r, status, key, s2, pk0);
-    group2(r, key, pk1, s2);
-    if (__builtin_expect((s2 & 0xffe0u) != 0u, 0)) repair_pair<K>(r, status, key, s2, pk1);
+    group2(c, key, pk0, s2);
+    if (__builtin_expect((s2 & 0xffe0u) != 0u, 0)) repair_pair<K>(c, status, key, s2, pk0);
+    group2(c, key, pk1, s2);
+    if (__builtin_expect((s2 & 0xffe0u) != 0u, 0)) repair_pair<K>(c, status, key, s2, pk1);
 }
 
 // Eight symbols of a 4-bit alphabet whose codes do not fit the table's window.
@@ -793,8 +820,10 @@ struct EmitDot {
 
 // 8-bit alphabets: G lookups per window refill (group4 / group2 above).
 template <int K, int G, class Emit>
-__device__ __forceinline__ void rows_single(Win& r, uint32_t* status, LutKey key, Emit& emit, uint32_t sub)
+__device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status, LutKey key, Emit& emit, uint32_t sub)
 {
+    Cur r;
+    cur_init(r, start);
     for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
         uint32_t pk[4];
         if (G == 4) {
@@ -814,12 +843,15 @@ __device__ __forceinline__ void rows_single(Win& r, uint32_t* status, LutKey key
         }
         emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
     }
+    return cur_bit_addr(r);
 }
 
 // 4-bit alphabets: eight symbols per lookup.
 template <int K, class Emit>
-__device__ __forceinline__ void rows_oct(Win& r, uint32_t* status, Emit& emit, uint32_t sub)
+__device__ __forceinline__ uint32_t rows_oct(uint32_t start, uint32_t* status, Emit& emit, uint32_t sub)
 {
+    Win r;
+    win_init<false>(r, (start >> 5) << 2, start & 31u);
     for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
         win_refill<false>(r);
         const uint32_t idx = r.hi >> (32 - K);
@@ -829,6 +861,7 @@ __device__ __forceinline__ void rows_oct(Win& r, uint32_t* status, Emit& emit, u
         else win_skip(r, n);
         emit(v);
     }
+    return r.next * 8u - (uint32_t)win_valid_bits(r.k);
 }
 
 // What decode_start leaves for decode_finish: where this lane begins and must end.
@@ -900,10 +933,8 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         return;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    Win w;
     const bool oct = aux_ptr<K>()->oct != 0;
-    if (oct) win_init<false>(w, (L.start >> 5) << 2, L.start & 31u);
-    else win_init<true>(w, (L.start >> 5) << 2, L.start & 31u);
+    uint32_t stood;            // where the lane stands after its sub-block
     if (kGemv) {
         // the chunk starts gs0 steps of 256 weights into the matrix; a row is rs steps long
         const uint32_t rs = G->cols >> 8;
@@ -917,33 +948,33 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         em.xaddr = em.xlane + k0 * 512u;
         em.acc = 0.f;
         em.yrow = G->y32 + row0;
-        if (oct) rows_oct<K>(w, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
-        else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        if (oct) stood = rows_oct<K>(L.start, status, em, sub);
+        else if (aux_ptr<K>()->group == 4u) stood = rows_single<K, 4>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        else stood = rows_single<K, 2>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
         em.finish();
     } else if (kSink == kSinkBytes) {
         EmitBytes em;
         em.dst = reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(T.out) + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
-        if (oct) rows_oct<K>(w, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
-        else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        if (oct) stood = rows_oct<K>(L.start, status, em, sub);
+        else if (aux_ptr<K>()->group == 4u) stood = rows_single<K, 4>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        else stood = rows_single<K, 2>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
     } else if (kSink == kSinkNibbles) {
         EmitNibbles em;
         em.dst = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(T.out) + (((uint64_t)r.c * T.chunk_symbols) >> 1) +
                                              lane * 4u);
-        if (oct) rows_oct<K>(w, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
-        else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        if (oct) stood = rows_oct<K>(L.start, status, em, sub);
+        else if (aux_ptr<K>()->group == 4u) stood = rows_single<K, 4>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        else stood = rows_single<K, 2>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
     } else {
         EmitStore em;
         em.dst = reinterpret_cast<uint4*>(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
-        if (oct) rows_oct<K>(w, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) rows_single<K, 4>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
-        else rows_single<K, 2>(w, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        if (oct) stood = rows_oct<K>(L.start, status, em, sub);
+        else if (aux_ptr<K>()->group == 4u) stood = rows_single<K, 4>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        else stood = rows_single<K, 2>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
         em.finish();
     }
     // the lane must stand exactly at the end of its sub-block
-    if (w.next * 8u - (uint32_t)win_valid_bits(w.k) != L.end) atomicOr(status, kStatCorrupt);
+    if (stood != L.end) atomicOr(status, kStatCorrupt);
     __syncwarp();   // all lanes are done with these bytes before the ring reuses them
 }
 
