@@ -121,8 +121,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
         aux.max_len = max_len;
         // eight symbols per lookup pay off while eight codes usually fit the table's window
         aux.oct = (T.nsym <= 16 && mean_len * 8.f <= (float)lut_bits - 1.5f) ? 1u : 0u;
-        // four lookups per window refill while their lengths almost always sum to < 32 bits
-        aux.group = mean_len <= 6.0f ? 4u : 2u;
+        aux.group = 2u;            // decided below, from the chance that a group needs 32 bits or more
         aux.expm = (uint32_t)kExpBitsMin;
         for (int j = 0; j < 16; ++j) need_mass[j] = 0.f;
     }
@@ -138,6 +137,42 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
         if (r > l) r = l;
         const uint32_t need = l > r + 1u ? l - r - 1u : 0u;
         atomicAdd(&need_mass[need < 15u ? need : 15u], exp2f(-(float)l));
+    }
+    __syncthreads();
+    // Lookups per group: a group stands only if its codes use fewer than 32 bits together.
+    // With 2^-length for the chance of a symbol, fail[g] = chance that g lengths sum to 32 or
+    // more, by repeated convolution of the length distribution (bin 32 collects the rest).
+    {
+        __shared__ float by_len[33], dist[2][33], fail[5];
+        if (tid <= 32) {
+            by_len[tid] = tid ? (float)count[tid] * exp2f(-(float)tid) : 0.f;
+            dist[0][tid] = tid == 0 ? 1.f : 0.f;
+        }
+        __syncthreads();
+        for (int g = 1; g <= 4; ++g) {
+            const float* in = dist[(g - 1) & 1];
+            float* o = dist[g & 1];
+            if (tid < 32) {
+                float v = 0.f;
+                for (int j = 0; j <= tid; ++j) v += in[j] * by_len[tid - j];
+                o[tid] = v;
+            }
+            __syncthreads();
+            if (tid == 0) {
+                float in_range = 0.f;
+                for (int j = 0; j < 32; ++j) in_range += o[j];
+                fail[g] = fmaxf(1.f - in_range, 0.f);
+                o[32] = 0.f;
+            }
+            __syncthreads();
+        }
+        if (tid == 0) {
+            const float mean_len = (float)T.offsets[T.n_chunks] / (float)T.n;   // guards against a codebook that does not fit the data
+            // a failing lane stalls its warp: the limits keep the warp's failures to a few per cent
+            if (fail[4] < 3e-4f && mean_len <= 4.0f) aux.group = 8u;        // two groups of four under one check
+            else if (fail[4] < 3e-3f && mean_len <= 5.2f) aux.group = 4u;
+            else if (fail[3] < 2.4e-3f && mean_len <= 8.5f) aux.group = 3u;
+        }
     }
     __syncthreads();
     if (tid == 0 && !aux.oct) {
@@ -426,6 +461,40 @@ __device__ __forceinline__ void group2(Cur& c, LutKey key, uint32_t& pk0, uint32
         : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk0), "=&r"(unused), "=&r"(s)
         : "r"(key.lane), "r"(key.mask));
 }
+// Three lookups, for the streams whose groups of four would too often need 32 bits or more.
+// Eight symbols go out as 3 + 3 + 2, so the pairs of values straddle the groups: with kTail
+// false, first = the pair (v0, v1) and second = the third entry as it is; with kTail true,
+// first = the first entry as it is and second = the pair (v1, v2).
+template <bool kTail>
+__device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint32_t& second, uint32_t& s)
+{
+    if (!kTail)
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            ".reg .b32 t, w, a, h, e0, e1;\n\t"
+            ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("e0", "h")
+            "shf.l.wrap.b32 w, 0, h, e0;\n\t" ENTRO_LOOKUP("e1", "w")
+            "add.u32 %6, e0, e1;\n\t"
+            "shf.l.wrap.b32 w, 0, h, %6;\n\t" ENTRO_LOOKUP("%5", "w")
+            "add.u32 %6, %6, %5;\n\t"
+            "prmt.b32 %4, e0, e1, 0x7632;\n\t" ENTRO_MOVE_ON "}"
+            : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s)
+            : "r"(key.lane), "r"(key.mask));
+    else
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            ".reg .b32 t, w, a, h, e1, e2;\n\t"
+            ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("%4", "h")
+            "shf.l.wrap.b32 w, 0, h, %4;\n\t" ENTRO_LOOKUP("e1", "w")
+            "add.u32 %6, %4, e1;\n\t"
+            "shf.l.wrap.b32 w, 0, h, %6;\n\t" ENTRO_LOOKUP("e2", "w")
+            "add.u32 %6, %6, e2;\n\t"
+            "prmt.b32 %5, e1, e2, 0x7632;\n\t" ENTRO_MOVE_ON "}"
+            : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s)
+            : "r"(key.lane), "r"(key.mask));
+}
 #undef ENTRO_LOOKUP
 #undef ENTRO_OPEN
 #undef ENTRO_MOVE_ON
@@ -471,6 +540,22 @@ __device__ __forceinline__ void repair_pair(Cur& c, uint32_t* status, LutKey key
     const uint32_t e0 = next_symbol<K, false>(r, status, key);
     const uint32_t e1 = next_symbol<K, false>(r, status, key);
     pk = __byte_perm(e0, e1, 0x7632);
+    cur_init(c, r.next * 8u - (uint32_t)win_valid_bits(r.k));
+}
+
+// The same for a group of three (rare by the choice of the group size).
+template <int K, bool kTail>
+__device__ __forceinline__ void repair_triple(Cur& c, uint32_t* status, LutKey key, uint32_t s, uint32_t& first,
+                                              uint32_t& second)
+{
+    const uint32_t at = rewind_group(c, s);
+    Win r;
+    win_init<true>(r, (at >> 5) << 2, at & 31u);
+    const uint32_t e0 = next_symbol<K, false>(r, status, key);
+    const uint32_t e1 = next_symbol<K, false>(r, status, key);
+    const uint32_t e2 = next_symbol<K, false>(r, status, key);
+    first = kTail ? e0 : __byte_perm(e0, e1, 0x7632);
+    second = kTail ? __byte_perm(e1, e2, 0x7632) : e2;
     cur_init(c, r.next * 8u - (uint32_t)win_valid_bits(r.k));
 }
 
@@ -818,7 +903,9 @@ struct EmitDot {
     }
 };
 
-// 8-bit alphabets: G lookups per window refill (group4 / group2 above).
+// 8-bit alphabets, eight symbols per turn.  G = 2, 3 (as 3 + 3 + 2), 4: groups of that many
+// lookups, each checked.  G = 8: two groups of four under one check, for streams whose groups
+// of four almost never fail; if either failed, both are done again one by one.
 template <int K, int G, class Emit>
 __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status, LutKey key, Emit& emit, uint32_t sub)
 {
@@ -826,13 +913,37 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
     cur_init(r, start);
     for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
         uint32_t pk[4];
-        if (G == 4) {
-#pragma unroll
-            for (int g = 0; g < 2; ++g) {
-                uint32_t s;
-                group4(r, key, pk[2 * g], pk[2 * g + 1], s);
-                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_quad<K>(r, status, key, s, pk[2 * g], pk[2 * g + 1]);
+        bool again = G == 4;
+        if (G == 8) {
+            uint32_t s0, s1;
+            group4(r, key, pk[0], pk[1], s0);
+            group4(r, key, pk[2], pk[3], s1);
+            if (__builtin_expect(((s0 | s1) & 0xffe0u) != 0u, 0)) {
+                // back over both: the position moved by s0 + s1, the words by one per flip of bit 5
+                const uint32_t p1 = r.pos - s1, p0 = p1 - s0;
+                const uint32_t steps = (((p0 ^ p1) >> 5) & 1u) + (((p1 ^ r.pos) >> 5) & 1u);
+                cur_init(r, (r.next - 8u - 4u * steps) * 8u + (p0 & 31u));
+                again = true;
             }
+        }
+        if (G == 4 || G == 8) {
+            if (again) {
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    uint32_t s;
+                    group4(r, key, pk[2 * g], pk[2 * g + 1], s);
+                    if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_quad<K>(r, status, key, s, pk[2 * g], pk[2 * g + 1]);
+                }
+            }
+        } else if (G == 3) {
+            uint32_t s, a2, b0;
+            group3<false>(r, key, pk[0], a2, s);
+            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_triple<K, false>(r, status, key, s, pk[0], a2);
+            group3<true>(r, key, b0, pk[2], s);
+            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_triple<K, true>(r, status, key, s, b0, pk[2]);
+            pk[1] = __byte_perm(a2, b0, 0x7632);
+            group2(r, key, pk[3], s);
+            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_pair<K>(r, status, key, s, pk[3]);
         } else {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
@@ -862,6 +973,22 @@ __device__ __forceinline__ uint32_t rows_oct(uint32_t start, uint32_t* status, E
         emit(v);
     }
     return r.next * 8u - (uint32_t)win_valid_bits(r.k);
+}
+
+// The whole sub-block of a lane in the mode build_tables_kernel chose for the tensor;
+// returns where the lane stands afterwards.
+template <int K, class Emit>
+__device__ __forceinline__ uint32_t rows_any(const DecodeAux* aux, uint32_t start, uint32_t* status, Emit& emit, uint32_t sub,
+                                             uint32_t lane)
+{
+    if (aux->oct) return rows_oct<K>(start, status, emit, sub);
+    const LutKey key = lut_key(aux->expm, lane);
+    switch (aux->group) {
+        case 8u: return rows_single<K, 8>(start, status, key, emit, sub);
+        case 4u: return rows_single<K, 4>(start, status, key, emit, sub);
+        case 3u: return rows_single<K, 3>(start, status, key, emit, sub);
+        default: return rows_single<K, 2>(start, status, key, emit, sub);
+    }
 }
 
 // What decode_start leaves for decode_finish: where this lane begins and must end.
@@ -933,7 +1060,6 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         return;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    const bool oct = aux_ptr<K>()->oct != 0;
     uint32_t stood;            // where the lane stands after its sub-block
     if (kGemv) {
         // the chunk starts gs0 steps of 256 weights into the matrix; a row is rs steps long
@@ -948,29 +1074,21 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         em.xaddr = em.xlane + k0 * 512u;
         em.acc = 0.f;
         em.yrow = G->y32 + row0;
-        if (oct) stood = rows_oct<K>(L.start, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) stood = rows_single<K, 4>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
-        else stood = rows_single<K, 2>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
         em.finish();
     } else if (kSink == kSinkBytes) {
         EmitBytes em;
         em.dst = reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(T.out) + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
-        if (oct) stood = rows_oct<K>(L.start, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) stood = rows_single<K, 4>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
-        else stood = rows_single<K, 2>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
     } else if (kSink == kSinkNibbles) {
         EmitNibbles em;
         em.dst = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(T.out) + (((uint64_t)r.c * T.chunk_symbols) >> 1) +
                                              lane * 4u);
-        if (oct) stood = rows_oct<K>(L.start, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) stood = rows_single<K, 4>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
-        else stood = rows_single<K, 2>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
     } else {
         EmitStore em;
         em.dst = reinterpret_cast<uint4*>(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
-        if (oct) stood = rows_oct<K>(L.start, status, em, sub);
-        else if (aux_ptr<K>()->group == 4u) stood = rows_single<K, 4>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
-        else stood = rows_single<K, 2>(L.start, status, lut_key(aux_ptr<K>()->expm, lane), em, sub);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
         em.finish();
     }
     // the lane must stand exactly at the end of its sub-block
