@@ -114,7 +114,7 @@ def test_decode_of_oracle_streams_small_and_ragged(bits, chunk):
 @pytest.mark.parametrize("bits,chunk", [(8, 4096), (4, 8192)])
 def test_decode_flat_histograms(bits, chunk):
     """Inputs without heavy tails spread the symbols over many levels: the 8-bit path then uses
-    the wider exponent-indexed table and groups of two, the 4-bit path one symbol per lookup.
+    the wider exponent-indexed table and groups of three, the 4-bit path one symbol per lookup.
     A uniform histogram (every code the same length) is resolved by no table cell at all and
     runs entirely on the symbol-by-symbol repair."""
     for n in (chunk - 1, 9 * chunk, 33 * chunk + 77):
@@ -130,6 +130,32 @@ def test_decode_flat_histograms(bits, chunk):
                                  E.Codebook.from_lengths(ln.tolist(), cd.tolist()), 0.03125, nsym // 2)
     torch.cuda.synchronize()
     assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.dequant(q, 0.03125, nsym // 2))
+    assert_status_ok()
+
+
+@pytest.mark.parametrize("sigma_levels,foreign", [(2.0, False), (6.0, False), (14.0, False), (40.0, False), (40.0, True)])
+def test_decode_every_group_size(sigma_levels, foreign):
+    """The decoder picks the number of lookups per group from the code lengths and the bits
+    per symbol: narrow histograms take two fours under one check, wider ones four, three,
+    and a codebook that does not fit its data (here: built for a narrow histogram, used on a
+    wide one, about 14 bits per symbol) two.  Symbols are drawn directly, as rounded
+    Gaussians of the given width in quantisation levels; the values check the symbols."""
+    chunk, n = 4096, 21 * 4096 + 333
+    rng = np.random.default_rng(int(sigma_levels * 10) + foreign)
+    q = np.clip(np.rint(rng.normal(128.0, sigma_levels, n)), 0, 255).astype(np.uint8)
+    counts = np.bincount(q, minlength=256)
+    if foreign:
+        narrow = np.clip(np.rint(rng.normal(128.0, 3.0, n)), 0, 255).astype(np.uint8)
+        counts = np.bincount(narrow, minlength=256) + 1          # every symbol keeps a code
+    ln = oracle.huffman_lengths(counts.tolist())
+    cd = oracle.canonical_codes(ln)
+    enc = oracle.encode(q, ln, cd, chunk)
+    if foreign:
+        assert int(enc.offsets[-1]) / n > 8.5
+    out = E.entro_decode_dequant(to_dev_stream(enc.stream), to_dev_index(enc), n, chunk,
+                                 E.Codebook.from_lengths(ln.tolist(), cd.tolist()), 0.0078125, 128)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.dequant(q, 0.0078125, 128))
     assert_status_ok()
 
 
