@@ -397,9 +397,9 @@ __device__ __forceinline__ void cur_init(Cur& c, uint32_t bit_addr)
 __device__ __forceinline__ uint32_t cur_bit_addr(const Cur& c) { return (c.next - 8u) * 8u + (c.pos & 31u); }
 
 // One group of lookups, hand-scheduled.  The group sees the 32 bits that start at the
-// reader's position (one funnel shift of the two words) and nothing behind them: lookup i
-// reads them shifted left by the lengths of the symbols before it (a funnel shift uses the
-// low five bits of the running sum of the entries), zeros moving in from the right.  Those
+// reader's position (one funnel shift of the two words) and nothing behind them: a lookup
+// reads them shifted left by the lengths found before it (a funnel shift uses the low five
+// bits of its count), zeros moving in from the right.  Those
 // zeros cannot mislead a lookup whose code ends inside the 32 bits: a cell is resolved only
 // if every window that maps to it begins with the same code, whatever follows.  s is the sum
 // of the G entries: the group stands iff (s & 0xffe0) == 0, that is, every cell was resolved
@@ -475,8 +475,8 @@ __device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint
             ".reg .b32 t, w, a, h, e0, e1;\n\t"
             ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("e0", "h")
             "shf.l.wrap.b32 w, 0, h, e0;\n\t" ENTRO_LOOKUP("e1", "w")
+            "shf.l.wrap.b32 w, 0, w, e1;\n\t" ENTRO_LOOKUP("%5", "w")
             "add.u32 %6, e0, e1;\n\t"
-            "shf.l.wrap.b32 w, 0, h, %6;\n\t" ENTRO_LOOKUP("%5", "w")
             "add.u32 %6, %6, %5;\n\t"
             "prmt.b32 %4, e0, e1, 0x7632;\n\t" ENTRO_MOVE_ON "}"
             : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s)
@@ -488,8 +488,8 @@ __device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint
             ".reg .b32 t, w, a, h, e1, e2;\n\t"
             ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("%4", "h")
             "shf.l.wrap.b32 w, 0, h, %4;\n\t" ENTRO_LOOKUP("e1", "w")
+            "shf.l.wrap.b32 w, 0, w, e1;\n\t" ENTRO_LOOKUP("e2", "w")
             "add.u32 %6, %4, e1;\n\t"
-            "shf.l.wrap.b32 w, 0, h, %6;\n\t" ENTRO_LOOKUP("e2", "w")
             "add.u32 %6, %6, e2;\n\t"
             "prmt.b32 %5, e1, e2, 0x7632;\n\t" ENTRO_MOVE_ON "}"
             : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s)
