@@ -50,6 +50,7 @@ extern "C" {
 #define ENTRO_STREAM_SLACK_WORDS 8
 #define ENTRO_MAX_CHUNK_SYMBOLS 16384
 #define ENTRO_STATIC_MAX_TENSORS 8
+#define ENTRO_GEMV_MAX_BATCH 8
 
 typedef enum {
     ENTRO_OK = 0,
@@ -233,23 +234,28 @@ entro_status entro_decode_dequant_batched_host(const entro_tensor_desc *descs_ho
  * pointers inside are device pointers. */
 typedef struct {
     uint32_t rows, cols;        /* W is [rows, cols] row-major, rows * cols = the tensor's n */
-    const void *x_fp16_dev;     /* cols fp16 values, 16-byte aligned */
-    void *y_fp16_dev;           /* rows fp16 results */
+    const void *x_fp16_dev;     /* [batch][cols] fp16 values, token after token, 16-byte aligned */
+    void *y_fp16_dev;           /* [batch][rows] fp16 results */
+    uint32_t batch;             /* tokens, 1 .. ENTRO_GEMV_MAX_BATCH */
+    uint32_t reserved;          /* 0 */
 } entro_gemv_io;
 
 /*
- * Decode + dequantise + batch-1 matrix-vector product in one pass, without ever writing the
- * fp16 weights: y[o] = fp16_rne( sum_i w_hat[o, i] * x[i] ), w_hat = fp16(s * (q - z)) as in
- * entro_decode_dequant, products and sums in fp32.  This is the token-generation use of
- * compressed weights: the paper attributes its generation speed-up to "reduced memory
- * transfers during the memory-bandwidth-limited decoding phase" (Section 4, Table 3); here
- * only the compressed stream crosses HBM.  descs_host[i].out_fp16_dev is not used and may be
- * NULL.  All ntensors products are independent and run in one launch.  The order of the
- * fp32 additions is not fixed (rows that span chunks are summed with atomics), so results
- * can differ from run to run in the last bits before the final rounding.
- * Limits: cols a multiple of 256 and at most 16384, chunk_symbols a multiple of 256
- * (ENTRO_ERR_UNSUPPORTED otherwise).  Asynchronous; malformed input is reported through
- * entro_last_device_status as for the decode calls.
+ * Decode + dequantise + matrix-vector product in one pass, for one token or a small batch,
+ * without ever writing the fp16 weights: y[b][o] = fp16_rne( sum_i w_hat[o, i] * x[b][i] ),
+ * w_hat = fp16(s * (q - z)) as in entro_decode_dequant, products and sums in fp32.  This is
+ * the token-generation use of compressed weights: the paper puts its generation speed-up
+ * down to the smaller amount of weight data that is moved while tokens are generated, a
+ * phase bound by memory bandwidth (Section 4, Table 3); here only the compressed stream
+ * crosses HBM, once for all tokens of the batch.  descs_host[i].out_fp16_dev is not used and may be NULL.  All ntensors
+ * products are independent and run in one launch.  The order of the fp32 additions is not
+ * fixed (rows that span chunks are summed with atomics), so results can differ from run to
+ * run in the last bits before the final rounding.
+ * Limits: cols a multiple of 256, batch * cols at most 32768 (x of all tokens is staged in
+ * shared memory), chunk_symbols a multiple of 256 (ENTRO_ERR_UNSUPPORTED otherwise); batch
+ * outside 1 .. ENTRO_GEMV_MAX_BATCH or reserved != 0 is ENTRO_ERR_INVALID_ARG.
+ * Asynchronous; malformed input is reported through entro_last_device_status as for the
+ * decode calls.
  */
 entro_status entro_decode_dequant_gemv(const entro_tensor_desc *descs_host, const entro_gemv_io *io_host,
                                        int ntensors, void *cuda_stream);

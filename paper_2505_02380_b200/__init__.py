@@ -25,6 +25,7 @@ MODE_AUTO, MODE_UNSIGNED, MODE_ASYMMETRIC = 0, 1, 2
 OK, ERR_INVALID_ARG, ERR_BUFFER_TOO_SMALL, ERR_NONFINITE, ERR_CODE_TOO_LONG, ERR_CORRUPT_STREAM, ERR_CUDA, \
     ERR_UNSUPPORTED, ERR_TOO_MANY_TENSORS = range(9)
 STATIC_MAX_TENSORS = 8
+GEMV_MAX_BATCH = 8
 DEFAULT_DECODE_CONFIG = (12, 32, 1, 1024)   # lut_bits, warps_per_cta, ctas_per_sm, chunks_per_item
 
 
@@ -69,7 +70,8 @@ class TensorDesc(C.Structure):
 
 
 class GemvIO(C.Structure):
-    _fields_ = [("rows", C.c_uint32), ("cols", C.c_uint32), ("x_fp16_dev", C.c_void_p), ("y_fp16_dev", C.c_void_p)]
+    _fields_ = [("rows", C.c_uint32), ("cols", C.c_uint32), ("x_fp16_dev", C.c_void_p), ("y_fp16_dev", C.c_void_p),
+                ("batch", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class HostIO(C.Structure):
@@ -309,28 +311,36 @@ def make_desc_no_out(stream_words: torch.Tensor, index: torch.Tensor, n: int, ch
     return d
 
 
+def _gemv_batch(x: torch.Tensor) -> int:
+    return int(x.shape[0]) if x.dim() == 2 else 1
+
+
 def make_gemv_io(xs: Sequence[torch.Tensor], ys: Sequence[torch.Tensor], shapes: Sequence):
     """The ctypes array entro_decode_dequant_gemv takes, for callers that repeat a call and want
-    to marshal once.  shapes[i] = (rows, cols) of W_i; xs[i] has cols, ys[i] rows fp16 values."""
+    to marshal once.  shapes[i] = (rows, cols) of W_i; xs[i] holds cols fp16 values (one token)
+    or [batch, cols] (a small batch), ys[i] rows or [batch, rows]."""
     n = len(xs)
     io = (GemvIO * n)()
     for i in range(n):
-        io[i] = GemvIO(int(shapes[i][0]), int(shapes[i][1]), _dev(xs[i], torch.float16), _dev(ys[i], torch.float16))
+        io[i] = GemvIO(int(shapes[i][0]), int(shapes[i][1]), _dev(xs[i], torch.float16), _dev(ys[i], torch.float16),
+                       _gemv_batch(xs[i]), 0)
     return io
 
 
 def entro_decode_dequant_gemv(descs, xs: Optional[Sequence[torch.Tensor]] = None, shapes: Optional[Sequence] = None,
                               ys: Optional[List[torch.Tensor]] = None, stream: Optional[torch.cuda.Stream] = None,
                               io=None):
-    """descs[i]: compressed W_i of shape shapes[i] = (rows, cols); xs[i]: fp16 vector of cols values.
-    -> fp16 vectors y_i = W_i x_i (the ys given, or new ones).  Pass io = make_gemv_io(...) instead of
-    xs / shapes / ys to skip the marshalling.  Asynchronous."""
+    """descs[i]: compressed W_i of shape shapes[i] = (rows, cols); xs[i]: fp16 vector of cols values,
+    or [batch, cols] for a batch of up to GEMV_MAX_BATCH tokens.  -> fp16 y_i = W_i x_i, rows values or
+    [batch, rows] (the ys given, or new ones).  Pass io = make_gemv_io(...) instead of xs / shapes / ys
+    to skip the marshalling.  Asynchronous."""
     if isinstance(descs, list):
         descs = desc_array(descs)
     n = len(descs)
     if io is None:
         if ys is None:
-            ys = [torch.empty(shapes[i][0], dtype=torch.float16, device=xs[i].device) for i in range(n)]
+            ys = [torch.empty((xs[i].shape[0], shapes[i][0]) if xs[i].dim() == 2 else shapes[i][0],
+                              dtype=torch.float16, device=xs[i].device) for i in range(n)]
         io = make_gemv_io(xs, ys, shapes)
     _check(lib().entro_decode_dequant_gemv(descs, io, n, _stream(stream)), "entro_decode_dequant_gemv")
     return ys

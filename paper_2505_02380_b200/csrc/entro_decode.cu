@@ -634,9 +634,12 @@ template <int K>
 constexpr uint32_t kGemvX = kGemvDesc<K> + (uint32_t)sizeof(GemvTensor);
 template <int K>
 __device__ __forceinline__ GemvTensor* gemv_ptr() { return reinterpret_cast<GemvTensor*>(smem + kGemvDesc<K>); }
-// Offset of the first ring.
-template <int K, bool kGemv>
-constexpr uint32_t kRingsAt = ((kGemv ? kGemvX<K> + 2u * kGemvMaxCols : kGemvDesc<K>) + 127u) & ~127u;
+// Offset of the first ring: behind the tensor, or behind x_bytes of staged x (a multiple of 128).
+template <int K>
+constexpr uint32_t rings_offset(bool gemv, uint32_t x_bytes)
+{
+    return ((gemv ? kGemvX<K> + x_bytes : kGemvDesc<K>) + 127u) & ~127u;
+}
 
 // What a warp carries from chunk to chunk (kept small: it lives in registers across the
 // decode loop).
@@ -759,7 +762,9 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32
 
 // Any symbol count per lane, words fetched straight from global memory, one value at a
 // time: the ragged last chunk of a tensor, odd chunk sizes, chunks larger than the ring.
-// With G set the values are not stored but multiplied into the matrix-vector product.
+// With G set (kB > 0 accumulators) the values are not stored but multiplied into the
+// matrix-vector products of the batch's tokens.
+template <int kB>
 __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t* status, const DevTensor& T,
                                                      const GemvTensor* G, int sink, uint32_t c, uint32_t excl,
                                                      uint32_t my_bits, uint32_t lane)
@@ -782,7 +787,9 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
     // this lane's symbols: groups lane, lane + 32, ... of 8 consecutive symbols
     for (uint32_t g = lane; g * 8u < m; g += kSubBlocks) {
         const uint32_t end = min(g * 8u + 8u, m);
-        float acc = 0.f;
+        float acc[kB > 0 ? kB : 1];
+#pragma unroll
+        for (int b = 0; b < (kB > 0 ? kB : 1); ++b) acc[b] = 0.f;
         uint32_t low = 0;                       // the even symbol of a nibble pair
         for (uint32_t i = g * 8u; i < end; ++i) {
             gwin_refill(r);
@@ -793,10 +800,13 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
             r.hi = __funnelshift_lc(r.lo, r.hi, n);
             r.lo = __funnelshift_lc(0u, r.lo, n);
             r.nb -= (int)n;
-            if (G) {
+            if (kB > 0) {
                 const uint32_t col = (uint32_t)((chunk_first + i) % G->cols);
-                acc = fmaf(__half2float(__ushort_as_half((uint16_t)(e >> 16))),
-                           __half2float(__ushort_as_half(__ldg(G->x + col))), acc);
+                const float v = __half2float(__ushort_as_half((uint16_t)(e >> 16)));
+#pragma unroll
+                for (int b = 0; b < kB; ++b)
+                    if ((uint32_t)b < G->batch)
+                        acc[b] = fmaf(v, __half2float(__ushort_as_half(__ldg(G->x + (uint64_t)b * G->cols + col))), acc[b]);
             } else if (sink == kSinkBytes) {
                 reinterpret_cast<uint8_t*>(T.out)[chunk_first + i] = (uint8_t)(e >> 16);
             } else if (sink == kSinkNibbles) {
@@ -809,7 +819,12 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
             }
         }
         // a group of 8 lies inside one row (cols is a multiple of 8)
-        if (G) atomicAdd(G->y32 + (chunk_first + g * 8u) / G->cols, acc);
+        if (kB > 0) {
+            const uint32_t row = (uint32_t)((chunk_first + g * 8u) / G->cols);
+#pragma unroll
+            for (int b = 0; b < kB; ++b)
+                if ((uint32_t)b < G->batch) atomicAdd(G->y32 + (uint64_t)b * G->rows + row, acc[b]);
+        }
     }
     const uint64_t used = ((uint64_t)r.next << 5) - (uint64_t)r.nb - bit;
     if (used != my_bits) atomicOr(status, kStatCorrupt);
@@ -861,38 +876,52 @@ struct EmitNibbles {
 
 // Fused matrix-vector product: the 8 values are weights of one row of W (stored [rows, cols],
 // cols a multiple of 256, so the 32 lanes of a step stay inside one row) and meet the 8
-// matching entries of x, staged in shared memory as fp16; products and sums in fp32.  When
-// the row ends the warp adds its lanes up and adds the result to the row's fp32 accumulator.
+// matching entries of x of every token, staged in shared memory as fp16 token after token
+// (tokens beyond the batch are zeros); products and sums in fp32, one accumulator per token.
+// When the row ends the warp adds its lanes up and adds the results to the row's fp32
+// accumulators.
+template <int B>
 struct EmitDot {
-    uint32_t xaddr;       // shared-window address of x[col .. col + 8) for this lane's next group
+    uint32_t xaddr;       // shared-window address of x[0][col .. col + 8) for this lane's next group
     uint32_t xlane;       // the same at the start of a row
+    uint32_t xstride;     // bytes from one token's x to the next
     uint32_t left;        // steps left in the current row
     uint32_t rs;          // steps per row (cols / 256)
-    float acc;
-    float* yrow;          // fp32 accumulator of the current row
+    float acc[B];
+    float* yrow;          // fp32 accumulator of the current row, first token
+    uint32_t rows, batch;
     uint32_t lane;
 
     __device__ __forceinline__ void flush()
     {
-        float v = acc;
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
-        if (lane == 0) atomicAdd(yrow, v);
-        acc = 0.f;
+        for (int b = 0; b < B; ++b) {
+            float v = acc[b];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+            if (lane == 0 && (uint32_t)b < batch) atomicAdd(yrow + (uint64_t)b * rows, v);
+            acc[b] = 0.f;
+        }
         ++yrow;
         left = rs;
         xaddr = xlane;
     }
     __device__ __forceinline__ void operator()(uint4 w)
     {
-        const uint4 x = lds128(xaddr);
-        const uint32_t wv[4] = {w.x, w.y, w.z, w.w}, xv[4] = {x.x, x.y, x.z, x.w};
+        const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
+        float2 wf[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&wv[i]));
-            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&xv[i]));
-            acc = fmaf(a.x, b.x, acc);
-            acc = fmaf(a.y, b.y, acc);
+        for (int i = 0; i < 4; ++i) wf[i] = __half22float2(*reinterpret_cast<const __half2*>(&wv[i]));
+#pragma unroll
+        for (int b = 0; b < B; ++b) {
+            const uint4 x = lds128(xaddr + (uint32_t)b * xstride);
+            const uint32_t xv[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xv[i]));
+                acc[b] = fmaf(wf[i].x, xf.x, acc[b]);
+                acc[b] = fmaf(wf[i].y, xf.y, acc[b]);
+            }
         }
         xaddr += 512u;
         if (--left == 0u) flush();
@@ -1037,7 +1066,8 @@ __device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status
 template <int K, int kSink>
 __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Ready& r, Lane L, uint32_t lane)
 {
-    constexpr bool kGemv = kSink == kSinkGemv;
+    constexpr int kBatch = kGemvBatchOf<kSink>;
+    constexpr bool kGemv = kBatch > 0;
     if (L.kind == kSkip) return;
     const DevTensor& T = *tensor_ptr<K>();
     const GemvTensor* G = kGemv ? gemv_ptr<K>() : nullptr;
@@ -1056,7 +1086,7 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         }
     }
     if (L.kind == kGeneral) {
-        decode_chunk_general(aux_ptr<K>(), status, T, G, kSink, r.c, L.start, L.end, lane);
+        decode_chunk_general<kBatch>(aux_ptr<K>(), status, T, G, kSink, r.c, L.start, L.end, lane);
         return;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
@@ -1066,14 +1096,18 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         const uint32_t rs = G->cols >> 8;
         const uint32_t gs0 = (uint32_t)(((uint64_t)r.c * T.chunk_symbols) >> 8);
         const uint32_t row0 = gs0 / rs, k0 = gs0 - row0 * rs;
-        EmitDot em;
+        EmitDot<kGemv ? kBatch : 1> em;
         em.lane = lane;
         em.rs = rs;
         em.left = rs - k0;
         em.xlane = kSmemBase + kGemvX<K> + lane * 16u;
         em.xaddr = em.xlane + k0 * 512u;
-        em.acc = 0.f;
+        em.xstride = G->cols * 2u;
+#pragma unroll
+        for (int b = 0; b < (kGemv ? kBatch : 1); ++b) em.acc[b] = 0.f;
         em.yrow = G->y32 + row0;
+        em.rows = G->rows;
+        em.batch = G->batch;
         stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
         em.finish();
     } else if (kSink == kSinkBytes) {
@@ -1109,9 +1143,10 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                                                          const TensorTables* __restrict__ tables,
                                                          uint32_t stage_bytes,
                                                          uint32_t* __restrict__ control,
-                                                         const GemvTensor* __restrict__ gemv)
+                                                         const GemvTensor* __restrict__ gemv, uint32_t rings_at)
 {
-    constexpr bool kGemv = kSink == kSinkGemv;
+    constexpr int kBatch = kGemvBatchOf<kSink>;
+    constexpr bool kGemv = kBatch > 0;
     // layout: [tables][aux][tensor]([gemv descriptor][x])[per-warp rings][over-read pad][mbarriers][index slots][item + claim slots]
     if (smem_addr(smem) != kSmemBase) {   // the lookups' address arithmetic would be wrong: refuse to run
         if (threadIdx.x == 0) atomicOr(control + 1, kStatInternal);
@@ -1121,7 +1156,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     DevTensor* s_tensor = tensor_ptr<K>();
     const uint32_t warps = blockDim.x >> 5;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr uint32_t kRings = kRingsAt<K, kGemv>;
+    const uint32_t kRings = rings_at;          // rings_offset<K>(kGemv, bytes of staged x)
     const uint32_t after = kRings + warps * stage_bytes + kOverRead;          // offset in smem, a multiple of 16
     const uint32_t slots = after + warps * 16u;
     volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(smem + slots + warps * 2u * kSlotBytes);   // [2]
@@ -1177,10 +1212,13 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                 const uint4* gg = reinterpret_cast<const uint4*>(gemv + cur);
                 uint4* sg = reinterpret_cast<uint4*>(gemv_ptr<K>());
                 if (threadIdx.x < sizeof(GemvTensor) / 16) sg[threadIdx.x] = __ldg(gg + threadIdx.x);
+                // x of the batch's tokens, then zeros for the accumulators that have no token
                 const uint4* gx = reinterpret_cast<const uint4*>(gemv[cur].x);      // cols is a multiple of 256
                 uint4* sx = reinterpret_cast<uint4*>(smem + kGemvX<K>);
                 const uint32_t n16 = gemv[cur].cols / 8u;
-                for (uint32_t i = threadIdx.x; i < n16; i += blockDim.x) sx[i] = __ldg(gx + i);
+                const uint32_t have = n16 * gemv[cur].batch, want = n16 * (uint32_t)kBatch;
+                for (uint32_t i = threadIdx.x; i < want; i += blockDim.x)
+                    sx[i] = i < have ? __ldg(gx + i) : make_uint4(0u, 0u, 0u, 0u);
             }
             if (__ldg(&tt->aux.oct)) {
                 const uint4* g1 = tt->oct_val;
@@ -1246,10 +1284,10 @@ struct Shape {
 };
 
 // Shared memory of one CTA for a launch shape; stage_bytes == 0 if it cannot fit.
-Shape shape_for(const DecodeConfig& cfg, int max_smem, bool gemv = false)
+Shape shape_for(const DecodeConfig& cfg, int max_smem, bool gemv = false, uint32_t x_bytes = 0)
 {
     size_t fixed = lut_bytes(cfg.lut_bits) + sizeof(DecodeAux) + sizeof(DevTensor) + 128 + kOverRead;
-    if (gemv) fixed += sizeof(GemvTensor) + 2 * kGemvMaxCols;
+    if (gemv) fixed += sizeof(GemvTensor) + x_bytes;
     size_t per_warp_fixed = 16 + 2 * kSlotBytes;   // two mbarriers, two index slots
     size_t tail = 16;
     size_t budget = (size_t)max_smem / cfg.ctas_per_sm;
@@ -1267,11 +1305,12 @@ Shape shape_for(const DecodeConfig& cfg, int max_smem, bool gemv = false)
 template <int K, int kSink>
 entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
                            const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
-                           const GemvTensor* gemv, cudaStream_t s)
+                           const GemvTensor* gemv, cudaStream_t s, uint32_t x_bytes)
 {
-    Shape sh = shape_for(cfg, ws->max_smem_optin, kSink == kSinkGemv);
+    constexpr bool kGemv = kGemvBatchOf<kSink> > 0;
+    Shape sh = shape_for(cfg, ws->max_smem_optin, kGemv, x_bytes);
     if (sh.stage_bytes == 0) return ENTRO_ERR_UNSUPPORTED;
-    static int configured_smem[64] = {0};
+    static int configured_smem[64] = {0};      // per instantiation of this template
     if ((int)sh.smem > configured_smem[ws->device]) {
         ENTRO_CUDA(cudaFuncSetAttribute(decode_kernel<K, kSink>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sh.smem));
@@ -1282,7 +1321,7 @@ entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTens
     const bool timed = ws->prof_used < ws->prof_cap;
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_start[ws->prof_used], s));
     decode_kernel<K, kSink><<<grid, cfg.warps_per_cta * 32, sh.smem, s>>>(
-        tensors, ntensors, item_start, tables, sh.stage_bytes, ws->control, gemv);
+        tensors, ntensors, item_start, tables, sh.stage_bytes, ws->control, gemv, rings_offset<K>(kGemv, x_bytes));
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_stop[ws->prof_used++], s));
@@ -1292,21 +1331,32 @@ entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTens
 template <int kSink>
 entro_status launch_decode_sink(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
                                 const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
-                                const GemvTensor* gemv, cudaStream_t s)
+                                const GemvTensor* gemv, cudaStream_t s, uint32_t x_bytes = 0)
 {
     switch (cfg.lut_bits) {
-        case 10: return launch_decode<10, kSink>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
-        case 11: return launch_decode<11, kSink>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
-        case 12: return launch_decode<12, kSink>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
+        case 10: return launch_decode<10, kSink>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s, x_bytes);
+        case 11: return launch_decode<11, kSink>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s, x_bytes);
+        case 12: return launch_decode<12, kSink>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s, x_bytes);
     }
     return ENTRO_ERR_UNSUPPORTED;
 }
 
+// gemv != nullptr: the fused matrix-vector kernel with `batch` accumulators per lane (1, 2,
+// 4 or 8) and x_bytes of shared memory for x.
 entro_status launch_decode_any(Workspace* ws, const DecodeConfig& cfg, const DevTensor* tensors, int ntensors,
                                const uint32_t* item_start, uint32_t total_items, const TensorTables* tables,
-                               cudaStream_t s, const GemvTensor* gemv = nullptr, int sink = kSinkFp16)
+                               cudaStream_t s, const GemvTensor* gemv = nullptr, int sink = kSinkFp16, int batch = 1,
+                               uint32_t x_bytes = 0)
 {
-    if (gemv) return launch_decode_sink<kSinkGemv>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s);
+    if (gemv) {
+        switch (batch) {
+            case 1: return launch_decode_sink<kSinkGemv>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s, x_bytes);
+            case 2: return launch_decode_sink<kSinkGemv2>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s, x_bytes);
+            case 4: return launch_decode_sink<kSinkGemv4>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s, x_bytes);
+            case 8: return launch_decode_sink<kSinkGemv8>(ws, cfg, tensors, ntensors, item_start, total_items, tables, gemv, s, x_bytes);
+        }
+        return ENTRO_ERR_UNSUPPORTED;
+    }
     switch (sink) {
         case kSinkFp16: return launch_decode_sink<kSinkFp16>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
         case kSinkBytes: return launch_decode_sink<kSinkBytes>(ws, cfg, tensors, ntensors, item_start, total_items, tables, nullptr, s);
@@ -1578,7 +1628,8 @@ __global__ void __launch_bounds__(256) gemv_finalize_kernel(const GemvTensor* __
 {
     for (int t = blockIdx.y; t < ntensors; t += gridDim.y) {
         const GemvTensor G = g[t];
-        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < G.rows; i += gridDim.x * blockDim.x)
+        const uint32_t n = G.rows * G.batch;      // both are [batch][rows]
+        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
             G.y[i] = __half_as_ushort(__float2half_rn(G.y32[i]));
     }
 }
@@ -1620,6 +1671,7 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
     if (ntensors < 0 || (ntensors > 0 && (!descs_host || !io_host))) return ENTRO_ERR_INVALID_ARG;
     if (ntensors == 0) return ENTRO_OK;
     uint64_t total_rows = 0;
+    uint32_t max_batch = 1;
     for (int i = 0; i < ntensors; ++i) {
         const entro_tensor_desc& d = descs_host[i];
         const entro_gemv_io& g = io_host[i];
@@ -1629,9 +1681,20 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
         if (!g.x_fp16_dev || !g.y_fp16_dev || !aligned(g.x_fp16_dev, 16) || !aligned(g.y_fp16_dev, 2))
             return ENTRO_ERR_INVALID_ARG;
         if (g.rows == 0 || g.cols == 0 || (uint64_t)g.rows * g.cols != d.n) return ENTRO_ERR_INVALID_ARG;
-        if (g.cols % 256u || g.cols > kGemvMaxCols || d.chunk_symbols % 256u) return ENTRO_ERR_UNSUPPORTED;
-        total_rows += g.rows;
+        if (g.batch < 1 || g.batch > ENTRO_GEMV_MAX_BATCH || g.reserved != 0) return ENTRO_ERR_INVALID_ARG;
+        if ((uint64_t)g.rows * g.batch > 0xffffffffull) return ENTRO_ERR_UNSUPPORTED;
+        if (g.cols % 256u || (uint64_t)g.cols * g.batch > kGemvMaxX || d.chunk_symbols % 256u) return ENTRO_ERR_UNSUPPORTED;
+        total_rows += (uint64_t)g.rows * g.batch;
+        if (g.batch > max_batch) max_batch = g.batch;
     }
+    // accumulators per lane: the batch rounded up to 1, 2, 4 or 8; x of that many tokens is staged
+    const uint32_t lanes_batch = max_batch <= 1 ? 1u : max_batch <= 2 ? 2u : max_batch <= 4 ? 4u : 8u;
+    uint32_t x_bytes = 0;
+    for (int i = 0; i < ntensors; ++i) {
+        const uint32_t need = (io_host[i].cols * lanes_batch * 2u + 127u) & ~127u;
+        if (need > x_bytes) x_bytes = need;
+    }
+    if (x_bytes > 2u * kGemvMaxX) return ENTRO_ERR_UNSUPPORTED;   // a wide matrix beside a larger batch elsewhere in the call
     cudaStream_t s = (cudaStream_t)cuda_stream;
     Guard guard;
     Workspace* ws = workspace();
@@ -1664,7 +1727,9 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
         hg[i].y = static_cast<uint16_t*>(io_host[i].y_fp16_dev);
         hg[i].rows = io_host[i].rows;
         hg[i].cols = io_host[i].cols;
-        row0 += io_host[i].rows;
+        hg[i].batch = io_host[i].batch;
+        hg[i].pad[0] = hg[i].pad[1] = hg[i].pad[2] = 0;
+        row0 += (uint64_t)io_host[i].rows * io_host[i].batch;
     }
     hitems[ntensors] = (uint32_t)items;
     DevTensor* dt = reinterpret_cast<DevTensor*>(base);
@@ -1677,7 +1742,8 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
     build_tables_kernel<<<ntensors, 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
-    entro_status st = launch_decode_any(ws, cfg, dt, ntensors, ditems, (uint32_t)items, dtables, s, dg);
+    entro_status st = launch_decode_any(ws, cfg, dt, ntensors, ditems, (uint32_t)items, dtables, s, dg, kSinkGemv,
+                                        (int)lanes_batch, x_bytes);
     if (st != ENTRO_OK) return st;
     dim3 grid(16, (unsigned)(ntensors < 64 ? ntensors : 64));
     gemv_finalize_kernel<<<grid, 256, 0, s>>>(dg, ntensors);

@@ -41,13 +41,15 @@ static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vecto
 
 // The matrix-vector side of one tensor for the fused decode + GEMV kernel.
 struct GemvTensor {
-    const uint16_t* x;    // cols fp16 values
-    float* y32;           // rows fp32 accumulators (workspace), zero before the kernel
-    uint16_t* y;          // rows fp16 results
+    const uint16_t* x;    // [batch][cols] fp16 values
+    float* y32;           // [batch][rows] fp32 accumulators (workspace), zero before the kernel
+    uint16_t* y;          // [batch][rows] fp16 results
     uint32_t rows, cols;
+    uint32_t batch;       // tokens, 1 .. ENTRO_GEMV_MAX_BATCH
+    uint32_t pad[3];
 };
-static_assert(sizeof(GemvTensor) == 32, "GemvTensor is read as two 16-byte vectors");
-constexpr uint32_t kGemvMaxCols = 16384;      // x is staged in shared memory as fp16
+static_assert(sizeof(GemvTensor) == 48, "GemvTensor is read as three 16-byte vectors");
+constexpr uint32_t kGemvMaxX = 32768;         // fp16 values of x (all tokens) staged in shared memory
 
 // Per-tensor canonical-code description beside the lookup tables.
 struct DecodeAux {
@@ -87,10 +89,16 @@ struct DecodeConfig {
 // Where the decode kernel sends the decoded values.
 enum Sink : int {
     kSinkFp16 = 0,      // dequantised fp16 values to the output tensor
-    kSinkGemv = 1,      // dequantised fp16 values into a matrix-vector product
+    kSinkGemv = 1,      // dequantised fp16 values into a matrix-vector product, one token
     kSinkBytes = 2,     // the symbols, one per byte
-    kSinkNibbles = 3    // the symbols, two per byte, the earlier one in the low nibble
+    kSinkNibbles = 3,   // the symbols, two per byte, the earlier one in the low nibble
+    kSinkGemv2 = 4,     // ... into the products with up to 2, 4, 8 tokens
+    kSinkGemv4 = 5,
+    kSinkGemv8 = 6
 };
+// Accumulators per lane of a matrix-vector sink (0: not such a sink).
+template <int kSink>
+constexpr int kGemvBatchOf = kSink == kSinkGemv ? 1 : kSink == kSinkGemv2 ? 2 : kSink == kSinkGemv4 ? 4 : kSink == kSinkGemv8 ? 8 : 0;
 
 // Per-device workspace owned by the library.
 struct Workspace {
