@@ -906,22 +906,29 @@ struct EmitDot {
         left = rs;
         xaddr = xlane;
     }
+    // acc += w.lo * x.lo, then acc += w.hi * x.hi: fp16 operands, fp32 sum, one rounding per step
+    // (the product of two fp16 values is exact in fp32, so this is fmaf on the converted values).
+    static __device__ __forceinline__ void fma2(float& acc, uint32_t w, uint32_t x)
+    {
+        asm("{\n\t"
+            ".reg .b16 wl, wh, xl, xh;\n\t"
+            "mov.b32 {wl, wh}, %1;\n\t"
+            "mov.b32 {xl, xh}, %2;\n\t"
+            "fma.rn.f32.f16 %0, wl, xl, %0;\n\t"
+            "fma.rn.f32.f16 %0, wh, xh, %0;\n\t"
+            "}"
+            : "+f"(acc)
+            : "r"(w), "r"(x));
+    }
     __device__ __forceinline__ void operator()(uint4 w)
     {
-        const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
-        float2 wf[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) wf[i] = __half22float2(*reinterpret_cast<const __half2*>(&wv[i]));
 #pragma unroll
         for (int b = 0; b < B; ++b) {
             const uint4 x = lds128(xaddr + (uint32_t)b * xstride);
-            const uint32_t xv[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xv[i]));
-                acc[b] = fmaf(wf[i].x, xf.x, acc[b]);
-                acc[b] = fmaf(wf[i].y, xf.y, acc[b]);
-            }
+            fma2(acc[b], w.x, x.x);
+            fma2(acc[b], w.y, x.y);
+            fma2(acc[b], w.z, x.z);
+            fma2(acc[b], w.w, x.w);
         }
         xaddr += 512u;
         if (--left == 0u) flush();
