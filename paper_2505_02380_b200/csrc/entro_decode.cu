@@ -1412,7 +1412,7 @@ ItemPlan plan_items(const DecodeConfig& cfg, const entro_tensor_desc* descs, int
     if (want < (uint64_t)cfg.warps_per_cta) want = cfg.warps_per_cta;
     p.base = want < (uint64_t)cfg.chunks_per_item ? (uint32_t)want : (uint32_t)cfg.chunks_per_item;
     p.tail = p.base / 8 < (uint32_t)cfg.warps_per_cta ? (uint32_t)cfg.warps_per_cta : p.base / 8;
-    p.graded = live >= 8 && p.base == (uint32_t)cfg.chunks_per_item;
+    p.graded = live >= 8 && p.base >= 8u * (uint32_t)cfg.warps_per_cta;   // a tail item still gives every warp a chunk
     return p;
 }
 
