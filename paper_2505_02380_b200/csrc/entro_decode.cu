@@ -82,6 +82,9 @@ __device__ __forceinline__ uint32_t range_decode(const DecodeAux& aux, uint32_t 
 }
 
 // One block per tensor.
+// The grid is (tensors, kTableSlices): every block of a tensor works out the small things
+// for itself and fills its share of the tables' entries.
+constexpr unsigned kTableSlices = 8;
 __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __restrict__ tensors, int lut_bits,
                                                            TensorTables* __restrict__ tables,
                                                            uint32_t* __restrict__ control)
@@ -94,7 +97,8 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     const int tid = threadIdx.x;
     const DevTensor& T = tensors[t];
     TensorTables& out = tables[t];
-    if (t == 0 && tid == 0) control[0] = 0;   // work counter of the decode kernel that follows
+    const uint32_t first = blockIdx.y * 256u + (uint32_t)tid, stride = gridDim.y * 256u;   // this thread's entries
+    if (t == 0 && first == 0) control[0] = 0;   // work counter of the decode kernel that follows
     if (tid <= ENTRO_MAX_CODE_LEN) count[tid] = 0;
     len[tid] = (uint32_t)tid < T.nsym ? T.len[tid] : 0;
     __syncthreads();
@@ -198,7 +202,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
 
     if (aux.oct) {
         const uint32_t entries = 1u << lut_bits;
-        for (uint32_t i = tid; i < entries; i += 256) {
+        for (uint32_t i = first; i < entries; i += stride) {
             uint32_t window = i << (32 - lut_bits);
             uint32_t used = 0;
             uint32_t v[8];
@@ -223,7 +227,7 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     {
         // cell (e5, mant): windows that start with r ones and a zero, followed by the bits ~mant
         const uint32_t kExpBits = aux.expm;
-        for (uint32_t i = tid; i < (32u << kExpBits); i += 256) {
+        for (uint32_t i = first; i < (32u << kExpBits); i += stride) {
             const uint32_t e5 = i >> kExpBits, mant = i & ((1u << kExpBits) - 1u);
             const uint32_t r = (30u - e5) & 31u;
             const uint32_t avail = 31u - r;                               // window bits after the zero
@@ -250,7 +254,8 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     }
     const uint32_t* src = reinterpret_cast<const uint32_t*>(&aux);
     uint32_t* dst = reinterpret_cast<uint32_t*>(&out.aux);
-    for (uint32_t i = tid; i < sizeof(DecodeAux) / 4; i += 256) dst[i] = src[i];
+    if (blockIdx.y == 0)
+        for (uint32_t i = tid; i < sizeof(DecodeAux) / 4; i += 256) dst[i] = src[i];
 }
 
 // ------------------------------------------------------------------ bit reader
@@ -1487,7 +1492,7 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     TensorTables* dtables = reinterpret_cast<TensorTables*>(base + upload_bytes);
     ENTRO_CUDA(cudaMemcpyAsync(dt, ht, upload_bytes, cudaMemcpyHostToDevice, s));
     mark_pinned_in_use(ws, s);
-    build_tables_kernel<<<live, 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
+    build_tables_kernel<<<dim3((unsigned)live, kTableSlices), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     return launch_decode_any(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, s, nullptr, sink);
@@ -1746,7 +1751,7 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
     ENTRO_CUDA(cudaMemcpyAsync(dt, ht, upload_bytes, cudaMemcpyHostToDevice, s));
     mark_pinned_in_use(ws, s);
     ENTRO_CUDA(cudaMemsetAsync(y32, 0, y32_bytes, s));
-    build_tables_kernel<<<ntensors, 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
+    build_tables_kernel<<<dim3((unsigned)ntensors, kTableSlices), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     entro_status st = launch_decode_any(ws, cfg, dt, ntensors, ditems, (uint32_t)items, dtables, s, dg, kSinkGemv,
@@ -1889,7 +1894,7 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
     static_upload_kernel<<<1, 256, 0, s>>>(up, sc);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
-    build_tables_kernel<<<live, 256, 0, s>>>(sc->tensors, cfg.lut_bits, sc->tables, sc->control);
+    build_tables_kernel<<<dim3((unsigned)live, kTableSlices), 256, 0, s>>>(sc->tensors, cfg.lut_bits, sc->tables, sc->control);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     // launch_decode reads only these fields of a workspace; no timing records are taken here
