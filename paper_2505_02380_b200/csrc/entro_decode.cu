@@ -87,7 +87,8 @@ __device__ __forceinline__ uint32_t range_decode(const DecodeAux& aux, uint32_t 
 constexpr unsigned kTableSlices = 8;
 __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __restrict__ tensors, int lut_bits,
                                                            TensorTables* __restrict__ tables,
-                                                           uint32_t* __restrict__ control)
+                                                           uint32_t* __restrict__ control,
+                                                           const GemvTensor* __restrict__ gemv)
 {
     __shared__ DecodeAux aux;
     __shared__ uint32_t count[ENTRO_MAX_CODE_LEN + 1];
@@ -99,6 +100,11 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     TensorTables& out = tables[t];
     const uint32_t first = blockIdx.y * 256u + (uint32_t)tid, stride = gridDim.y * 256u;   // this thread's entries
     if (t == 0 && first == 0) control[0] = 0;   // work counter of the decode kernel that follows
+    if (gemv) {                                 // and the fp32 sums of the fused matrix-vector products
+        float* y32 = gemv[t].y32;
+        const uint32_t n = gemv[t].rows * gemv[t].batch;
+        for (uint32_t i = first; i < n; i += stride) y32[i] = 0.f;
+    }
     if (tid <= ENTRO_MAX_CODE_LEN) count[tid] = 0;
     len[tid] = (uint32_t)tid < T.nsym ? T.len[tid] : 0;
     __syncthreads();
@@ -1492,7 +1498,7 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     TensorTables* dtables = reinterpret_cast<TensorTables*>(base + upload_bytes);
     ENTRO_CUDA(cudaMemcpyAsync(dt, ht, upload_bytes, cudaMemcpyHostToDevice, s));
     mark_pinned_in_use(ws, s);
-    build_tables_kernel<<<dim3((unsigned)live, kTableSlices), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
+    build_tables_kernel<<<dim3((unsigned)live, kTableSlices), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control, nullptr);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     return launch_decode_any(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, s, nullptr, sink);
@@ -1750,8 +1756,7 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
     TensorTables* dtables = reinterpret_cast<TensorTables*>(base + upload_bytes);
     ENTRO_CUDA(cudaMemcpyAsync(dt, ht, upload_bytes, cudaMemcpyHostToDevice, s));
     mark_pinned_in_use(ws, s);
-    ENTRO_CUDA(cudaMemsetAsync(y32, 0, y32_bytes, s));
-    build_tables_kernel<<<dim3((unsigned)ntensors, kTableSlices), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control);
+    build_tables_kernel<<<dim3((unsigned)ntensors, kTableSlices), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control, dg);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     entro_status st = launch_decode_any(ws, cfg, dt, ntensors, ditems, (uint32_t)items, dtables, s, dg, kSinkGemv,
@@ -1894,7 +1899,7 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
     static_upload_kernel<<<1, 256, 0, s>>>(up, sc);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
-    build_tables_kernel<<<dim3((unsigned)live, kTableSlices), 256, 0, s>>>(sc->tensors, cfg.lut_bits, sc->tables, sc->control);
+    build_tables_kernel<<<dim3((unsigned)live, kTableSlices), 256, 0, s>>>(sc->tensors, cfg.lut_bits, sc->tables, sc->control, nullptr);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     // launch_decode reads only these fields of a workspace; no timing records are taken here

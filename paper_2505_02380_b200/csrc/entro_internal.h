@@ -42,7 +42,7 @@ static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vecto
 // The matrix-vector side of one tensor for the fused decode + GEMV kernel.
 struct GemvTensor {
     const uint16_t* x;    // [batch][cols] fp16 values
-    float* y32;           // [batch][rows] fp32 accumulators (workspace), zero before the kernel
+    float* y32;           // [batch][rows] fp32 accumulators (workspace), zeroed by the table build
     uint16_t* y;          // [batch][rows] fp16 results
     uint32_t rows, cols;
     uint32_t batch;       // tokens, 1 .. ENTRO_GEMV_MAX_BATCH
