@@ -73,6 +73,8 @@ def lib():
         L.oracle_quantize_one.restype = C.c_uint8
         L.oracle_quantize_one.argtypes = [C.c_uint16, C.c_float, C.c_int, C.c_int]
         L.oracle_quantize_tensor.argtypes = [u16p, C.c_uint64, C.c_int, C.c_int, u8p, C.POINTER(_QParams)]
+        L.oracle_quantize_blocks.argtypes = [u16p, C.c_uint64, C.c_int, C.c_int, C.c_uint64, u8p,
+                                             C.POINTER(C.c_float), C.POINTER(C.c_int32)]
         L.oracle_dequant_one.restype = C.c_uint16
         L.oracle_dequant_one.argtypes = [C.c_uint8, C.c_float, C.c_int]
         L.oracle_dequant.restype = None
@@ -167,6 +169,19 @@ def quantize_tensor(w: np.ndarray, bits: int, mode: int = MODE_AUTO):
     _check(lib().oracle_quantize_tensor(_ptr(w, C.c_uint16), w.size, bits, mode, _ptr(q, C.c_uint8),
                                         C.byref(qp)))
     return q, QParams(qp.bits, qp.mode, qp.scale, qp.zero_point, qp.lo, qp.hi)
+
+
+def quantize_blocks(w: np.ndarray, bits: int, block: int, mode: int = MODE_AUTO):
+    """Block-based quantisation, the paper's comparison grid (Section 3, Table 2 "SOTA"): every run of
+    `block` weights by itself.  -> (q uint8 [n], scales float32 [blocks], zero points int32 [blocks])"""
+    w = _as_u16(w)
+    nb = (w.size + block - 1) // block
+    q = np.empty(w.size, dtype=np.uint8)
+    scales = np.empty(nb, dtype=np.float32)
+    zps = np.empty(nb, dtype=np.int32)
+    _check(lib().oracle_quantize_blocks(_ptr(w, C.c_uint16), w.size, bits, mode, block, _ptr(q, C.c_uint8),
+                                        _ptr(scales, C.c_float), _ptr(zps, C.c_int32)))
+    return q, scales, zps
 
 
 def dequant(q: np.ndarray, s: float, z: int) -> np.ndarray:

@@ -197,6 +197,29 @@ int oracle_quantize_tensor(const uint16_t *w, uint64_t n, int bits, int mode, ui
     return ORACLE_OK;
 }
 
+/*
+ * The grid the paper compares against (Section 3, "Mixed Quantization Scheme"; Table 2,
+ * column "SOTA"): block-based quantisation, every run of `block` consecutive weights
+ * ("e.g., blocks of 32 weights") with a range, scale and zero point of its own, by the same
+ * Eq. 1.  The last block may be shorter.  scales / zps (one per block) may be NULL.
+ */
+int oracle_quantize_blocks(const uint16_t *w, uint64_t n, int bits, int mode, uint64_t block, uint8_t *q,
+                           float *scales, int32_t *zps)
+{
+    if (!w || !q || n == 0 || block == 0) return ORACLE_ERR_ARG;
+    uint64_t b = 0;
+    for (uint64_t first = 0; first < n; first += block, ++b) {
+        const uint64_t m = n - first < block ? n - first : block;
+        oracle_qparams qp;
+        int rc = oracle_quant_params(w + first, m, bits, mode, &qp);
+        if (rc) return rc;
+        for (uint64_t i = 0; i < m; ++i) q[first + i] = oracle_quantize_one(w[first + i], qp.scale, qp.zero_point, bits);
+        if (scales) scales[b] = qp.scale;
+        if (zps) zps[b] = qp.zero_point;
+    }
+    return ORACLE_OK;
+}
+
 /* w_hat = fp16( s * (q - z) ), the product taken in fp32 and rounded once. */
 uint16_t oracle_dequant_one(uint8_t q, float s, int z)
 {
