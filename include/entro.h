@@ -113,6 +113,22 @@ entro_status entro_quantize_tensor(const void *w_fp16_dev, uint64_t n, int bits,
                                    uint8_t *q_dev, entro_qparams *qp_host, void *cuda_stream);
 
 /*
+ * The grid the paper argues against, for comparison (Section 3, "Mixed Quantization
+ * Scheme"; Table 2, column "SOTA"): block-based quantisation.  Every run of `block`
+ * consecutive weights (the paper's example is 32; the last run may be shorter) gets a range,
+ * mode, s and z of its own by the rules of entro_quantize_tensor, and is quantised with
+ * them.  The paper's point is that such grids flatten the histogram of the codes, so that
+ * entropy coding saves little; entro_histogram and entro_build_codebook on q_dev measure it.
+ * w_fp16_dev: n fp16 weights (device).  q_dev: n bytes (device), one symbol per byte.
+ * scales_dev / zero_points_dev: ceil(n / block) values each (device), or NULL if not wanted.
+ * Synchronises.  ENTRO_ERR_NONFINITE if a weight is NaN or infinite (blocks that hold one
+ * are left unwritten).
+ */
+entro_status entro_quantize_blocks(const void *w_fp16_dev, uint64_t n, int bits, entro_mode mode,
+                                   uint32_t block, uint8_t *q_dev, float *scales_dev,
+                                   int32_t *zero_points_dev, void *cuda_stream);
+
+/*
  * Symbol frequencies, the "score" each symbol gets in Section 3 ("Huffman weight
  * encoding").  counts_host[k] = number of symbols equal to k, k < 2^bits.  Synchronises.
  * ENTRO_ERR_INVALID_ARG if a symbol is >= 2^bits.

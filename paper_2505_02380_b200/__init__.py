@@ -92,6 +92,7 @@ def lib():
         vp, u64, u32, i32 = C.c_void_p, C.c_uint64, C.c_uint32, C.c_int
         L.entro_quantize_tensor.argtypes = [vp, u64, i32, i32, vp, C.POINTER(QParams), vp]
         L.entro_histogram.argtypes = [vp, u64, i32, C.POINTER(C.c_uint64), vp]
+        L.entro_quantize_blocks.argtypes = [vp, u64, i32, i32, u32, vp, vp, vp, vp]
         L.entro_build_codebook.argtypes = [C.POINTER(C.c_uint64), i32, C.POINTER(Codebook)]
         L.entro_build_codebook_limited.argtypes = [C.POINTER(C.c_uint64), i32, i32, C.POINTER(Codebook)]
         L.entro_stream_words.restype = u64
@@ -124,7 +125,7 @@ def lib():
 
 
 # Every symbol include/entro.h declares.
-EXPORTS = ["entro_quantize_tensor", "entro_histogram", "entro_build_codebook", "entro_build_codebook_limited", "entro_stream_words",
+EXPORTS = ["entro_quantize_tensor", "entro_quantize_blocks", "entro_histogram", "entro_build_codebook", "entro_build_codebook_limited", "entro_stream_words",
            "entro_encode_bound_words", "entro_index_bytes", "entro_encode", "entro_decode_dequant",
            "entro_decode_dequant_batched", "entro_decode_dequant_batched_host", "entro_decode_dequant_static",
            "entro_decode_dequant_gemv", "entro_gemv_fp16", "entro_decode_symbols_batched", "entro_last_device_status",
@@ -161,6 +162,20 @@ def entro_quantize_tensor(w_fp16: torch.Tensor, bits: int, mode: int = MODE_AUTO
     _check(lib().entro_quantize_tensor(_dev(w_fp16, torch.float16), n, bits, mode, q.data_ptr(), C.byref(qp),
                                        _stream(stream)), "entro_quantize_tensor")
     return q, qp
+
+
+def entro_quantize_blocks(w_fp16: torch.Tensor, bits: int, block: int = 32, mode: int = MODE_AUTO,
+                          stream: Optional[torch.cuda.Stream] = None):
+    """Block-based quantisation, the paper's comparison grid.
+    -> (q uint8 device tensor, scales float32 [blocks], zero points int32 [blocks])"""
+    n = w_fp16.numel()
+    nb = (n + block - 1) // block
+    q = torch.empty(n, dtype=torch.uint8, device=w_fp16.device)
+    scales = torch.empty(nb, dtype=torch.float32, device=w_fp16.device)
+    zps = torch.empty(nb, dtype=torch.int32, device=w_fp16.device)
+    _check(lib().entro_quantize_blocks(_dev(w_fp16, torch.float16), n, bits, mode, block, q.data_ptr(),
+                                       scales.data_ptr(), zps.data_ptr(), _stream(stream)), "entro_quantize_blocks")
+    return q, scales, zps
 
 
 def entro_histogram(q: torch.Tensor, bits: int, stream: Optional[torch.cuda.Stream] = None) -> np.ndarray:

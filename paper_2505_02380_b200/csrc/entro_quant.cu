@@ -129,6 +129,56 @@ __global__ void __launch_bounds__(kThreads) quantise_kernel(const uint16_t* __re
     }
 }
 
+// Block-based grid: one warp per block of `block` consecutive weights.  The warp finds the
+// block's range, every lane derives the same (s, z) from it with the arithmetic of the
+// per-tensor call (IEEE fp32, one rounding per operation), then the block is quantised.
+__global__ void __launch_bounds__(kThreads) quantise_blocks_kernel(const uint16_t* __restrict__ w, uint64_t n,
+                                                                   uint32_t block, uint64_t nblocks, int qmax, int mode,
+                                                                   uint8_t* __restrict__ q, float* __restrict__ scales,
+                                                                   int32_t* __restrict__ zps,
+                                                                   uint32_t* __restrict__ nonfinite)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warps = ((uint64_t)gridDim.x * kThreads) >> 5;
+    for (uint64_t b = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) >> 5; b < nblocks; b += warps) {
+        const uint64_t first = b * block;
+        const uint32_t m = (uint32_t)min((uint64_t)block, n - first);
+        float lo = INFINITY, hi = -INFINITY;
+        uint32_t bad = 0;
+        for (uint32_t i = lane; i < m; i += 32u) scan_half(w[first + i], lo, hi, bad);
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+            bad |= __shfl_xor_sync(0xffffffffu, bad, d);
+        }
+        if (bad) {
+            if (lane == 0) atomicOr(nonfinite, 1u);
+            continue;
+        }
+        if (lo == 0.0f) lo = 0.0f;   // -0 and +0 are the same bound
+        if (hi == 0.0f) hi = 0.0f;
+        const bool unsigned_grid = mode == ENTRO_MODE_UNSIGNED || (mode == ENTRO_MODE_AUTO && lo >= 0.0f);
+        float s;
+        int z = 0;
+        if (unsigned_grid) {
+            s = __fdiv_rn(hi, (float)qmax);
+            if (!(s > 0.0f)) s = 1.0f;
+        } else {
+            s = __fdiv_rn(__fsub_rn(hi, lo), (float)qmax);
+            if (!(s > 0.0f)) s = 1.0f;
+            float zr = rintf(__fdiv_rn(-lo, s));
+            zr = zr < 0.0f ? 0.0f : (zr > (float)qmax ? (float)qmax : zr);
+            z = (int)zr;
+        }
+        for (uint32_t i = lane; i < m; i += 32u) q[first + i] = (uint8_t)quantise_one(w[first + i], s, z, qmax);
+        if (lane == 0) {
+            if (scales) scales[b] = s;
+            if (zps) zps[b] = z;
+        }
+    }
+}
+
 // Per-warp shared-memory histograms, merged into 64-bit global counters.
 __global__ void __launch_bounds__(kThreads) histogram_kernel(const uint8_t* __restrict__ q, uint64_t n, uint32_t nsym,
                                                              unsigned long long* __restrict__ counts,
@@ -244,6 +294,34 @@ extern "C" entro_status entro_quantize_tensor(const void* w_fp16_dev, uint64_t n
     ENTRO_CUDA(cudaGetLastError());
     ENTRO_CUDA(cudaStreamSynchronize(s));
     return ENTRO_OK;
+}
+
+extern "C" entro_status entro_quantize_blocks(const void* w_fp16_dev, uint64_t n, int bits, entro_mode mode,
+                                              uint32_t block, uint8_t* q_dev, float* scales_dev,
+                                              int32_t* zero_points_dev, void* cuda_stream)
+{
+    if (!w_fp16_dev || !q_dev || n == 0 || block == 0 || (bits != 4 && bits != 8)) return ENTRO_ERR_INVALID_ARG;
+    if (mode != ENTRO_MODE_AUTO && mode != ENTRO_MODE_UNSIGNED && mode != ENTRO_MODE_ASYMMETRIC)
+        return ENTRO_ERR_INVALID_ARG;
+    if (!aligned(w_fp16_dev, 2) || (scales_dev && !aligned(scales_dev, 4)) || (zero_points_dev && !aligned(zero_points_dev, 4)))
+        return ENTRO_ERR_INVALID_ARG;
+    Guard g;
+    Workspace* ws = workspace();
+    if (!ws) return ENTRO_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (!reserve_device(ws, 16) || !reserve_pinned(ws, 16)) return ENTRO_ERR_CUDA;
+    uint32_t* flag = static_cast<uint32_t*>(ws->dev);
+    ENTRO_CUDA(cudaMemsetAsync(flag, 0, 4, s));
+    const uint64_t nblocks = (n + block - 1) / block;
+    const int grid = grid_for(nblocks * 32, ws->sm_count, 8);
+    quantise_blocks_kernel<<<grid, kThreads, 0, s>>>(static_cast<const uint16_t*>(w_fp16_dev), n, block, nblocks,
+                                                     (1 << bits) - 1, (int)mode, q_dev, scales_dev, zero_points_dev, flag);
+    count_launch();
+    ENTRO_CUDA(cudaGetLastError());
+    uint32_t* host = static_cast<uint32_t*>(ws->pinned);
+    ENTRO_CUDA(cudaMemcpyAsync(host, flag, 4, cudaMemcpyDeviceToHost, s));
+    ENTRO_CUDA(cudaStreamSynchronize(s));
+    return *host ? ENTRO_ERR_NONFINITE : ENTRO_OK;
 }
 
 extern "C" entro_status entro_histogram(const uint8_t* q_dev, uint64_t n, int bits, uint64_t* counts_host,

@@ -58,6 +58,32 @@ def test_quantise_refuses_nonfinite():
 
 
 @pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("n,block", [(1, 32), (31, 32), (32, 32), (33, 32), (5000, 32), (4096, 128), (100000, 32),
+                                     (777, 1000), (1 << 20, 32)])
+def test_block_quantiser_matches_oracle(bits, n, block):
+    """The comparison grid of Table 2: codes, scales and zero points of every block, bit for bit."""
+    w_np, w = _values(n, 0.02, 13 * n + bits + block)
+    q_ref, s_ref, z_ref = oracle.quantize_blocks(w_np, bits, block)
+    q, scales, zps = E.entro_quantize_blocks(w, bits, block)
+    assert np.array_equal(q.cpu().numpy(), q_ref)
+    assert np.array_equal(scales.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(zps.cpu().numpy(), z_ref)
+    for mode in (E.MODE_UNSIGNED, E.MODE_ASYMMETRIC):
+        q_ref, s_ref, z_ref = oracle.quantize_blocks(w_np, bits, block, mode)
+        q, scales, zps = E.entro_quantize_blocks(w, bits, block, mode)
+        assert np.array_equal(q.cpu().numpy(), q_ref), mode
+        assert np.array_equal(zps.cpu().numpy(), z_ref), mode
+
+
+def test_block_quantiser_refuses_nonfinite():
+    w = torch.zeros(256, dtype=torch.float16, device="cuda")
+    w[77] = float("nan")
+    with pytest.raises(E.EntroError) as e:
+        E.entro_quantize_blocks(w, 8, 32)
+    assert e.value.status == E.ERR_NONFINITE
+
+
+@pytest.mark.parametrize("bits", [4, 8])
 def test_histogram_matches_oracle(bits):
     for n in (1, 15, 16, 17, 100_003, 1 << 21):
         w_np, _ = _values(n, 0.02, n % 1000 + bits)
