@@ -279,11 +279,13 @@ def time_e2e(E, model, steps, warmup):
     return ms, h2d, d2h
 
 
-def measure_gemv(E, max_layers, reps=5):
+def measure_gemv(E, max_layers, reps=5, chunk_symbols=0):
     """Config 5: mistral-7B-shaped 4-bit layer stack, batch-1 fp16 GEMV per projection.  Fused
     (decode + dequant + GEMV, one call per layer) against unfused (decode the layer to fp16,
     then seven plain fp16 GEMVs)."""
     wl = workloads.mistral_layer_stack(max_layers=max_layers)
+    if chunk_symbols:
+        wl = dataclasses.replace(wl, chunk_symbols=chunk_symbols)
     layers = {}
     for spec in wl.tensors:
         layers.setdefault(spec.name.split(".")[1], []).append(spec)
@@ -383,7 +385,7 @@ def measure_gemv(E, max_layers, reps=5):
         batches[str(B)] = {"fused_ms_per_layer": f / nl, "unfused_ms_per_layer": u / nl,
                            "fused_token_weights_per_s": B * n_weights / (f * 1e-3)}
         del calls, gemms
-    return {"workload": wl.name, "layers": nl, "weights": n_weights,
+    return {"workload": wl.name, "layers": nl, "weights": n_weights, "chunk_symbols": wl.chunk_symbols,
             "fused_ms_per_layer": out["fused"] / nl, "unfused_ms_per_layer": out["unfused"] / nl,
             "speedup_fused_vs_unfused": out["unfused"] / out["fused"],
             "weights_per_s": n_weights / (out["fused"] * 1e-3),
@@ -527,6 +529,7 @@ def main():
                     help="use length-limited codes (not the paper's optimal code); 0 = unrestricted Huffman")
     ap.add_argument("--chunk-symbols", type=int, default=0,
                     help="code the main workload with this chunk size instead of its own (a multiple of 256)")
+    ap.add_argument("--gemv-chunk-symbols", type=int, default=0, help="chunk size of the fused-GEMV section's streams")
     ap.add_argument("--lut-bits", type=int, default=0)
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
@@ -572,7 +575,7 @@ def main():
     gemv = None
     if not args.no_gemv and rank == 0 and world == 1:
         torch.cuda.empty_cache()
-        gemv = measure_gemv(E, args.max_layers)
+        gemv = measure_gemv(E, args.max_layers, chunk_symbols=args.gemv_chunk_symbols)
 
     if rank == 0:
         line = {
