@@ -1,0 +1,566 @@
+// One chunk of the decode kernel: bulk copy into the warp's ring, index slots, lane start
+// positions, the general path, and what happens to the decoded values (store, integer
+// output, matrix-vector product).  Included by entro_decode.cu only.
+#pragma once
+
+#include "entro_decode_reader.cuh"
+
+namespace entro {
+namespace {
+
+// ------------------------------------------------------------------ bulk copy + mbarrier
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// Bounded wait for phase `parity` of the barrier; false if the bound ran out.  Each try may
+// suspend the thread for up to the hinted time, so waiting costs few issue slots.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t tries = 0; tries < kWaitTries; ++tries) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity), "r"(20000u)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// ------------------------------------------------------------------ one chunk
+
+// Fixed places in shared memory: [tables][aux][tensor][rings ...].
+template <int K>
+__device__ __forceinline__ DecodeAux* aux_ptr() { return reinterpret_cast<DecodeAux*>(smem + lut_bytes(K)); }
+template <int K>
+__device__ __forceinline__ DevTensor* tensor_ptr()
+{
+    return reinterpret_cast<DevTensor*>(smem + lut_bytes(K) + sizeof(DecodeAux));
+}
+
+// The matrix-vector kernel keeps two more things behind the tensor: its GemvTensor and x.
+template <int K>
+constexpr uint32_t kGemvDesc = lut_bytes(K) + (uint32_t)sizeof(DecodeAux) + (uint32_t)sizeof(DevTensor);
+template <int K>
+constexpr uint32_t kGemvX = kGemvDesc<K> + (uint32_t)sizeof(GemvTensor);
+template <int K>
+__device__ __forceinline__ GemvTensor* gemv_ptr() { return reinterpret_cast<GemvTensor*>(smem + kGemvDesc<K>); }
+// Offset of the first ring: behind the tensor, or behind x_bytes of staged x (a multiple of 128).
+template <int K>
+constexpr uint32_t rings_offset(bool gemv, uint32_t x_bytes)
+{
+    return ((gemv ? kGemvX<K> + x_bytes : kGemvDesc<K>) + 127u) & ~127u;
+}
+
+// What a warp carries from chunk to chunk (kept small: it lives in registers across the
+// decode loop).
+struct WarpCtx {
+    uint32_t stage_addr;       // shared-window address of this warp's ring for compressed bytes
+    uint32_t bar;              // shared-window address of this warp's two mbarriers
+    uint32_t idx_addr;         // shared-window address of this warp's two index slots
+    uint32_t state;            // bulk copies issued so far; bit 31: a copy never completed, stop staging
+    __device__ __forceinline__ bool dead() const { return (state >> 31) != 0u; }
+};
+
+// An index slot holds one chunk's index entries, fetched asynchronously two chunks ahead:
+// the 32 sub-block lengths (64 bytes), then offsets[c] and offsets[c + 1].
+constexpr uint32_t kSlotBytes = 80;
+
+enum : uint32_t { kStaged = 0, kGeneral = 1, kSkip = 2 };
+
+// Chunk whose bytes have been asked for.  meta packs what the staging needs: ring offset /
+// 16 (12 bits), bytes / 16 (12 bits), ticket modulo 4 (2 bits), kind (2 bits), copy issued
+// (1 bit).  Everything else is re-read from the chunk's index slot when it is decoded.
+struct Ready {
+    uint32_t c;                // or kNone
+    uint32_t meta;
+    __device__ __forceinline__ uint32_t at() const { return (meta & 0xfffu) << 4; }
+    __device__ __forceinline__ uint32_t bytes() const { return ((meta >> 12) & 0xfffu) << 4; }
+    __device__ __forceinline__ uint32_t ticket() const { return (meta >> 24) & 3u; }
+    __device__ __forceinline__ uint32_t kind() const { return (meta >> 26) & 3u; }
+    __device__ __forceinline__ bool issued() const { return (meta >> 28) & 1u; }
+};
+__device__ __forceinline__ uint32_t ready_meta(uint32_t at, uint32_t bytes, uint32_t ticket, uint32_t kind)
+{
+    return (at >> 4) | ((bytes >> 4) << 12) | ((ticket & 3u) << 24) | (kind << 26);
+}
+
+__device__ __forceinline__ unsigned long long lds64(uint32_t addr)
+{
+    unsigned long long v;
+    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(addr));
+    return v;
+}
+
+// Ask for chunk c's index entries to be copied into the slot at shared address `slot`
+// (lanes 0..15 two sub-block lengths each, lanes 16 and 17 one offset each).  Nothing is
+// held in registers while the copies are in flight.
+__device__ __forceinline__ void fetch_index(const DevTensor& T, uint32_t c, uint32_t slot, uint32_t lane)
+{
+    if (c != kNone) {
+        if (lane < 16u) {
+            const char* src = reinterpret_cast<const char*>(T.sub_len + (uint64_t)c * kSubBlocks) + lane * 4u;
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(slot + lane * 4u), "l"(src) : "memory");
+        } else if (lane < 18u) {
+            const uint64_t* src = T.offsets + c + (lane - 16u);
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(slot + 64u + (lane - 16u) * 8u), "l"(src)
+                         : "memory");
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+__device__ __forceinline__ void issue_copy(const WarpCtx& cx, const DevTensor& T, Ready& r, uint64_t byte0, uint32_t lane)
+{
+    if (lane == 0)
+        bulk_load(cx.stage_addr + r.at(), reinterpret_cast<const char*>(T.stream) + byte0, r.bytes(),
+                  cx.bar + 8u * (r.ticket() & 1u));
+    r.meta |= 1u << 28;
+}
+
+// Bytes of the stream that decoding a chunk touches: from the 16-byte boundary below its
+// first bit to 13 bytes past its last (a window looks ahead), rounded up to 16.
+__device__ __forceinline__ void chunk_bytes(uint64_t off0, uint64_t off1, uint64_t& byte0, uint64_t& byte1)
+{
+    byte0 = (off0 >> 3) & ~15ull;
+    byte1 = ((off1 >> 3) + 13 + 15) & ~15ull;
+}
+
+// Chunk c's offsets have arrived in `slot`: check them, find a place in the ring next to
+// `prev` (the chunk decoded before this one, still undecoded), and start the bulk copy if
+// that place is free already.  All lanes compute the same values.
+__device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32_t stage_bytes, uint32_t* status,
+                                         uint32_t c, uint32_t slot, const Ready& prev, uint32_t lane)
+{
+    Ready r;
+    r.c = c;
+    r.meta = ready_meta(0, 0, 0, kSkip);
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncwarp();
+    if (c == kNone) return r;
+    const uint64_t off0 = lds64(slot + 64u), off1 = lds64(slot + 72u);
+    uint64_t byte0, byte1;
+    chunk_bytes(off0, off1, byte0, byte1);
+    if (off1 < off0 || off1 - off0 > 32ull * 65535ull || byte1 > T.stream_words * 4) {
+        if (lane == 0) atomicOr(status, kStatCorrupt);
+        return r;
+    }
+    const uint32_t sub = T.chunk_symbols / kSubBlocks;
+    const bool full = (uint64_t)(c + 1) * T.chunk_symbols <= T.n;
+    const uint32_t bytes = (uint32_t)(byte1 - byte0);
+    if (!full || (sub & 7u) || bytes > stage_bytes || cx.dead()) {
+        r.meta = ready_meta(0, 0, 0, kGeneral);
+        return r;
+    }
+    // ring placement: behind the previous chunk's bytes, else at the start if that does not
+    // overlap them, else at the start once the previous chunk has been decoded
+    uint32_t at = 0;
+    bool now = true;
+    if (prev.c != kNone && prev.kind() == kStaged) {
+        const uint32_t end = prev.at() + prev.bytes();
+        if (end + bytes <= stage_bytes) at = end;
+        else if (bytes > prev.at()) now = false;
+    }
+    r.meta = ready_meta(at, bytes, cx.state, kStaged);
+    cx.state++;
+    if (now) issue_copy(cx, T, r, byte0, lane);
+    else if (lane == 0)   // no room yet: at least bring the bytes into L2 while the previous chunk is decoded
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const char*>(T.stream) + byte0),
+                     "r"(bytes)
+                     : "memory");
+    return r;
+}
+
+// Any symbol count per lane, words fetched straight from global memory, one value at a
+// time: the ragged last chunk of a tensor, odd chunk sizes, chunks larger than the ring.
+// With G set (kB > 0 accumulators) the values are not stored but multiplied into the
+// matrix-vector products of the batch's tokens.
+template <int kB>
+__device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint32_t* status, const DevTensor& T,
+                                                     const GemvTensor* G, int sink, uint32_t c, uint32_t excl,
+                                                     uint32_t my_bits, uint32_t lane)
+{
+    const uint64_t chunk_first = (uint64_t)c * T.chunk_symbols;
+    const uint32_t m = (uint32_t)min((uint64_t)T.chunk_symbols, T.n - chunk_first);   // symbols in the chunk
+    const uint64_t pos = T.offsets[c] + excl;
+    const uint64_t word0 = pos >> 5;
+    GlobalWin r;
+    r.words = T.stream + word0;
+    r.count = word0 < T.stream_words ? T.stream_words - word0 : 0ull;
+    const uint32_t bit = (uint32_t)(pos & 31);
+    const uint32_t w0 = r.get(0), w1 = r.get(1);
+    r.hi = __funnelshift_l(w1, w0, bit);
+    r.lo = w1 << bit;
+    r.nb = 64 - (int)bit;
+    r.next = 2;
+    const bool oct = aux->oct != 0;
+    uint16_t* out = T.out + chunk_first;
+    // this lane's symbols: groups lane, lane + 32, ... of 8 consecutive symbols
+    for (uint32_t g = lane; g * 8u < m; g += kSubBlocks) {
+        const uint32_t end = min(g * 8u + 8u, m);
+        float acc[kB > 0 ? kB : 1];
+#pragma unroll
+        for (int b = 0; b < (kB > 0 ? kB : 1); ++b) acc[b] = 0.f;
+        uint32_t low = 0;                       // the even symbol of a nibble pair
+        for (uint32_t i = g * 8u; i < end; ++i) {
+            gwin_refill(r);
+            uint32_t e = kEscLen;
+            if (!oct) e = exp_lookup(lut_key(aux->expm, lane), ~r.hi);
+            if ((e & 0xffffu) > 32u) e = decode_by_range(aux, r.hi, status);
+            const uint32_t n = e & 0xffffu;
+            r.hi = __funnelshift_lc(r.lo, r.hi, n);
+            r.lo = __funnelshift_lc(0u, r.lo, n);
+            r.nb -= (int)n;
+            if (kB > 0) {
+                const uint32_t col = (uint32_t)((chunk_first + i) % G->cols);
+                const float v = __half2float(__ushort_as_half((uint16_t)(e >> 16)));
+#pragma unroll
+                for (int b = 0; b < kB; ++b)
+                    if ((uint32_t)b < G->batch)
+                        acc[b] = fmaf(v, __half2float(__ushort_as_half(__ldg(G->x + (uint64_t)b * G->cols + col))), acc[b]);
+            } else if (sink == kSinkBytes) {
+                reinterpret_cast<uint8_t*>(T.out)[chunk_first + i] = (uint8_t)(e >> 16);
+            } else if (sink == kSinkNibbles) {
+                // pairs never straddle a group of 8 and chunks hold an even number of symbols
+                if (i & 1u) reinterpret_cast<uint8_t*>(T.out)[(chunk_first + i) >> 1] = (uint8_t)(low | ((e >> 16) << 4));
+                else if (i + 1u == m) reinterpret_cast<uint8_t*>(T.out)[(chunk_first + i) >> 1] = (uint8_t)(e >> 16);
+                else low = (e >> 16) & 15u;
+            } else {
+                out[i] = (uint16_t)(e >> 16);
+            }
+        }
+        // a group of 8 lies inside one row (cols is a multiple of 8)
+        if (kB > 0) {
+            const uint32_t row = (uint32_t)((chunk_first + g * 8u) / G->cols);
+#pragma unroll
+            for (int b = 0; b < kB; ++b)
+                if ((uint32_t)b < G->batch) atomicAdd(G->y32 + (uint64_t)b * G->rows + row, acc[b]);
+        }
+    }
+    const uint64_t used = ((uint64_t)r.next << 5) - (uint64_t)r.nb - bit;
+    if (used != my_bits) atomicOr(status, kStatCorrupt);
+}
+
+// ------------------------------------------------------------------ what happens to decoded values
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// Plain decode: the 8 values of this lane's next group go to the output tensor.  A lane's
+// consecutive groups are 32 groups apart, so one call per lane writes 512 contiguous bytes.
+struct EmitStore {
+    uint4* dst;
+    __device__ __forceinline__ void operator()(uint4 v)
+    {
+        __stcs(dst, v);
+        dst += kSubBlocks;
+    }
+    __device__ __forceinline__ void finish() {}
+};
+
+// Integer output (the form the paper's decoder produces): the tables hold the symbols
+// themselves in their 16-bit value fields; a group of 8 leaves as 8 bytes ...
+struct EmitBytes {
+    uint2* dst;
+    __device__ __forceinline__ void operator()(uint4 v)
+    {
+        __stcs(dst, make_uint2(__byte_perm(v.x, v.y, 0x6420), __byte_perm(v.z, v.w, 0x6420)));
+        dst += kSubBlocks;
+    }
+};
+
+// ... or, for 4-bit symbols, as 4 bytes of two nibbles each, the earlier symbol low.
+struct EmitNibbles {
+    uint32_t* dst;
+    __device__ __forceinline__ void operator()(uint4 v)
+    {
+        const uint32_t a = __byte_perm(v.x, v.y, 0x6420), b = __byte_perm(v.z, v.w, 0x6420);   // s0..s3, s4..s7
+        const uint32_t ta = a | (a >> 4), tb = b | (b >> 4);                                   // bytes 0 and 2 hold the pairs
+        __stcs(dst, __byte_perm(ta, tb, 0x6420));
+        dst += kSubBlocks;
+    }
+};
+
+// Fused matrix-vector product: the 8 values are weights of one row of W (stored [rows, cols],
+// cols a multiple of 256, so the 32 lanes of a step stay inside one row) and meet the 8
+// matching entries of x of every token, staged in shared memory as fp16 token after token
+// (tokens beyond the batch are zeros); products and sums in fp32, one accumulator per token.
+// When the row ends the warp adds its lanes up and adds the results to the row's fp32
+// accumulators.
+template <int B>
+struct EmitDot {
+    uint32_t xaddr;       // shared-window address of x[0][col .. col + 8) for this lane's next group
+    uint32_t xlane;       // the same at the start of a row
+    uint32_t xstride;     // bytes from one token's x to the next
+    uint32_t left;        // steps left in the current row
+    uint32_t rs;          // steps per row (cols / 256)
+    float acc[B];
+    float* yrow;          // fp32 accumulator of the current row, first token
+    uint32_t rows, batch;
+    uint32_t lane;
+
+    __device__ __forceinline__ void flush()
+    {
+#pragma unroll
+        for (int b = 0; b < B; ++b) {
+            float v = acc[b];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+            if (lane == 0 && (uint32_t)b < batch) atomicAdd(yrow + (uint64_t)b * rows, v);
+            acc[b] = 0.f;
+        }
+        ++yrow;
+        left = rs;
+        xaddr = xlane;
+    }
+    // acc += w.lo * x.lo, then acc += w.hi * x.hi: fp16 operands, fp32 sum, one rounding per step
+    // (the product of two fp16 values is exact in fp32, so this is fmaf on the converted values).
+    static __device__ __forceinline__ void fma2(float& acc, uint32_t w, uint32_t x)
+    {
+        asm("{\n\t"
+            ".reg .b16 wl, wh, xl, xh;\n\t"
+            "mov.b32 {wl, wh}, %1;\n\t"
+            "mov.b32 {xl, xh}, %2;\n\t"
+            "fma.rn.f32.f16 %0, wl, xl, %0;\n\t"
+            "fma.rn.f32.f16 %0, wh, xh, %0;\n\t"
+            "}"
+            : "+f"(acc)
+            : "r"(w), "r"(x));
+    }
+    __device__ __forceinline__ void operator()(uint4 w)
+    {
+#pragma unroll
+        for (int b = 0; b < B; ++b) {
+            const uint4 x = lds128(xaddr + (uint32_t)b * xstride);
+            fma2(acc[b], w.x, x.x);
+            fma2(acc[b], w.y, x.y);
+            fma2(acc[b], w.z, x.z);
+            fma2(acc[b], w.w, x.w);
+        }
+        xaddr += 512u;
+        if (--left == 0u) flush();
+    }
+    __device__ __forceinline__ void finish()
+    {
+        if (left != rs) flush();     // the chunk ended inside a row
+    }
+};
+
+// 8-bit alphabets, eight symbols per turn.  G = 2, 3 (as 3 + 3 + 2), 4: groups of that many
+// lookups, each checked.  G = 8: two groups of four under one check, for streams whose groups
+// of four almost never fail; if either failed, both are done again one by one.
+template <int K, int G, class Emit>
+__device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status, LutKey key, Emit& emit, uint32_t sub)
+{
+    Cur r;
+    cur_init(r, start);
+    for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
+        uint32_t pk[4];
+        bool again = G == 4;
+        if (G == 8) {
+            uint32_t s0, s1;
+            group4(r, key, pk[0], pk[1], s0);
+            group4(r, key, pk[2], pk[3], s1);
+            if (__builtin_expect(((s0 | s1) & 0xffe0u) != 0u, 0)) {
+                // back over both: the position moved by s0 + s1, the words by one per flip of bit 5
+                const uint32_t p1 = r.pos - s1, p0 = p1 - s0;
+                const uint32_t steps = (((p0 ^ p1) >> 5) & 1u) + (((p1 ^ r.pos) >> 5) & 1u);
+                cur_init(r, (r.next - 8u - 4u * steps) * 8u + (p0 & 31u));
+                again = true;
+            }
+        }
+        if (G == 4 || G == 8) {
+            if (again) {
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    uint32_t s;
+                    group4(r, key, pk[2 * g], pk[2 * g + 1], s);
+                    if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_quad<K>(r, status, key, s, pk[2 * g], pk[2 * g + 1]);
+                }
+            }
+        } else if (G == 3) {
+            uint32_t s, a2, b0;
+            group3<false>(r, key, pk[0], a2, s);
+            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_triple<K, false>(r, status, key, s, pk[0], a2);
+            group3<true>(r, key, b0, pk[2], s);
+            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_triple<K, true>(r, status, key, s, b0, pk[2]);
+            pk[1] = __byte_perm(a2, b0, 0x7632);
+            group2(r, key, pk[3], s);
+            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_pair<K>(r, status, key, s, pk[3]);
+        } else {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                uint32_t s;
+                group2(r, key, pk[g], s);
+                if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_pair<K>(r, status, key, s, pk[g]);
+            }
+        }
+        emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
+    }
+    return cur_bit_addr(r);
+}
+
+// 4-bit alphabets: eight symbols per lookup.
+template <int K, class Emit>
+__device__ __forceinline__ uint32_t rows_oct(uint32_t start, uint32_t* status, Emit& emit, uint32_t sub)
+{
+    Win r;
+    win_init<false>(r, (start >> 5) << 2, start & 31u);
+    for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
+        win_refill<false>(r);
+        const uint32_t idx = r.hi >> (32 - K);
+        uint4 v = *reinterpret_cast<const uint4*>(smem + idx * 16u);
+        const uint32_t n = *(smem + (16u << K) + idx);
+        if (__builtin_expect(n == 0u, 0)) v = repair_oct<K>(r, status);
+        else win_skip(r, n);
+        emit(v);
+    }
+    return r.next * 8u - (uint32_t)win_valid_bits(r.k);
+}
+
+// The whole sub-block of a lane in the mode build_tables_kernel chose for the tensor;
+// returns where the lane stands afterwards.
+template <int K, class Emit>
+__device__ __forceinline__ uint32_t rows_any(const DecodeAux* aux, uint32_t start, uint32_t* status, Emit& emit, uint32_t sub,
+                                             uint32_t lane)
+{
+    if (aux->oct) return rows_oct<K>(start, status, emit, sub);
+    const LutKey key = lut_key(aux->expm, lane);
+    switch (aux->group) {
+        case 8u: return rows_single<K, 8>(start, status, key, emit, sub);
+        case 4u: return rows_single<K, 4>(start, status, key, emit, sub);
+        case 3u: return rows_single<K, 3>(start, status, key, emit, sub);
+        default: return rows_single<K, 2>(start, status, key, emit, sub);
+    }
+}
+
+// What decode_start leaves for decode_finish: where this lane begins and must end.
+struct Lane {
+    uint32_t start, end;       // staged: shared-window bit addresses; general: bits before this lane's, and its count
+    uint32_t kind;
+};
+
+// First half of decoding chunk r (its index slot is about to be reused): lane positions by
+// a warp prefix sum over the sub-block lengths, checked against the offsets.
+template <int K>
+__device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status, const Ready& r, uint32_t slot,
+                                             uint32_t lane)
+{
+    Lane L;
+    L.start = L.end = 0;
+    L.kind = r.c == kNone ? (uint32_t)kSkip : r.kind();
+    if (L.kind == kSkip) return L;
+    const uint32_t pair = lds32(slot + (lane >> 1) * 4u);
+    const uint32_t bits = (lane & 1u) ? pair >> 16 : pair & 0xffffu;
+    uint32_t incl = bits;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= (uint32_t)d) incl += t;
+    }
+    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+    const uint64_t off0 = lds64(slot + 64u), off1 = lds64(slot + 72u);
+    if (off1 - off0 != (uint64_t)total) {       // the recorded lengths do not add up to the chunk
+        if (lane == 0) atomicOr(status, kStatCorrupt);
+        L.kind = kSkip;
+        return L;
+    }
+    const uint32_t excl = incl - bits;
+    if (L.kind == kGeneral) {
+        L.start = excl;
+        L.end = bits;
+    } else {
+        const uint32_t byte0_bits = (uint32_t)off0 & ~127u;    // bit offset of the copied bytes' start, modulo 2^32
+        L.start = (cx.stage_addr + r.at()) * 8u + ((uint32_t)off0 - byte0_bits) + excl;
+        L.end = L.start + bits;
+    }
+    return L;
+}
+
+template <int K, int kSink>
+__device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Ready& r, Lane L, uint32_t lane)
+{
+    constexpr int kBatch = kGemvBatchOf<kSink>;
+    constexpr bool kGemv = kBatch > 0;
+    if (L.kind == kSkip) return;
+    const DevTensor& T = *tensor_ptr<K>();
+    const GemvTensor* G = kGemv ? gemv_ptr<K>() : nullptr;
+    if (L.kind == kStaged) {
+        if (!r.issued()) issue_copy(cx, T, r, (T.offsets[r.c] >> 3) & ~15ull, lane);
+        bool ok = mbar_wait(cx.bar + 8u * (r.ticket() & 1u), (r.ticket() >> 1) & 1u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) {
+            if (lane == 0) atomicOr(status, kStatTimeout);
+            cx.state |= 1u << 31;
+            // fall back to global memory: bits of the chunk before this lane's, and this lane's count
+            const uint32_t first = __shfl_sync(0xffffffffu, L.start, 0);
+            L.kind = kGeneral;
+            L.end -= L.start;
+            L.start -= first;
+        }
+    }
+    if (L.kind == kGeneral) {
+        decode_chunk_general<kBatch>(aux_ptr<K>(), status, T, G, kSink, r.c, L.start, L.end, lane);
+        return;
+    }
+    const uint32_t sub = T.chunk_symbols / kSubBlocks;
+    uint32_t stood;            // where the lane stands after its sub-block
+    if (kGemv) {
+        // the chunk starts gs0 steps of 256 weights into the matrix; a row is rs steps long
+        const uint32_t rs = G->cols >> 8;
+        const uint32_t gs0 = (uint32_t)(((uint64_t)r.c * T.chunk_symbols) >> 8);
+        const uint32_t row0 = gs0 / rs, k0 = gs0 - row0 * rs;
+        EmitDot<kGemv ? kBatch : 1> em;
+        em.lane = lane;
+        em.rs = rs;
+        em.left = rs - k0;
+        em.xlane = kSmemBase + kGemvX<K> + lane * 16u;
+        em.xaddr = em.xlane + k0 * 512u;
+        em.xstride = G->cols * 2u;
+#pragma unroll
+        for (int b = 0; b < (kGemv ? kBatch : 1); ++b) em.acc[b] = 0.f;
+        em.yrow = G->y32 + row0;
+        em.rows = G->rows;
+        em.batch = G->batch;
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
+        em.finish();
+    } else if (kSink == kSinkBytes) {
+        EmitBytes em;
+        em.dst = reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(T.out) + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
+    } else if (kSink == kSinkNibbles) {
+        EmitNibbles em;
+        em.dst = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(T.out) + (((uint64_t)r.c * T.chunk_symbols) >> 1) +
+                                             lane * 4u);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
+    } else {
+        EmitStore em;
+        em.dst = reinterpret_cast<uint4*>(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
+        em.finish();
+    }
+    // the lane must stand exactly at the end of its sub-block
+    if (stood != L.end) atomicOr(status, kStatCorrupt);
+    __syncwarp();   // all lanes are done with these bytes before the ring reuses them
+}
+
+}  // namespace
+}  // namespace entro
