@@ -231,13 +231,14 @@ entro_status entro_decode_symbols_batched(const entro_tensor_desc *descs_host, i
 typedef struct {
     const uint32_t *stream_host;  /* stream_words words (pinned memory for full speed) */
     const void *index_host;       /* entro_index_bytes bytes */
-    void *out_fp16_host;          /* n fp16 values */
+    void *out_fp16_host;          /* n fp16 values, or NULL: the result stays in out_fp16_dev only */
 } entro_host_io;
 
 /*
  * End-to-end form with host buffers: for every tensor, copy stream and index from
  * io_host[i] to the device buffers named in descs_host[i], decode + dequantise, and copy
- * the fp16 result back to io_host[i].out_fp16_host.  The work is ordered after what
+ * the fp16 result back to io_host[i].out_fp16_host (where that is NULL the result is left
+ * on the device: loading a compressed model from host memory).  The work is ordered after what
  * cuda_stream already holds; inside the call, uploads, decodes and downloads of different
  * groups of tensors overlap on two copy streams of the library's own.  Returns after
  * everything has completed (synchronises cuda_stream).

@@ -478,7 +478,7 @@ extern "C" entro_status entro_decode_dequant_batched_host(const entro_tensor_des
     uint64_t out_bytes = 0;
     for (int i = 0; i < ntensors; ++i) {
         if (!descs[i].n) continue;
-        if (!io[i].stream_host || !io[i].index_host || !io[i].out_fp16_host) return ENTRO_ERR_INVALID_ARG;
+        if (!io[i].stream_host || !io[i].index_host) return ENTRO_ERR_INVALID_ARG;
         entro_status st = validate_desc(descs[i]);
         if (st != ENTRO_OK) return st;
         out_bytes += descs[i].n * 2;
@@ -513,7 +513,7 @@ extern "C" entro_status entro_decode_dequant_batched_host(const entro_tensor_des
         ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_out, ws->ev_dec[group], 0));
         for (int i = first; i < last; ++i) {
             const entro_tensor_desc& d = descs[i];
-            if (!d.n) continue;
+            if (!d.n || !io[i].out_fp16_host) continue;     // no host buffer: the result stays on the device
             ENTRO_CUDA(cudaMemcpyAsync(io[i].out_fp16_host, d.out_fp16_dev, d.n * 2, cudaMemcpyDeviceToHost, ws->copy_out));
         }
         first = last;

@@ -354,6 +354,15 @@ def test_host_buffer_entry_point():
     E.entro_decode_dequant_batched_host(descs, io)
     assert np.array_equal(h_out.numpy().view(np.uint16), expected_out(c))
     assert_status_ok()
+    # without a host output buffer the result is left on the device
+    d_out.zero_()
+    d_stream.zero_()
+    h_out.zero_()
+    io = (E.HostIO * 1)(E.HostIO(h_stream.data_ptr(), h_index.data_ptr(), None))
+    E.entro_decode_dequant_batched_host(descs, io)
+    assert np.array_equal(d_out.cpu().numpy().view(np.uint16), expected_out(c))
+    assert not h_out.any()
+    assert_status_ok()
 
 
 # ----------------------------------------------------------------------------- malformed input
