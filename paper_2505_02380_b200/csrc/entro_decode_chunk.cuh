@@ -264,38 +264,59 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     return v;
 }
 
+// Where a lane's groups go in the output: group after group `stride` bytes apart (the 32
+// lanes' groups of one step are contiguous), from `base`.  The address is formed by one
+// multiply-add on the FMA pipe (the integer pipe is the busy one), and the byte offset
+// doubles as the loop counter of the lane's sub-block.
+struct OutCursor {
+    const void* base;
+    uint32_t off, end;
+    __device__ __forceinline__ void start(void* lane_first, uint32_t steps, uint32_t stride)
+    {
+        base = lane_first;
+        off = 0;
+        end = steps * stride;
+    }
+    __device__ __forceinline__ bool more() const { return off != end; }
+    __device__ __forceinline__ void* next(uint32_t stride)
+    {
+        unsigned long long a;
+        asm("mad.wide.u32 %0, %1, 1, %2;" : "=l"(a) : "r"(off), "l"(base));
+        off += stride;
+        return reinterpret_cast<void*>(a);
+    }
+};
+
 // Plain decode: the 8 values of this lane's next group go to the output tensor.  A lane's
 // consecutive groups are 32 groups apart, so one call per lane writes 512 contiguous bytes.
 struct EmitStore {
-    uint4* dst;
-    __device__ __forceinline__ void operator()(uint4 v)
-    {
-        __stcs(dst, v);
-        dst += kSubBlocks;
-    }
+    OutCursor out;
+    __device__ __forceinline__ bool more() const { return out.more(); }
+    __device__ __forceinline__ void operator()(uint4 v) { __stcs(static_cast<uint4*>(out.next(16u * kSubBlocks)), v); }
     __device__ __forceinline__ void finish() {}
 };
 
 // Integer output (the form the paper's decoder produces): the tables hold the symbols
 // themselves in their 16-bit value fields; a group of 8 leaves as 8 bytes ...
 struct EmitBytes {
-    uint2* dst;
+    OutCursor out;
+    __device__ __forceinline__ bool more() const { return out.more(); }
     __device__ __forceinline__ void operator()(uint4 v)
     {
-        __stcs(dst, make_uint2(__byte_perm(v.x, v.y, 0x6420), __byte_perm(v.z, v.w, 0x6420)));
-        dst += kSubBlocks;
+        __stcs(static_cast<uint2*>(out.next(8u * kSubBlocks)),
+               make_uint2(__byte_perm(v.x, v.y, 0x6420), __byte_perm(v.z, v.w, 0x6420)));
     }
 };
 
 // ... or, for 4-bit symbols, as 4 bytes of two nibbles each, the earlier symbol low.
 struct EmitNibbles {
-    uint32_t* dst;
+    OutCursor out;
+    __device__ __forceinline__ bool more() const { return out.more(); }
     __device__ __forceinline__ void operator()(uint4 v)
     {
         const uint32_t a = __byte_perm(v.x, v.y, 0x6420), b = __byte_perm(v.z, v.w, 0x6420);   // s0..s3, s4..s7
         const uint32_t ta = a | (a >> 4), tb = b | (b >> 4);                                   // bytes 0 and 2 hold the pairs
-        __stcs(dst, __byte_perm(ta, tb, 0x6420));
-        dst += kSubBlocks;
+        __stcs(static_cast<uint32_t*>(out.next(4u * kSubBlocks)), __byte_perm(ta, tb, 0x6420));
     }
 };
 
@@ -316,6 +337,8 @@ struct EmitDot {
     float* yrow;          // fp32 accumulator of the current row, first token
     uint32_t rows, batch;
     uint32_t lane;
+    uint32_t todo;        // groups left in the lane's sub-block
+    __device__ __forceinline__ bool more() const { return todo != 0u; }
 
     __device__ __forceinline__ void flush()
     {
@@ -356,6 +379,7 @@ struct EmitDot {
             fma2(acc[b], w.w, x.w);
         }
         xaddr += 512u;
+        --todo;
         if (--left == 0u) flush();
     }
     __device__ __forceinline__ void finish()
@@ -368,11 +392,11 @@ struct EmitDot {
 // lookups, each checked.  G = 8: two groups of four under one check, for streams whose groups
 // of four almost never fail; if either failed, both are done again one by one.
 template <int K, int G, class Emit>
-__device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status, LutKey key, Emit& emit, uint32_t sub)
+__device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status, LutKey key, Emit& emit)
 {
     Cur r;
     cur_init(r, start);
-    for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
+    while (emit.more()) {
         uint32_t pk[4];
         bool again = G == 4;
         if (G == 8) {
@@ -420,11 +444,11 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
 
 // 4-bit alphabets: eight symbols per lookup.
 template <int K, class Emit>
-__device__ __forceinline__ uint32_t rows_oct(uint32_t start, uint32_t* status, Emit& emit, uint32_t sub)
+__device__ __forceinline__ uint32_t rows_oct(uint32_t start, uint32_t* status, Emit& emit)
 {
     Win r;
     win_init<false>(r, (start >> 5) << 2, start & 31u);
-    for (uint32_t t0 = 0; t0 < sub; t0 += 8) {
+    while (emit.more()) {
         win_refill<false>(r);
         const uint32_t idx = r.hi >> (32 - K);
         uint4 v = *reinterpret_cast<const uint4*>(smem + idx * 16u);
@@ -439,16 +463,16 @@ __device__ __forceinline__ uint32_t rows_oct(uint32_t start, uint32_t* status, E
 // The whole sub-block of a lane in the mode build_tables_kernel chose for the tensor;
 // returns where the lane stands afterwards.
 template <int K, class Emit>
-__device__ __forceinline__ uint32_t rows_any(const DecodeAux* aux, uint32_t start, uint32_t* status, Emit& emit, uint32_t sub,
+__device__ __forceinline__ uint32_t rows_any(const DecodeAux* aux, uint32_t start, uint32_t* status, Emit& emit,
                                              uint32_t lane)
 {
-    if (aux->oct) return rows_oct<K>(start, status, emit, sub);
+    if (aux->oct) return rows_oct<K>(start, status, emit);
     const LutKey key = lut_key(aux->expm, lane);
     switch (aux->group) {
-        case 8u: return rows_single<K, 8>(start, status, key, emit, sub);
-        case 4u: return rows_single<K, 4>(start, status, key, emit, sub);
-        case 3u: return rows_single<K, 3>(start, status, key, emit, sub);
-        default: return rows_single<K, 2>(start, status, key, emit, sub);
+        case 8u: return rows_single<K, 8>(start, status, key, emit);
+        case 4u: return rows_single<K, 4>(start, status, key, emit);
+        case 3u: return rows_single<K, 3>(start, status, key, emit);
+        default: return rows_single<K, 2>(start, status, key, emit);
     }
 }
 
@@ -540,21 +564,22 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         em.yrow = G->y32 + row0;
         em.rows = G->rows;
         em.batch = G->batch;
-        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
+        em.todo = sub >> 3;
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
         em.finish();
     } else if (kSink == kSinkBytes) {
         EmitBytes em;
-        em.dst = reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(T.out) + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
-        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
+        em.out.start(reinterpret_cast<uint8_t*>(T.out) + (uint64_t)r.c * T.chunk_symbols + lane * 8u, sub >> 3, 8u * kSubBlocks);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
     } else if (kSink == kSinkNibbles) {
         EmitNibbles em;
-        em.dst = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(T.out) + (((uint64_t)r.c * T.chunk_symbols) >> 1) +
-                                             lane * 4u);
-        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
+        em.out.start(reinterpret_cast<uint8_t*>(T.out) + (((uint64_t)r.c * T.chunk_symbols) >> 1) + lane * 4u, sub >> 3,
+                     4u * kSubBlocks);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
     } else {
         EmitStore em;
-        em.dst = reinterpret_cast<uint4*>(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u);
-        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, sub, lane);
+        em.out.start(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u, sub >> 3, 16u * kSubBlocks);
+        stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
         em.finish();
     }
     // the lane must stand exactly at the end of its sub-block
