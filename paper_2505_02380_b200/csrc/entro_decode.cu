@@ -387,7 +387,7 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     TensorTables* dtables = reinterpret_cast<TensorTables*>(base + upload_bytes);
     ENTRO_CUDA(cudaMemcpyAsync(dt, ht, upload_bytes, cudaMemcpyHostToDevice, s));
     mark_pinned_in_use(ws, s);
-    build_tables_kernel<<<dim3((unsigned)live, kTableSlices), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control, nullptr);
+    build_tables_kernel<<<dim3((unsigned)live, table_slices(live, ws->sm_count)), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control, nullptr);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     return launch_decode_any(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, s, nullptr, sink);
@@ -645,7 +645,7 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
     TensorTables* dtables = reinterpret_cast<TensorTables*>(base + upload_bytes);
     ENTRO_CUDA(cudaMemcpyAsync(dt, ht, upload_bytes, cudaMemcpyHostToDevice, s));
     mark_pinned_in_use(ws, s);
-    build_tables_kernel<<<dim3((unsigned)ntensors, kTableSlices), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control, dg);
+    build_tables_kernel<<<dim3((unsigned)ntensors, table_slices(ntensors, ws->sm_count)), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control, dg);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     entro_status st = launch_decode_any(ws, cfg, dt, ntensors, ditems, (uint32_t)items, dtables, s, dg, kSinkGemv,
@@ -788,7 +788,7 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
     static_upload_kernel<<<1, 256, 0, s>>>(up, sc);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
-    build_tables_kernel<<<dim3((unsigned)live, kTableSlices), 256, 0, s>>>(sc->tensors, cfg.lut_bits, sc->tables, sc->control, nullptr);
+    build_tables_kernel<<<dim3((unsigned)live, table_slices(live, sd->sm_count)), 256, 0, s>>>(sc->tensors, cfg.lut_bits, sc->tables, sc->control, nullptr);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     // launch_decode reads only these fields of a workspace; no timing records are taken here

@@ -24,9 +24,16 @@ __device__ __forceinline__ uint32_t range_decode(const DecodeAux& aux, uint32_t 
 }
 
 // One block per tensor.
-// The grid is (tensors, kTableSlices): every block of a tensor works out the small things
-// for itself and fills its share of the tables' entries.
-constexpr unsigned kTableSlices = 8;
+// The grid is (tensors, slices): every block of a tensor works out the small things for
+// itself and fills its share of the tables' entries.  Slicing pays when a launch has few
+// tensors (one layer: the 4096-entry eight-symbol table took one block 62 us); with a whole
+// model in the launch the tensors already fill the GPU and more blocks only repeat the
+// small things.
+inline unsigned table_slices(int tensors, int sm_count)
+{
+    const int s = 2 * sm_count / (tensors > 0 ? tensors : 1);
+    return (unsigned)(s < 1 ? 1 : s > 8 ? 8 : s);
+}
 __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __restrict__ tensors, int lut_bits,
                                                            TensorTables* __restrict__ tables,
                                                            uint32_t* __restrict__ control,
