@@ -407,7 +407,7 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
                 // back over both: the position moved by s0 + s1, the words by one per flip of bit 5
                 const uint32_t p1 = r.pos - s1, p0 = p1 - s0;
                 const uint32_t steps = (((p0 ^ p1) >> 5) & 1u) + (((p1 ^ r.pos) >> 5) & 1u);
-                cur_init(r, (r.next - 8u - 4u * steps) * 8u + (p0 & 31u));
+                cur_init(r, (r.next - kCurBytes - 4u * steps) * 8u + (p0 & 31u));
                 again = true;
             }
         }

@@ -129,27 +129,31 @@ __device__ __forceinline__ uint32_t decode_by_range(const DecodeAux* aux, uint32
     return ((uint32_t)aux->val[sym] << 16) | len;
 }
 
-// Reader of the grouped lookups of 8-bit alphabets: two consecutive stream words
+// Reader of the grouped lookups of 8-bit alphabets: three consecutive stream words
 // (complemented) in registers and a bit position whose low five bits say where in w0 the
 // next code starts.  Only those five bits and bit 5 (has a word boundary been crossed?) are
-// ever used, so the upper bits of pos may hold anything.
+// ever used, so the upper bits of pos may hold anything.  A group reads w0 and w1 only; w2
+// is held ahead so that the word read from shared memory when a boundary is crossed is not
+// needed before the boundary after it (the read is off the chain from group to group).
 struct Cur {
-    uint32_t w0, w1;
+    uint32_t w0, w1, w2;
     uint32_t pos;
-    uint32_t next;            // shared-window address of the word after w1
+    uint32_t next;            // shared-window address of the word after w2
 };
+constexpr uint32_t kCurBytes = 12;   // bytes from w0's address to next
 
 __device__ __forceinline__ void cur_init(Cur& c, uint32_t bit_addr)
 {
     const uint32_t a = (bit_addr >> 5) << 2;
     c.w0 = ~lds32(a);
     c.w1 = ~lds32(a + 4);
-    c.next = a + 8;
+    c.w2 = ~lds32(a + 8);
+    c.next = a + kCurBytes;
     c.pos = bit_addr;
 }
 
 // Shared-window bit address the reader stands at.
-__device__ __forceinline__ uint32_t cur_bit_addr(const Cur& c) { return (c.next - 8u) * 8u + (c.pos & 31u); }
+__device__ __forceinline__ uint32_t cur_bit_addr(const Cur& c) { return (c.next - kCurBytes) * 8u + (c.pos & 31u); }
 
 // One group of lookups, hand-scheduled.  The group sees the 32 bits that start at the
 // reader's position (one funnel shift of the two words) and nothing behind them: a lookup
@@ -160,14 +164,15 @@ __device__ __forceinline__ uint32_t cur_bit_addr(const Cur& c) { return (c.next 
 // of the G entries: the group stands iff (s & 0xffe0) == 0, that is, every cell was resolved
 // (an unresolved one adds 64) and fewer than 32 bits were used, so all codes did end inside
 // the 32 bits.  Then the position moves on by s and, if that crosses into the next word
-// (bit 5 of the position flips), w1 becomes w0 and one new word is pulled in, predicated.
+// (bit 5 of the position flips), the words move up by one and a new third word is pulled
+// in, predicated.
 // If the group does not stand the caller repairs it from rewind_group, which needs only
 // pos, next and s.
 #define ENTRO_LOOKUP(dst, win)                       \
     "cvt.rz.f32.u32 f, " win ";\n\t"                  \
     "mov.b32 a, f;\n\t"                               \
     "shr.u32 a, a, 12;\n\t"                           \
-    "lop3.b32 a, a, %8, %7, 0xEA;\n\t"                \
+    "lop3.b32 a, a, %9, %8, 0xEA;\n\t"                \
     "ld.shared.b32 " dst ", [a+1024];\n\t"
 #define ENTRO_OPEN                                   \
     "shf.l.wrap.b32 h, %1, %0, %2;\n\t"
@@ -178,9 +183,10 @@ __device__ __forceinline__ uint32_t cur_bit_addr(const Cur& c) { return (c.next 
     "and.b32 a, a, 32;\n\t"                           \
     "setp.ne.u32 p, a, 0;\n\t"                        \
     "@p mov.b32 %0, %1;\n\t"                          \
+    "@p mov.b32 %1, %7;\n\t"                          \
     "@p ld.shared.b32 t, [%3];\n\t"                   \
     "@p add.u32 %3, %3, 4;\n\t"                       \
-    "@p not.b32 %1, t;\n\t"
+    "@p not.b32 %7, t;\n\t"
 
 __device__ __forceinline__ void group4(Cur& c, LutKey key, uint32_t& pk0, uint32_t& pk1, uint32_t& s)
 {
@@ -197,7 +203,7 @@ __device__ __forceinline__ void group4(Cur& c, LutKey key, uint32_t& pk0, uint32
         "add.u32 %6, %6, e3;\n\t"
         "prmt.b32 %4, e0, e1, 0x7632;\n\t"
         "prmt.b32 %5, e2, e3, 0x7632;\n\t" ENTRO_MOVE_ON "}"
-        : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk0), "=&r"(pk1), "=&r"(s)
+        : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk0), "=&r"(pk1), "=&r"(s), "+r"(c.w2)
         : "r"(key.lane), "r"(key.mask));
 }
 
@@ -213,7 +219,7 @@ __device__ __forceinline__ void group2(Cur& c, LutKey key, uint32_t& pk0, uint32
         "add.u32 %6, e0, e1;\n\t"
         "prmt.b32 %4, e0, e1, 0x7632;\n\t"
         "mov.b32 %5, 0;\n\t" ENTRO_MOVE_ON "}"
-        : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk0), "=&r"(unused), "=&r"(s)
+        : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk0), "=&r"(unused), "=&r"(s), "+r"(c.w2)
         : "r"(key.lane), "r"(key.mask));
 }
 // Three lookups, for the streams whose groups of four would too often need 32 bits or more.
@@ -234,7 +240,7 @@ __device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint
             "add.u32 %6, e0, e1;\n\t"
             "add.u32 %6, %6, %5;\n\t"
             "prmt.b32 %4, e0, e1, 0x7632;\n\t" ENTRO_MOVE_ON "}"
-            : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s)
+            : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s), "+r"(c.w2)
             : "r"(key.lane), "r"(key.mask));
     else
         asm volatile(
@@ -247,7 +253,7 @@ __device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint
             "add.u32 %6, %4, e1;\n\t"
             "add.u32 %6, %6, e2;\n\t"
             "prmt.b32 %5, e1, e2, 0x7632;\n\t" ENTRO_MOVE_ON "}"
-            : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s)
+            : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s), "+r"(c.w2)
             : "r"(key.lane), "r"(key.mask));
 }
 #undef ENTRO_LOOKUP
@@ -280,7 +286,7 @@ __device__ __forceinline__ uint32_t rewind_group(const Cur& c, uint32_t s)
 {
     const uint32_t before = c.pos - s;
     const uint32_t crossed = ((before ^ c.pos) >> 5) & 1u;
-    return (c.next - 8u - 4u * crossed) * 8u + (before & 31u);
+    return (c.next - kCurBytes - 4u * crossed) * 8u + (before & 31u);
 }
 
 // Repair of a group of two symbols that did not stand (kept inline: a call here would park
