@@ -185,6 +185,34 @@ def test_decode_every_group_size(sigma_levels, foreign):
     assert_status_ok()
 
 
+@pytest.mark.parametrize("sigma_levels,lo,hi", [(0.3, 1.0, 1.3), (0.5, 1.32, 1.74), (0.6, 1.32, 1.74), (1.5, 1.8, 4.0)])
+def test_decode_four_bit_modes(sigma_levels, lo, hi):
+    """4-bit alphabets are decoded eight symbols per lookup while eight codes usually fit
+    the table's window (up to 1.31 bit per symbol) and one by one above.  Symbols are drawn
+    directly as rounded Gaussians; the bit rate is checked so that the cases lie on both
+    sides of that limit, close to it and far from it; output as fp16 values, and as packed
+    nibbles (the integer sink of the same loops)."""
+    chunk, n = 8192, 19 * 8192 + 4101
+    rng = np.random.default_rng(int(sigma_levels * 100))
+    q = np.clip(np.rint(rng.normal(8.0, sigma_levels, n)), 0, 15).astype(np.uint8)
+    q[:: 997] = rng.integers(0, 16, q[:: 997].size)          # every symbol occurs, some codes are long
+    ln = oracle.huffman_lengths(np.bincount(q, minlength=16).tolist())
+    cd = oracle.canonical_codes(ln)
+    enc = oracle.encode(q, ln, cd, chunk)
+    assert lo <= int(enc.offsets[-1]) / n <= hi
+    cb = E.Codebook.from_lengths(ln.tolist(), cd.tolist())
+    s, ix = to_dev_stream(enc.stream), to_dev_index(enc)
+    out = E.entro_decode_dequant(s, ix, n, chunk, cb, 0.0625, 8)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.dequant(q, 0.0625, 8))
+    packed = torch.full(((n + 1) // 2,), 0xEE, dtype=torch.uint8, device="cuda")
+    E.entro_decode_symbols_batched([E.make_desc_bytes(s, ix, n, chunk, cb, packed)], True)
+    torch.cuda.synchronize()
+    q2 = np.concatenate([q, np.zeros(n & 1, dtype=np.uint8)])
+    assert np.array_equal(packed.cpu().numpy(), (q2[0::2] | (q2[1::2] << 4)).astype(np.uint8))
+    assert_status_ok()
+
+
 @pytest.mark.parametrize("bits,chunk,packed", [(8, 4096, False), (4, 8192, False), (4, 8192, True), (4, 1024, True),
                                                (8, 96, False), (4, 64, True)])
 def test_decode_to_integer_symbols(bits, chunk, packed):
