@@ -138,10 +138,19 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                 for (uint32_t i = threadIdx.x; i < (uint32_t)kExpEntriesMin; i += blockDim.x) s3[i] = __ldg(tt->exp_small + i);
             } else {
                 // cell-major copies, 64 KB in all: word w holds cell w / copies
-                uint32_t* s1 = reinterpret_cast<uint32_t*>(smem);
                 const uint32_t shift = 9u - __ldg(&tt->aux.expm);       // log2 of the number of copies
-                for (uint32_t w = threadIdx.x; w < (uint32_t)kExpEntriesMax; w += blockDim.x)
-                    s1[w] = __ldg(tt->exp_lut() + (w >> shift));
+                if (shift >= 2u) {
+                    // four or more copies: the four words of a 16-byte store belong to one cell
+                    uint4* s4 = reinterpret_cast<uint4*>(smem);
+                    for (uint32_t q = threadIdx.x; q < (uint32_t)kExpEntriesMax / 4u; q += blockDim.x) {
+                        const uint32_t v = __ldg(tt->exp_lut() + ((4u * q) >> shift));
+                        s4[q] = make_uint4(v, v, v, v);
+                    }
+                } else {
+                    uint32_t* s1 = reinterpret_cast<uint32_t*>(smem);
+                    for (uint32_t w = threadIdx.x; w < (uint32_t)kExpEntriesMax; w += blockDim.x)
+                        s1[w] = __ldg(tt->exp_lut() + (w >> shift));
+                }
             }
             __syncthreads();
         }
