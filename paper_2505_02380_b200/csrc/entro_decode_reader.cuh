@@ -1,4 +1,4 @@
-// Bit readers and table lookups of the decode kernel: the 64-bit window, the two-word
+// Bit readers and table lookups of the decode kernel: the 64-bit window, the three-word
 // reader of the grouped lookups, the hand-scheduled groups and their repairs.
 // Included by entro_decode.cu only.
 #pragma once
@@ -156,7 +156,7 @@ __device__ __forceinline__ void cur_init(Cur& c, uint32_t bit_addr)
 __device__ __forceinline__ uint32_t cur_bit_addr(const Cur& c) { return (c.next - kCurBytes) * 8u + (c.pos & 31u); }
 
 // One group of lookups, hand-scheduled.  The group sees the 32 bits that start at the
-// reader's position (one funnel shift of the two words) and nothing behind them: a lookup
+// reader's position (one funnel shift of the first two words) and nothing behind them: a lookup
 // reads them shifted left by the lengths found before it (a funnel shift uses the low five
 // bits of its count), zeros moving in from the right.  Those
 // zeros cannot mislead a lookup whose code ends inside the 32 bits: a cell is resolved only
