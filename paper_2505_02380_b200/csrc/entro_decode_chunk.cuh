@@ -166,14 +166,18 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32
         r.meta = ready_meta(0, 0, 0, kGeneral);
         return r;
     }
-    // ring placement: behind the previous chunk's bytes, else at the start if that does not
-    // overlap them, else at the start once the previous chunk has been decoded
+    // ring placement: at the other end of the ring from the previous chunk's bytes (chunks
+    // alternate between the start and the end, so two chunks that fit together never wait for
+    // one another, whatever their sizes), else at the start once the previous chunk has been
+    // decoded
     uint32_t at = 0;
     bool now = true;
     if (prev.c != kNone && prev.kind() == kStaged) {
-        const uint32_t end = prev.at() + prev.bytes();
-        if (end + bytes <= stage_bytes) at = end;
-        else if (bytes > prev.at()) now = false;
+        const uint32_t p_at = prev.at(), p_end = p_at + prev.bytes();
+        const uint32_t top = stage_bytes - bytes;          // a multiple of 16, as both are
+        if (bytes <= p_at) at = 0;
+        else if (top >= p_end) at = top;
+        else now = false;
     }
     r.meta = ready_meta(at, bytes, cx.state, kStaged);
     cx.state++;
