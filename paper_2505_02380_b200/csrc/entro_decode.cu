@@ -334,6 +334,7 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, ItemPlan& plan, DevTensor& 
     t.sub_len = reinterpret_cast<const uint16_t*>(t.offsets + nc + 1);
     t.out = static_cast<uint16_t*>(d.out_fp16_dev);
     t.stream_words = d.stream_words;
+    t.last_bit = d.stream_words * 4 >= 28 ? (d.stream_words * 4 - 28) * 8 + 7 : 0;
     t.n = d.n;
     t.chunk_symbols = d.chunk_symbols;
     t.n_chunks = (uint32_t)nc;
@@ -348,7 +349,8 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, ItemPlan& plan, DevTensor& 
     t.item_chunks = per_item;
     plan.seen += nc;
     t.raw_symbols = 0;
-    t.pad = 0;
+    t.full_chunks = (uint32_t)(d.n / d.chunk_symbols);
+    t.pad[0] = t.pad[1] = 0;
     for (int j = 0; j < ENTRO_MAX_SYMBOLS; ++j) t.len[j] = j < d.cb.nsym ? d.cb.len[j] : 0;
     return (nc + t.item_chunks - 1) / t.item_chunks;
 }

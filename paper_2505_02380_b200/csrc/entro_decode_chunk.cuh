@@ -111,15 +111,11 @@ __device__ __forceinline__ unsigned long long lds64(uint32_t addr)
 // held in registers while the copies are in flight.
 __device__ __forceinline__ void fetch_index(const DevTensor& T, uint32_t c, uint32_t slot, uint32_t lane)
 {
-    if (c != kNone) {
-        if (lane < 16u) {
-            const char* src = reinterpret_cast<const char*>(T.sub_len + (uint64_t)c * kSubBlocks) + lane * 4u;
-            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(slot + lane * 4u), "l"(src) : "memory");
-        } else if (lane < 18u) {
-            const uint64_t* src = T.offsets + c + (lane - 16u);
-            asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(slot + 64u + (lane - 16u) * 8u), "l"(src)
-                         : "memory");
-        }
+    if (c != kNone && lane < 20u) {
+        // 4 bytes per lane: lanes 0..15 the sub-block lengths, lanes 16..19 the two offsets
+        const char* src = lane < 16u ? reinterpret_cast<const char*>(T.sub_len + (uint64_t)c * kSubBlocks) + lane * 4u
+                                     : reinterpret_cast<const char*>(T.offsets + c) + (lane - 16u) * 4u;
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(slot + lane * 4u), "l"(src) : "memory");
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
@@ -155,12 +151,13 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32
     const uint64_t off0 = lds64(slot + 64u), off1 = lds64(slot + 72u);
     uint64_t byte0, byte1;
     chunk_bytes(off0, off1, byte0, byte1);
-    if (off1 < off0 || off1 - off0 > 32ull * 65535ull || byte1 > T.stream_words * 4) {
+    // (off1 < off0 wraps to a huge difference; off1 <= last_bit keeps byte1 inside the buffer)
+    if (off1 - off0 > 32ull * 65535ull || off1 > T.last_bit) {
         if (lane == 0) atomicOr(status, kStatCorrupt);
         return r;
     }
     const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    const bool full = (uint64_t)(c + 1) * T.chunk_symbols <= T.n;
+    const bool full = c < T.full_chunks;
     const uint32_t bytes = (uint32_t)(byte1 - byte0);
     if (!full || (sub & 7u) || bytes > stage_bytes || cx.dead()) {
         r.meta = ready_meta(0, 0, 0, kGeneral);
@@ -505,8 +502,9 @@ __device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status
         if (lane >= (uint32_t)d) incl += t;
     }
     const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
-    const uint64_t off0 = lds64(slot + 64u), off1 = lds64(slot + 72u);
-    if (off1 - off0 != (uint64_t)total) {       // the recorded lengths do not add up to the chunk
+    // (prepare has checked that the chunk is shorter than 2^21 bits: the low words decide)
+    const uint32_t off0 = lds32(slot + 64u), off1 = lds32(slot + 72u);
+    if (off1 - off0 != total) {                 // the recorded lengths do not add up to the chunk
         if (lane == 0) atomicOr(status, kStatCorrupt);
         L.kind = kSkip;
         return L;
@@ -516,8 +514,8 @@ __device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status
         L.start = excl;
         L.end = bits;
     } else {
-        const uint32_t byte0_bits = (uint32_t)off0 & ~127u;    // bit offset of the copied bytes' start, modulo 2^32
-        L.start = (cx.stage_addr + r.at()) * 8u + ((uint32_t)off0 - byte0_bits) + excl;
+        const uint32_t byte0_bits = off0 & ~127u;              // bit offset of the copied bytes' start, modulo 2^32
+        L.start = (cx.stage_addr + r.at()) * 8u + (off0 - byte0_bits) + excl;
         L.end = L.start + bits;
     }
     return L;

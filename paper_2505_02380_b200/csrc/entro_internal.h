@@ -26,6 +26,7 @@ struct DevTensor {
     const uint16_t* sub_len;      // n_chunks * 32
     uint16_t* out;                // fp16 bit patterns
     uint64_t stream_words;
+    uint64_t last_bit;            // a chunk may end at this stream bit at most: 28 bytes behind it are still inside the buffer
     uint64_t n;
     uint32_t chunk_symbols;
     uint32_t n_chunks;
@@ -34,7 +35,8 @@ struct DevTensor {
     int32_t zero_point;
     uint32_t item_chunks;         // chunks per work item of this tensor
     uint32_t raw_symbols;         // 1: the tables hold the symbols themselves, not dequantised values
-    uint32_t pad;
+    uint32_t full_chunks;         // chunks that hold chunk_symbols symbols (all but a ragged last one)
+    uint32_t pad[2];
     uint8_t len[ENTRO_MAX_SYMBOLS];
 };
 static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vectors");
