@@ -391,7 +391,8 @@ struct EmitDot {
 
 // 8-bit alphabets, eight symbols per turn.  G = 2, 3 (as 3 + 3 + 2), 4: groups of that many
 // lookups, each checked.  G = 8: two groups of four under one check, for streams whose groups
-// of four almost never fail; if either failed, both are done again one by one.
+// of four almost never fail; if either failed, both are done again one by one.  G = 16: all
+// eight lookups on one view (at most 2 bit per symbol), done again as two fours if it fails.
 template <int K, int G, class Emit>
 __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status, LutKey key, Emit& emit)
 {
@@ -400,6 +401,16 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
     while (emit.more()) {
         uint32_t pk[4];
         bool again = G == 4;
+        if (G == 16) {
+            uint4 v;
+            uint32_t s;
+            group8(r, key, v, s);
+            pk[0] = v.x, pk[1] = v.y, pk[2] = v.z, pk[3] = v.w;
+            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) {
+                cur_init(r, rewind_group(r, s));
+                again = true;
+            }
+        }
         if (G == 8) {
             uint32_t s0, s1;
             group4(r, key, pk[0], pk[1], s0);
@@ -412,7 +423,7 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
                 again = true;
             }
         }
-        if (G == 4 || G == 8) {
+        if (G == 4 || G == 8 || G == 16) {
             if (again) {
 #pragma unroll
                 for (int g = 0; g < 2; ++g) {
@@ -470,6 +481,7 @@ __device__ __forceinline__ uint32_t rows_any(const DecodeAux* aux, uint32_t star
     if (aux->oct) return rows_oct<K>(start, status, emit);
     const LutKey key = lut_key(aux->expm, lane);
     switch (aux->group) {
+        case 16u: return rows_single<K, 16>(start, status, key, emit);
         case 8u: return rows_single<K, 8>(start, status, key, emit);
         case 4u: return rows_single<K, 4>(start, status, key, emit);
         case 3u: return rows_single<K, 3>(start, status, key, emit);

@@ -256,6 +256,40 @@ __device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint
             : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s), "+r"(c.w2)
             : "r"(key.lane), "r"(key.mask));
 }
+// Eight lookups on one view, for streams of so few bits per symbol (at most 2) that eight
+// codes almost always fit 32 bits: 4-bit alphabets beyond the reach of the eight-symbol table.
+#define ENTRO_LOOKUP8(dst, win)                      \
+    "cvt.rz.f32.u32 f, " win ";\n\t"                  \
+    "mov.b32 a, f;\n\t"                               \
+    "shr.u32 a, a, 12;\n\t"                           \
+    "lop3.b32 a, a, %11, %10, 0xEA;\n\t"              \
+    "ld.shared.b32 " dst ", [a+1024];\n\t"
+#define ENTRO_NEXT8(e)                               \
+    "add.u32 %6, %6, " e ";\n\t"                      \
+    "shf.l.wrap.b32 w, 0, h, %6;\n\t"
+__device__ __forceinline__ void group8(Cur& c, LutKey key, uint4& pk, uint32_t& s)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b32 t, w, a, h, e0, e1, e2, e3, e4, e5, e6, e7;\n\t"
+        ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP8("e0", "h")
+        "shf.l.wrap.b32 w, 0, h, e0;\n\t" ENTRO_LOOKUP8("e1", "w")
+        "add.u32 %6, e0, e1;\n\t"
+        "shf.l.wrap.b32 w, 0, h, %6;\n\t" ENTRO_LOOKUP8("e2", "w") ENTRO_NEXT8("e2") ENTRO_LOOKUP8("e3", "w")
+        ENTRO_NEXT8("e3") ENTRO_LOOKUP8("e4", "w") ENTRO_NEXT8("e4") ENTRO_LOOKUP8("e5", "w")
+        ENTRO_NEXT8("e5") ENTRO_LOOKUP8("e6", "w") ENTRO_NEXT8("e6") ENTRO_LOOKUP8("e7", "w")
+        "add.u32 %6, %6, e7;\n\t"
+        "prmt.b32 %4, e0, e1, 0x7632;\n\t"
+        "prmt.b32 %5, e2, e3, 0x7632;\n\t"
+        "prmt.b32 %8, e4, e5, 0x7632;\n\t"
+        "prmt.b32 %9, e6, e7, 0x7632;\n\t" ENTRO_MOVE_ON "}"
+        : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk.x), "=&r"(pk.y), "=&r"(s), "+r"(c.w2), "=&r"(pk.z),
+          "=&r"(pk.w)
+        : "r"(key.lane), "r"(key.mask));
+}
+#undef ENTRO_LOOKUP8
+#undef ENTRO_NEXT8
 #undef ENTRO_LOOKUP
 #undef ENTRO_OPEN
 #undef ENTRO_MOVE_ON

@@ -102,13 +102,13 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     // With 2^-length for the chance of a symbol, fail[g] = chance that g lengths sum to 32 or
     // more, by repeated convolution of the length distribution (bin 32 collects the rest).
     {
-        __shared__ float by_len[33], dist[2][33], fail[5];
+        __shared__ float by_len[33], dist[2][33], fail[9];
         if (tid <= 32) {
             by_len[tid] = tid ? (float)count[tid] * exp2f(-(float)tid) : 0.f;
             dist[0][tid] = tid == 0 ? 1.f : 0.f;
         }
         __syncthreads();
-        for (int g = 1; g <= 4; ++g) {
+        for (int g = 1; g <= 8; ++g) {
             const float* in = dist[(g - 1) & 1];
             float* o = dist[g & 1];
             if (tid < 32) {
@@ -128,7 +128,10 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
         if (tid == 0) {
             const float mean_len = (float)T.offsets[T.n_chunks] / (float)T.n;   // guards against a codebook that does not fit the data
             // a failing lane stalls its warp: the limits keep the warp's failures to a few per cent
-            if (fail[4] < 3e-4f && mean_len <= 4.0f) aux.group = 8u;        // two groups of four under one check
+            // (with a 4-bit alphabet one symbol is far ahead of the rest and 2^-length says little:
+            // there the bit rate alone decides about the eight lookups on one view)
+            if (mean_len <= 2.0f && (T.nsym <= 16 || fail[8] < 3e-4f)) aux.group = 16u;
+            else if (fail[4] < 3e-4f && mean_len <= 4.0f) aux.group = 8u;   // two groups of four under one check
             else if (fail[4] < 3e-3f && mean_len <= 5.2f) aux.group = 4u;
             else if (fail[3] < 2.4e-3f && mean_len <= 8.5f) aux.group = 3u;
         }

@@ -62,7 +62,7 @@ struct DecodeAux {
     uint8_t sorted[ENTRO_MAX_SYMBOLS];                 // symbols by (length, symbol)
     uint32_t max_len;
     uint32_t oct;      // 1: eight symbols per lookup (alphabets of <= 16 symbols)
-    uint32_t group;    // one-symbol lookups per group: 2, 3, 4, or 8 = two groups of four under one check
+    uint32_t group;    // one-symbol lookups per group: 2, 3, 4; 8 = two groups of four under one check; 16 = eight on one view
     uint32_t expm;     // mantissa bits of this tensor's exponent-indexed table
 };
 static_assert(sizeof(DecodeAux) % 16 == 0, "DecodeAux is copied as 16-byte vectors");

@@ -159,10 +159,12 @@ def test_decode_flat_histograms(bits, chunk):
     assert_status_ok()
 
 
-@pytest.mark.parametrize("sigma_levels,foreign", [(2.0, False), (6.0, False), (14.0, False), (40.0, False), (40.0, True)])
+@pytest.mark.parametrize("sigma_levels,foreign", [(0.6, False), (2.0, False), (6.0, False), (14.0, False), (40.0, False),
+                                                  (40.0, True)])
 def test_decode_every_group_size(sigma_levels, foreign):
     """The decoder picks the number of lookups per group from the code lengths and the bits
-    per symbol: narrow histograms take two fours under one check, wider ones four, three,
+    per symbol: below 2 bit per symbol eight lookups share one view, narrow histograms take two
+    fours under one check, wider ones four, three,
     and a codebook that does not fit its data (here: built for a narrow histogram, used on a
     wide one, about 14 bits per symbol) two.  Symbols are drawn directly, as rounded
     Gaussians of the given width in quantisation levels; the values check the symbols."""
@@ -188,7 +190,8 @@ def test_decode_every_group_size(sigma_levels, foreign):
 @pytest.mark.parametrize("sigma_levels,lo,hi", [(0.3, 1.0, 1.3), (0.5, 1.32, 1.74), (0.6, 1.32, 1.74), (1.5, 1.8, 4.0)])
 def test_decode_four_bit_modes(sigma_levels, lo, hi):
     """4-bit alphabets are decoded eight symbols per lookup while eight codes usually fit
-    the table's window (up to 1.31 bit per symbol) and one by one above.  Symbols are drawn
+    the table's window (up to 1.31 bit per symbol) and one by one above (eight lookups on one
+    32-bit view up to 2 bit per symbol).  Symbols are drawn
     directly as rounded Gaussians; the bit rate is checked so that the cases lie on both
     sides of that limit, close to it and far from it; output as fp16 values, and as packed
     nibbles (the integer sink of the same loops)."""
