@@ -94,11 +94,10 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     while (true) {
         const uint32_t item = s_item[slot];
         if (item >= total_items) break;
-        // claim the next item early; it is read after the barrier that ends this one
-        if (threadIdx.x == 0) {
-            s_item[slot ^ 1u] = atomicAdd(control, 1u);
-            s_claim[slot ^ 1u] = 0;
-        }
+        // claim the next item early; the answer of the global counter is not waited for here
+        // but put on record when this item is done, before the barrier that ends it
+        uint32_t next_item = 0;
+        if (threadIdx.x == 0) next_item = atomicAdd(control, 1u);
         // tensor of this item: last t with item_start[t] <= item
         int lo = 0, hi = ntensors - 1;
         while (lo < hi) {
@@ -186,6 +185,10 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             sp = other;
         }
         asm volatile("cp.async.wait_all;" ::: "memory");
+        if (threadIdx.x == 0) {
+            s_item[slot ^ 1u] = next_item;
+            s_claim[slot ^ 1u] = 0;
+        }
         __syncthreads();   // tables may be replaced; s_item / s_claim [slot ^ 1] are now visible
         slot ^= 1u;
     }
