@@ -360,11 +360,38 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, ItemPlan& plan, DevTensor& 
 
 }  // namespace
 
+// A chunk is decoded from shared memory only if its bytes fit the warp's ring; otherwise its
+// lanes read global memory word by word, about six times slower.  Where most of a launch's
+// symbols sit in chunks that (going by the streams' sizes) do not fit the ring of the
+// configured shape, the launch runs with half or a quarter of the warps and accordingly
+// larger rings: slower per SM than the full shape, but far better than the fallback.
+DecodeConfig config_for(const DecodeConfig& base, const entro_tensor_desc* descs, int ntensors, int max_smem)
+{
+    DecodeConfig cfg = base;
+    for (int step = 0; step < 2; ++step) {
+        const Shape sh = shape_for(cfg, max_smem);
+        if (sh.stage_bytes == 0 || cfg.warps_per_cta < 16) break;
+        uint64_t total = 0, too_big = 0;
+        for (int i = 0; i < ntensors; ++i) {
+            const entro_tensor_desc& d = descs[i];
+            if (!d.chunk_symbols || d.n < d.chunk_symbols || d.stream_words < ENTRO_STREAM_SLACK_WORDS)
+                continue;                             // nothing, or only a ragged chunk (general path anyway), or not valid
+            total += d.n;
+            const uint64_t stream_bytes = (d.stream_words - ENTRO_STREAM_SLACK_WORDS) * 4;
+            const uint64_t chunk_bytes = stream_bytes * d.chunk_symbols / d.n + 48;   // mean chunk, margins of the copy
+            if (chunk_bytes > sh.stage_bytes) too_big += d.n;
+        }
+        if (too_big * 2 <= total) break;
+        cfg.warps_per_cta /= 2;
+    }
+    return shape_for(cfg, max_smem).stage_bytes ? cfg : base;
+}
+
 // Upload descriptors, build the tables and run the persistent decode kernel.
 entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs, int ntensors, cudaStream_t s,
                                    int sink = kSinkFp16)
 {
-    const DecodeConfig cfg = decode_config();
+    const DecodeConfig cfg = config_for(decode_config(), descs, ntensors, ws->max_smem_optin);
     ItemPlan plan = plan_items(cfg, descs, ntensors, ws->sm_count);
     int live = 0;
     for (int i = 0; i < ntensors; ++i) {

@@ -187,6 +187,33 @@ def test_decode_every_group_size(sigma_levels, foreign):
     assert_status_ok()
 
 
+@pytest.mark.parametrize("chunk", [8192, 16384])
+def test_chunks_larger_than_a_warps_ring(chunk):
+    """At 8 bit per symbol a chunk of 8192 or 16384 symbols does not fit the 5 KB of shared
+    memory a warp has in the usual launch shape; the library then launches fewer warps with
+    larger rings (and whatever still does not fit is decoded from global memory)."""
+    rng = np.random.default_rng(chunk)
+    tensors = []
+    for n in (6 * chunk + 77, 3 * chunk):
+        q = rng.integers(0, 256, n).astype(np.uint8)
+        ln = oracle.huffman_lengths(np.bincount(q, minlength=256).tolist())
+        cd = oracle.canonical_codes(ln)
+        tensors.append((q, ln, cd, oracle.encode(q, ln, cd, chunk)))
+    descs, outs, keep = [], [], []
+    for q, ln, cd, enc in tensors:
+        assert int(enc.offsets[1]) // 8 > 6000
+        s, ix = to_dev_stream(enc.stream), to_dev_index(enc)
+        out = torch.empty(q.size, dtype=torch.float16, device="cuda")
+        keep += [s, ix]
+        descs.append(E.make_desc(s, ix, q.size, chunk, E.Codebook.from_lengths(ln.tolist(), cd.tolist()), 0.03125, 128, out))
+        outs.append(out)
+    E.entro_decode_dequant_batched(descs)
+    torch.cuda.synchronize()
+    assert_status_ok()
+    for (q, _, _, _), out in zip(tensors, outs):
+        assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.dequant(q, 0.03125, 128))
+
+
 @pytest.mark.parametrize("sigma_levels,lo,hi", [(0.3, 1.0, 1.3), (0.5, 1.32, 1.74), (0.6, 1.32, 1.74), (1.5, 1.8, 4.0)])
 def test_decode_four_bit_modes(sigma_levels, lo, hi):
     """4-bit alphabets are decoded eight symbols per lookup while eight codes usually fit
