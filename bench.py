@@ -31,6 +31,7 @@ import numpy as np
 import torch
 
 import workloads
+from workloads.device import DeviceModel
 
 METRIC = "Huffman decode+dequant GB/s (compressed in + fp16 out)"
 NOMINAL_HBM_GBS = 8000.0
@@ -133,63 +134,6 @@ def physical_gpu_index(local_rank: int) -> int:
 
 
 # ----------------------------------------------------------------------------- this library
-
-class DeviceModel:
-    """A synthetic model compressed on the device with the library's own offline stages."""
-
-    def __init__(self, wl, E, lut_bits: int, keep_q: bool = False, max_code_len: int = 0):
-        self.wl = wl
-        self.q = []              # quantised symbols per tensor (only with keep_q)
-        self.qparams = []
-        self.cbs = []
-        self.keep = []           # device buffers
-        descs = []
-        # per-tensor decode tables read from HBM: canonical ranges + the lookup table of the tensor's mode
-        lut_bytes = 1312 + (2048 if wl.bits == 8 else (17 << lut_bits))
-        total = sum((t.numel + 15) // 16 * 16 for t in wl.tensors)
-        self.out = torch.empty(total, dtype=torch.float16, device="cuda")
-        self.out_slices = []
-        self.n = 0
-        self.stream_bytes = 0    # ceil(total_bits / 8) per tensor
-        self.stream_buf_bytes = 0
-        self.index_bytes = 0
-        self.table_bytes = 0
-        self.max_len = 0
-        pos = 0
-        self.host_meta = []
-        self.compress_s = 0.0    # wall time of quantise + histogram + codebook + encode over all tensors
-        for spec in wl.tensors:
-            w = workloads.make_tensor(spec, "cuda").view(-1)
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            q, qp = E.entro_quantize_tensor(w, wl.bits)
-            counts = E.entro_histogram(q, wl.bits)
-            cb = (E.entro_build_codebook_limited(counts.tolist(), max_code_len) if max_code_len
-                  else E.entro_build_codebook(counts.tolist()))
-            enc = E.entro_encode(q, cb, wl.chunk_symbols, stream_words=E.entro_stream_words(counts.tolist(), cb))
-            torch.cuda.synchronize()
-            self.compress_s += time.perf_counter() - t0
-            self.qparams.append((qp.scale, qp.zero_point))
-            self.cbs.append(cb)
-            if keep_q:
-                self.q.append(q)
-            del w, q
-            out = self.out[pos:pos + spec.numel]
-            pos += (spec.numel + 15) // 16 * 16
-            descs.append(E.make_desc(enc.stream, enc.index, spec.numel, wl.chunk_symbols, cb, qp.scale,
-                                     qp.zero_point, out))
-            self.keep.append(enc)
-            self.out_slices.append(out)
-            self.n += spec.numel
-            self.stream_bytes += (enc.total_bits + 7) // 8
-            self.stream_buf_bytes += enc.stream.numel() * 4
-            self.index_bytes += enc.index.numel()
-            self.table_bytes += lut_bytes
-            self.max_len = max(self.max_len, cb.max_len)
-        self.descs = E.desc_array(descs)
-        self.algorithmic_bytes = self.stream_bytes + self.index_bytes + self.table_bytes + 2 * self.n
-        self.bits_per_weight = 8.0 * self.stream_bytes / self.n
-
 
 def time_steps(E, model, steps, warmup, world, sampler_index):
     import torch.distributed as dist
@@ -409,6 +353,46 @@ def measure_gemv(E, max_layers, reps=5, chunk_symbols=0):
                     "2, 4, 8 tokens per step, fused (two launches per layer) against decode + 7 library GEMMs"}
 
 
+def measure_other(E, name, steps, peak):
+    """One of the other configurations, briefly: its own model build, a few warm-up passes, `steps`
+    timed passes (CUDA events around the whole step, and the library's events around the decode
+    kernel alone).  Outside the headline's timed region."""
+    wl = pick_workload(name, None)
+    model = DeviceModel(wl, E, E.DEFAULT_DECODE_CONFIG[0])
+    for _ in range(3):
+        E.entro_decode_dequant_batched(model.descs)
+    torch.cuda.synchronize()
+    E.entro_profile_begin(steps)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(steps):
+        E.entro_decode_dequant_batched(model.descs)
+    ev1.record()
+    torch.cuda.synchronize()
+    step_ms = ev0.elapsed_time(ev1) / steps
+    kernel_ms = E.entro_profile_read(steps)
+    E.entro_profile_begin(0)
+    assert E.entro_last_device_status() == E.OK
+    k_ms = float(np.mean(kernel_ms))
+    achieved = model.algorithmic_bytes / (k_ms * 1e-3) / 1e9
+    in_l2 = model.algorithmic_bytes < 100e6
+    out = {"workload": wl.name + " full-model decode", "bits": wl.bits, "chunk_symbols": wl.chunk_symbols,
+           "tensors": len(wl.tensors), "weights": model.n, "bits_per_weight": model.bits_per_weight,
+           "max_code_len": model.max_len, "steps": steps, "ms_per_step": step_ms,
+           "value": model.algorithmic_bytes / (step_ms * 1e-3) / 1e9, "unit": "GB/s",
+           "weights_per_s": model.n / (step_ms * 1e-3), "bytes_per_step": model.algorithmic_bytes,
+           "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak[0], "unit": "GB/s",
+                        "frac": achieved / peak[0], "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS, "kernel_ms": k_ms,
+                        "kernel_ms_min": float(np.min(kernel_ms))}}
+    if in_l2:
+        out["us_per_call"] = 1e3 * step_ms
+        out["note"] = ("latency-bound: the whole tensor (%.1f MB of traffic) stays in L2 and the call is a handful of "
+                       "microseconds of launches; the roofline fraction is not a roofline point" % (model.algorithmic_bytes / 1e6))
+    del model
+    torch.cuda.empty_cache()
+    return out
+
+
 # ----------------------------------------------------------------------------- CPU oracle legs
 
 def oracle_sample(wl, max_symbols):
@@ -551,6 +535,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-gemv", action="store_true", help="skip the fused decode+GEMV section (config 5)")
+    ap.add_argument("--others", default="smollm8,phi3_4,single,mistral8-paperbits,mistral4-paperbits",
+                    help="further workloads, each timed briefly and listed under 'others' ('' = none)")
+    ap.add_argument("--others-steps", type=int, default=10)
     ap.add_argument("--max-code-len", type=int, default=0,
                     help="use length-limited codes (not the paper's optimal code); 0 = unrestricted Huffman")
     ap.add_argument("--chunk-symbols", type=int, default=0,
@@ -603,6 +590,13 @@ def main():
         torch.cuda.empty_cache()
         gemv = measure_gemv(E, args.max_layers, chunk_symbols=args.gemv_chunk_symbols)
 
+    others = []
+    if args.others and rank == 0 and world == 1:
+        for name in args.others.split(","):
+            if name and name not in (args.workload, args.also):
+                torch.cuda.empty_cache()
+                others.append(measure_other(E, name, args.others_steps, peak))
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": main_res["value"], "unit": "GB/s", "n_gpus": world, "steps": args.steps,
@@ -631,6 +625,8 @@ def main():
             line["also"] = also
         if gemv:
             line["gemv"] = gemv
+        if others:
+            line["others"] = others
         line["paper_context"] = ("paper: 6.66 s (uint8) / 1.66 s (uint4) to decode phi3-mini-4k on a Jetson P3450, "
                                  "4 CPU threads, integer output (Table 3) -- other hardware, context only")
         print(json.dumps(line))

@@ -20,18 +20,30 @@
  *    serialised by an internal lock.
  *
  * Compressed format (fixed here; the paper leaves it open)
- *  - Stream: 32-bit words; stream bit i is bit (31 - i % 32) of word i / 32; codewords are
- *    concatenated MSB-first in row-major element order; unused bits are zero.  A stream
- *    buffer holds ceil(total_bits / 32) + ENTRO_STREAM_SLACK_WORDS words, the slack zero,
- *    and starts on a 16-byte boundary.
+ *  - Stream: 32-bit words; stream bit i is bit (31 - i % 32) of word i / 32; a codeword is
+ *    written MSB-first, codewords follow one another without gaps in the order given below;
+ *    unused bits are zero.  A stream buffer holds ceil(total_bits / 32) +
+ *    ENTRO_STREAM_SLACK_WORDS words, the slack zero, and starts on a 16-byte boundary.
  *  - Segments: the paper decodes independent segments with known boundaries in parallel
  *    (Section 3, "Segmentation for parallel Huffman decoding"; Fig. 3).  Here a segment is
- *    a chunk of chunk_symbols consecutive symbols of one tensor (the last chunk may be
- *    short).  The index of a tensor with n_chunks = ceil(n / chunk_symbols) chunks is
- *        uint64_t offsets[n_chunks + 1];      bit position where each chunk starts,
+ *    a chunk of chunk_symbols consecutive symbols of one tensor in row-major element order
+ *    (the last chunk may be short); the chunks' bits follow one another in the stream.
+ *  - Order inside a chunk (the paper fixes the boundaries, not this).  The chunk's m symbols
+ *    e[0 .. m) form groups of 8 consecutive symbols: group g = e[8 g .. 8 g + 8) (the last
+ *    group is short if m is not a multiple of 8).  Group g belongs to sub-block g mod 32.
+ *    The stream holds sub-block 0 first, then sub-block 1, ... sub-block 31; a sub-block
+ *    holds its groups in ascending g (l, l + 32, l + 64, ...), and a group its symbols in
+ *    element order.  A sub-block without a group (short last chunk) is empty.  So the
+ *    stored order of a full chunk of 4096 symbols starts e[0..8), e[256..264), e[512..520),
+ *    ..., e[3840..3848), then sub-block 1: e[8..16), e[264..272), ...
+ *    (32 decoder lanes can then start inside a chunk without searching, and what they decode
+ *    in one step is contiguous in the output.)
+ *  - Index of a tensor with n_chunks = ceil(n / chunk_symbols) chunks:
+ *        uint64_t offsets[n_chunks + 1];      stream bit at which each chunk starts,
  *                                             offsets[n_chunks] = total bits
- *        uint16_t sub_len[n_chunks][32];      each chunk is cut into 32 sub-blocks of
- *                                             chunk_symbols / 32 symbols; bit length of each
+ *        uint16_t sub_len[n_chunks][32];      bits of sub-block l of chunk c (0 if empty);
+ *                                             the 32 values of a chunk sum to
+ *                                             offsets[c + 1] - offsets[c]
  *    stored back to back (entro_index_bytes bytes), 8-byte aligned.
  *  - chunk_symbols is a multiple of 32, at least 32 and at most 16384.
  */
@@ -64,8 +76,9 @@ typedef enum {
     ENTRO_ERR_TOO_MANY_TENSORS = 8 /* more tensors than entro_decode_dequant_static has room for */
 } entro_status;
 
-/* The paper applies "either unsigned or asymmetric quantization per layer, based on its
- * weight distribution" (Section 3, Eq. 1).  AUTO: unsigned iff every weight is >= 0. */
+/* Every tensor is quantised in one of two modes, unsigned or asymmetric, chosen from its
+ * weight distribution (Section 3, "Mixed Quantization Scheme", Eq. 1).  The paper does not
+ * give the rule; AUTO: unsigned iff every weight is >= 0. */
 typedef enum { ENTRO_MODE_AUTO = 0, ENTRO_MODE_UNSIGNED = 1, ENTRO_MODE_ASYMMETRIC = 2 } entro_mode;
 
 typedef struct {
@@ -154,10 +167,9 @@ entro_status entro_build_codebook(const uint64_t *counts_host, int nsym, entro_c
  * uses the unrestricted Huffman code, which no prefix code beats; a capped code costs more
  * (measured on the benchmark's 8-bit weights: +0.045 bit per weight at max_len = 12, +0.18
  * at 10; nothing at 4 bits) and bounds the decoder's table depth.  An optional variant of
- * the format; streams made with it decode with the ordinary decode calls, a little more
- * slowly than Huffman streams (4.0 against 3.8 ms on the benchmark model): this library's
- * tables are shaped for codes that grow long towards the all-ones end, which a capped code
- * does less.  Steps (fixed so that
+ * the format; streams made with it decode with the ordinary decode calls, somewhat more
+ * slowly than Huffman streams: this library's tables are shaped for codes that grow long
+ * towards the all-ones end, which a capped code does less.  Steps (fixed so that
  * the result is unique): leaves ascending by (count, symbol); for level j = max_len .. 1 the
  * list is the leaves merged with the packages of level j + 1, ascending by weight, a leaf
  * before a package of equal weight, packages in the order they were made; packages are the
@@ -180,12 +192,13 @@ uint64_t entro_index_bytes(uint64_t n, uint32_t chunk_symbols);
 
 /*
  * Encode symbols into the compressed format described at the top (Section 3: variable
- * length codes, segments with known boundaries).  stream_dev (16-byte aligned,
+ * length codes, segments with known boundaries).  q_dev: n symbols, one per byte (device,
+ * 16-byte aligned).  stream_dev (16-byte aligned,
  * stream_cap_words words) is zeroed and filled; index_dev (8-byte aligned) receives the
  * offsets and sub-block lengths; *total_bits_host the stream length in bits.  Synchronises.
  * ENTRO_ERR_BUFFER_TOO_SMALL if the stream needs more than stream_cap_words -
  * ENTRO_STREAM_SLACK_WORDS words or the index more than index_cap_bytes;
- * ENTRO_ERR_INVALID_ARG if a symbol has no code.
+ * ENTRO_ERR_INVALID_ARG if a symbol has no code or a buffer is not aligned as stated.
  */
 entro_status entro_encode(const uint8_t *q_dev, uint64_t n, const entro_codebook *cb_host,
                           uint32_t chunk_symbols, uint32_t *stream_dev, uint64_t stream_cap_words,

@@ -20,16 +20,18 @@
  *  - Eq. 1 gives W_int = round(W_fp / s) (unsigned) and round((W_fp - z) / s)
  *    (asymmetric).  The integer-domain form is used: q = clamp(rne(w / s) + z, 0, qmax)
  *    with an integer zero-point z in [0, qmax], so that w_hat = s * (q - z).
- *  - "Based on its weight distribution" (Section 3, mixed quantisation): a tensor is
- *    unsigned iff all of its weights are >= 0, else asymmetric.
+ *  - The mode is chosen per tensor from its weight distribution (Section 3, mixed
+ *    quantisation), the rule is not given: a tensor is unsigned iff all of its weights
+ *    are >= 0, else asymmetric.
  *  - s comes from the tensor's min/max; round() is round-half-to-even in fp32.
  *  - Huffman (Section 3, Huffman weight encoding): repeated merging of the two
  *    smallest nodes; ties are broken by (weight, leaf-before-internal, symbol value or
  *    creation order); code length = depth; unused symbols have length 0; a single
  *    used symbol gets length 1.
  *  - Canonical codes: symbols ordered by (length, symbol); first code 0.
- *  - Bitstream: codewords concatenated MSB-first in row-major element order, stored in
- *    32-bit words, stream bit i being bit (31 - i % 32) of word i / 32.
+ *  - Bitstream: codewords concatenated MSB-first, chunk after chunk and inside a chunk in
+ *    the order given under "Segments", stored in 32-bit words, stream bit i being bit
+ *    (31 - i % 32) of word i / 32.
  *  - Segments (Section 3, segmentation for parallel decoding): fixed-size chunks of
  *    chunk_symbols consecutive symbols of one tensor, offsets[c] = bit position where
  *    chunk c starts, offsets[n_chunks] = total bits.  The paper fixes that segments have
@@ -199,9 +201,8 @@ int oracle_quantize_tensor(const uint16_t *w, uint64_t n, int bits, int mode, ui
 
 /*
  * The grid the paper compares against (Section 3, "Mixed Quantization Scheme"; Table 2,
- * column "SOTA"): block-based quantisation, every run of `block` consecutive weights
- * ("e.g., blocks of 32 weights") with a range, scale and zero point of its own, by the same
- * Eq. 1.  The last block may be shorter.  scales / zps (one per block) may be NULL.
+ * column "SOTA"): block-based quantisation, every run of `block` consecutive weights (the
+ * paper's example is 32) with a range, scale and zero point of its own, by the same Eq. 1.  The last block may be shorter.  scales / zps (one per block) may be NULL.
  */
 int oracle_quantize_blocks(const uint16_t *w, uint64_t n, int bits, int mode, uint64_t block, uint8_t *q,
                            float *scales, int32_t *zps)
@@ -315,8 +316,8 @@ int oracle_huffman_lengths(const uint64_t *counts, int nsym, uint8_t *len)
  * Optimal prefix-code lengths under a cap: no code longer than max_len, total cost
  * sum(count * length) minimal among such codes (the package-merge construction of Larmore
  * and Hirschberg).  This departs from the paper, which uses the unrestricted Huffman code
- * ("no other prefix code can offer a more efficient representation", Section 3); it is an
- * optional format variant.  Steps, fixed so that exactly one answer exists:
+ * and states that no prefix code is more efficient (Section 3, Huffman weight encoding); it
+ * is an optional format variant.  Steps, fixed so that exactly one answer exists:
  *   - leaves = used symbols, ascending by (count, symbol);
  *   - for level j = max_len down to 1: the level's list is the leaves merged with the
  *     packages made at level j + 1 (none at level max_len), ascending by weight; on equal

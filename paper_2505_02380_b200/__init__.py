@@ -20,6 +20,8 @@ LIB_PATH = os.path.join(_HERE, "libentro.so")
 MAX_SYMBOLS = 256
 SUB_BLOCKS = 32
 STREAM_SLACK_WORDS = 8
+MAX_CODE_LEN = 32
+MAX_CHUNK_SYMBOLS = 16384
 MODE_AUTO, MODE_UNSIGNED, MODE_ASYMMETRIC = 0, 1, 2
 
 OK, ERR_INVALID_ARG, ERR_BUFFER_TOO_SMALL, ERR_NONFINITE, ERR_CODE_TOO_LONG, ERR_CORRUPT_STREAM, ERR_CUDA, \

@@ -49,6 +49,37 @@ class CompressedTensor:
         return E.Codebook.from_lengths(self.lengths)      # the decoder reads the lengths only
 
 
+def _check_entry(path: str, e: dict, stream_words: int, index_bytes: int) -> None:
+    """The sizes a header entry states must agree with one another before anything is handed to
+    the decoder: it sizes its reads of the index from shape and chunk size, and of the stream
+    from total_bits, not from the sizes of the blobs."""
+    def bad(what: str):
+        raise ValueError(f"{path}: {e.get('name')!r}: {what}")
+
+    shape, chunk, bits, lengths = e["shape"], e["chunk_symbols"], e["bits"], e["lengths"]
+    if bits not in (4, 8):
+        bad(f"bits = {bits}")
+    if not isinstance(lengths, list) or not 1 <= len(lengths) <= (1 << bits) or \
+            any(not isinstance(l, int) or l < 0 or l > E.MAX_CODE_LEN for l in lengths):
+        bad("code lengths do not describe an alphabet of this width")
+    if any(not isinstance(d, int) or d < 0 for d in shape):
+        bad(f"shape = {shape}")
+    numel = int(np.prod(shape, dtype=np.int64)) if shape else 1
+    if not isinstance(chunk, int) or chunk < E.SUB_BLOCKS or chunk % E.SUB_BLOCKS or chunk > E.MAX_CHUNK_SYMBOLS:
+        bad(f"chunk_symbols = {chunk}")
+    if numel == 0:
+        bad("empty tensor")
+    n_chunks = (numel + chunk - 1) // chunk
+    if index_bytes != 8 * (n_chunks + 1) + 2 * E.SUB_BLOCKS * n_chunks:
+        bad(f"index of {index_bytes} bytes does not fit {numel} symbols in chunks of {chunk}")
+    total_bits = e["total_bits"]
+    if not isinstance(total_bits, int) or total_bits < 0 or \
+            stream_words < (total_bits + 31) // 32 + E.STREAM_SLACK_WORDS:
+        bad(f"stream of {stream_words} words is too short for {total_bits} bits")
+    if not 0 <= e["zero_point"] < (1 << bits):
+        bad(f"zero_point = {e['zero_point']}")
+
+
 class CompressedModel:
     def __init__(self, tensors: List[CompressedTensor]):
         self.tensors = tensors
@@ -113,6 +144,7 @@ class CompressedModel:
                     if got != nbytes:
                         raise ValueError(f"{path}: {e['name']}: short read")
                     bufs[key] = t.view(dtype)
+                _check_entry(path, e, bufs["stream"].numel(), bufs["index"].numel())
                 scale = float(np.uint32(e["scale_bits"]).view(np.float32))
                 tensors.append(CompressedTensor(e["name"], tuple(e["shape"]), e["bits"], e["chunk_symbols"], scale,
                                                 e["zero_point"], e["lengths"], bufs["stream"], bufs["index"],

@@ -529,41 +529,49 @@ extern "C" entro_status entro_decode_dequant_batched_host(const entro_tensor_des
     if (!ws || !copy_streams_ready(ws)) return ENTRO_ERR_CUDA;
     // groups of consecutive tensors, about equal in output bytes
     const uint64_t per_group = out_bytes / Workspace::kCopyGroups + 1;
-    // the copy streams start after what the caller has queued, and the caller's stream ends after them
-    ENTRO_CUDA(cudaEventRecord(ws->ev_edge, s));
-    ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_in, ws->ev_edge, 0));
-    ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_out, ws->ev_edge, 0));
-    int first = 0, group = 0;
-    while (first < ntensors) {
-        int last = first;
-        uint64_t bytes = 0;
-        while (last < ntensors && (bytes < per_group || group == Workspace::kCopyGroups - 1)) bytes += descs[last++].n * 2;
-        for (int i = first; i < last; ++i) {
-            const entro_tensor_desc& d = descs[i];
-            if (!d.n) continue;
-            ENTRO_CUDA(cudaMemcpyAsync(const_cast<uint32_t*>(d.stream_dev), io[i].stream_host, d.stream_words * 4,
-                                       cudaMemcpyHostToDevice, ws->copy_in));
-            ENTRO_CUDA(cudaMemcpyAsync(const_cast<void*>(d.index_dev), io[i].index_host,
-                                       entro_index_bytes(d.n, d.chunk_symbols), cudaMemcpyHostToDevice, ws->copy_in));
+    auto enqueue = [&]() -> entro_status {
+        // the copy streams start after what the caller has queued, and the caller's stream ends after them
+        ENTRO_CUDA(cudaEventRecord(ws->ev_edge, s));
+        ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_in, ws->ev_edge, 0));
+        ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_out, ws->ev_edge, 0));
+        int first = 0, group = 0;
+        while (first < ntensors) {
+            int last = first;
+            uint64_t bytes = 0;
+            while (last < ntensors && (bytes < per_group || group == Workspace::kCopyGroups - 1)) bytes += descs[last++].n * 2;
+            for (int i = first; i < last; ++i) {
+                const entro_tensor_desc& d = descs[i];
+                if (!d.n) continue;
+                ENTRO_CUDA(cudaMemcpyAsync(const_cast<uint32_t*>(d.stream_dev), io[i].stream_host, d.stream_words * 4,
+                                           cudaMemcpyHostToDevice, ws->copy_in));
+                ENTRO_CUDA(cudaMemcpyAsync(const_cast<void*>(d.index_dev), io[i].index_host,
+                                           entro_index_bytes(d.n, d.chunk_symbols), cudaMemcpyHostToDevice, ws->copy_in));
+            }
+            ENTRO_CUDA(cudaEventRecord(ws->ev_in[group], ws->copy_in));
+            ENTRO_CUDA(cudaStreamWaitEvent(s, ws->ev_in[group], 0));
+            entro_status st = decode_batched_locked(ws, descs + first, last - first, s);
+            if (st != ENTRO_OK) return st;
+            ENTRO_CUDA(cudaEventRecord(ws->ev_dec[group], s));
+            ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_out, ws->ev_dec[group], 0));
+            for (int i = first; i < last; ++i) {
+                const entro_tensor_desc& d = descs[i];
+                if (!d.n || !io[i].out_fp16_host) continue;     // no host buffer: the result stays on the device
+                ENTRO_CUDA(cudaMemcpyAsync(io[i].out_fp16_host, d.out_fp16_dev, d.n * 2, cudaMemcpyDeviceToHost, ws->copy_out));
+            }
+            first = last;
+            ++group;
         }
-        ENTRO_CUDA(cudaEventRecord(ws->ev_in[group], ws->copy_in));
-        ENTRO_CUDA(cudaStreamWaitEvent(s, ws->ev_in[group], 0));
-        entro_status st = decode_batched_locked(ws, descs + first, last - first, s);
-        if (st != ENTRO_OK) return st;
-        ENTRO_CUDA(cudaEventRecord(ws->ev_dec[group], s));
-        ENTRO_CUDA(cudaStreamWaitEvent(ws->copy_out, ws->ev_dec[group], 0));
-        for (int i = first; i < last; ++i) {
-            const entro_tensor_desc& d = descs[i];
-            if (!d.n || !io[i].out_fp16_host) continue;     // no host buffer: the result stays on the device
-            ENTRO_CUDA(cudaMemcpyAsync(io[i].out_fp16_host, d.out_fp16_dev, d.n * 2, cudaMemcpyDeviceToHost, ws->copy_out));
-        }
-        first = last;
-        ++group;
-    }
-    ENTRO_CUDA(cudaEventRecord(ws->ev_edge, ws->copy_out));
-    ENTRO_CUDA(cudaStreamWaitEvent(s, ws->ev_edge, 0));
-    ENTRO_CUDA(cudaStreamSynchronize(s));
-    return ENTRO_OK;
+        ENTRO_CUDA(cudaEventRecord(ws->ev_edge, ws->copy_out));
+        ENTRO_CUDA(cudaStreamWaitEvent(s, ws->ev_edge, 0));
+        return ENTRO_OK;
+    };
+    const entro_status st = enqueue();
+    // Whatever was queued, on the copy streams or the caller's, has finished with the caller's
+    // buffers before the call returns, on the error paths too.
+    const cudaError_t e_in = cudaStreamSynchronize(ws->copy_in), e_out = cudaStreamSynchronize(ws->copy_out),
+                      e_s = cudaStreamSynchronize(s);
+    if (st != ENTRO_OK) return st;
+    return (e_in == cudaSuccess && e_out == cudaSuccess && e_s == cudaSuccess) ? ENTRO_OK : ENTRO_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------ matrix-vector products
@@ -809,7 +817,7 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
         if (status_dev) ENTRO_CUDA(cudaMemsetAsync(status_dev, 0, sizeof(uint32_t), s));
         return ENTRO_OK;
     }
-    const DecodeConfig cfg = decode_config();
+    const DecodeConfig cfg = config_for(decode_config(), descs_host, ntensors, sd->max_smem_optin);   // host arithmetic only
     ItemPlan plan = plan_items(cfg, descs_host, ntensors, sd->sm_count);
 
     StaticUpload up;

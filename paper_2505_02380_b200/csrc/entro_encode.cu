@@ -176,7 +176,8 @@ extern "C" entro_status entro_encode(const uint8_t* q_dev, uint64_t n, const ent
     if (!q_dev || !cb || !stream_dev || !index_dev || !total_bits_host || n == 0) return ENTRO_ERR_INVALID_ARG;
     if (chunk_symbols < kSubBlocks || chunk_symbols % kSubBlocks || chunk_symbols > ENTRO_MAX_CHUNK_SYMBOLS)
         return ENTRO_ERR_INVALID_ARG;
-    if (!aligned(stream_dev, 16) || !aligned(index_dev, 8)) return ENTRO_ERR_INVALID_ARG;
+    // q is read as 8-byte vectors (a group of eight symbols at a time)
+    if (!aligned(q_dev, 16) || !aligned(stream_dev, 16) || !aligned(index_dev, 8)) return ENTRO_ERR_INVALID_ARG;
     if (!codebook_lengths_valid(cb)) return ENTRO_ERR_INVALID_ARG;
     const uint64_t nc64 = num_chunks(n, chunk_symbols);
     if (nc64 > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;

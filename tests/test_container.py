@@ -44,6 +44,52 @@ def test_file_round_trip_on_the_host(tmp_path):
         container.CompressedModel.load(path, pin=False)
 
 
+def _doctored(tmp_path, change):
+    """A valid one-tensor file whose header entry has been changed by `change`."""
+    import json
+    import struct
+    w = workloads.make_values(3 * 5000, 0.02, 9).numpy()
+    model = container.CompressedModel([_from_oracle("w", (3, 5000), w, 8, 4096)[1]])
+    path = str(tmp_path / "d.entro")
+    model.save(path)
+    raw = open(path, "rb").read()
+    (hlen,) = struct.unpack("<Q", raw[8:16])
+    head = json.loads(raw[16:16 + hlen].decode())
+    change(head["tensors"][0])
+    new = json.dumps(head).encode()
+    start_old = (16 + hlen + container.ALIGN - 1) // container.ALIGN * container.ALIGN
+    start_new = (16 + len(new) + container.ALIGN - 1) // container.ALIGN * container.ALIGN
+    with open(path, "wb") as f:
+        f.write(raw[:8] + struct.pack("<Q", len(new)) + new)
+        f.seek(start_new)
+        f.write(raw[start_old:])
+    return path
+
+
+@pytest.mark.parametrize("change", [
+    lambda e: e.__setitem__("shape", [30, 5000]),            # more chunks than the index holds
+    lambda e: e.__setitem__("chunk_symbols", 1024),          # likewise
+    lambda e: e.__setitem__("chunk_symbols", 4100),          # not a multiple of 32
+    lambda e: e.__setitem__("total_bits", 10 ** 9),          # more bits than the stream holds
+    lambda e: e.__setitem__("bits", 5),
+    lambda e: e.__setitem__("lengths", [1] * 300),
+    lambda e: e.__setitem__("lengths", [40, 1]),
+    lambda e: e.__setitem__("zero_point", 256),
+    lambda e: e["index"].__setitem__(1, e["index"][1] - 64),  # a truncated index blob
+])
+def test_inconsistent_header_is_refused_on_load(tmp_path, change):
+    """The decoder trusts the index to have the size that shape and chunk size imply; a file
+    whose header says otherwise must not get as far as the device."""
+    path = _doctored(tmp_path, change)
+    with pytest.raises(ValueError):
+        container.CompressedModel.load(path, pin=False)
+
+
+def test_consistent_header_loads(tmp_path):
+    path = _doctored(tmp_path, lambda e: None)
+    assert container.CompressedModel.load(path, pin=False).tensors[0].shape == (3, 5000)
+
+
 @pytest.mark.gpu
 @pytest.mark.parametrize("bits", [8, 4])
 def test_compress_save_load_decode_matches_oracle(tmp_path, bits):

@@ -112,6 +112,30 @@ def test_encode_matches_oracle_stream_and_index(bits, chunk):
         assert np.array_equal(enc.sub_len(), c.enc.sub_len)
 
 
+@pytest.mark.parametrize("bits,chunk,n", [(8, 4096, 2 * 4096 + 1000), (4, 8192, 2 * 8192 + 77), (8, 512, 3 * 512 + 20),
+                                          (8, 32, 100), (8, 4096, 5)])
+def test_format_stated_in_the_header_is_the_format_the_library_uses(bits, chunk, n):
+    """An encoder written from the words of include/entro.h alone (tests/format_from_header.py):
+    the library's encoder writes the same stream and index, and the library's decoder turns
+    that encoder's stream into the dequantised symbols, bit for bit."""
+    import format_from_header
+    w_np, w_dev = _values(n, 0.02, 777 + n)
+    q, qp = E.entro_quantize_tensor(w_dev, bits)
+    counts = E.entro_histogram(q, bits).tolist()
+    cb = E.entro_build_codebook(counts)
+    q_np = q.cpu().numpy()
+    stream, offsets, sub_len = format_from_header.encode(q_np.tolist(), cb.lengths().tolist(), cb.codes().tolist(), chunk)
+    enc = E.entro_encode(q, cb, chunk, stream_words=E.entro_stream_words(counts, cb))
+    assert np.array_equal(enc.stream_np(), stream)
+    assert np.array_equal(enc.offsets(), offsets)
+    assert np.array_equal(enc.sub_len(), sub_len)
+    index = torch.from_numpy(format_from_header.index_bytes(offsets, sub_len).copy()).cuda()
+    out = E.entro_decode_dequant(to_dev_stream(stream), index, n, chunk, cb, qp.scale, qp.zero_point)
+    torch.cuda.synchronize()
+    assert_status_ok()
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.dequant(q_np, qp.scale, qp.zero_point))
+
+
 def test_encode_errors():
     q = torch.tensor([0, 1, 2, 3] * 100, dtype=torch.uint8).cuda()
     cb = E.entro_build_codebook([5, 5, 5, 0])              # symbol 3 has no code

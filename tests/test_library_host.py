@@ -120,6 +120,8 @@ def test_argument_errors_are_found_before_any_launch():
     total = C.c_uint64()
     assert L.entro_encode(None, 16, C.byref(cb), 4096, None, 0, None, 0, C.byref(total), None) == E.ERR_INVALID_ARG
     assert L.entro_encode(16, 16, C.byref(cb), 100, 16, 64, 16, 4096, C.byref(total), None) == E.ERR_INVALID_ARG
+    # symbols that do not start on a 16-byte boundary (an offset view of a tensor: q[1:]) are refused
+    assert L.entro_encode(17, 16, C.byref(cb), 4096, 16, 64, 16, 4096, C.byref(total), None) == E.ERR_INVALID_ARG
     assert L.entro_decode_dequant(None, 0, None, 16, 4096, C.byref(cb), 1.0, 0, None, None) == E.ERR_INVALID_ARG
     assert L.entro_decode_dequant(16, 100, 16, 16, 4096, C.byref(cb), 1.0, 0, 24, None) == E.ERR_INVALID_ARG  # misaligned out
     bad = E.Codebook.from_lengths([1, 1, 1, 0])        # over-subscribed lengths

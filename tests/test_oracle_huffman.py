@@ -274,6 +274,20 @@ def test_stream_is_concatenation_of_codewords_and_index_is_consistent(bits, chun
         assert int(enc.sub_len[k].sum()) == int(enc.offsets[k + 1] - enc.offsets[k])
 
 
+@pytest.mark.parametrize("bits,chunk,n", [(8, 4096, 2 * 4096 + 1000), (4, 8192, 8192 + 77), (8, 512, 3 * 512 + 20),
+                                          (8, 32, 100), (4, 64, 64), (8, 4096, 5)])
+def test_oracle_stream_and_index_equal_an_encoder_written_from_the_public_header(bits, chunk, n):
+    """tests/format_from_header.py restates the header's format text as loops; the oracle's
+    stream, chunk offsets and sub-block lengths must be what those loops write."""
+    import format_from_header
+    w = workloads.make_values(n, 0.02, 4242 + n).numpy()
+    c = oracle.compress(w, bits, chunk)
+    stream, offsets, sub_len = format_from_header.encode(c.q.tolist(), c.lengths.tolist(), c.codes.tolist(), chunk)
+    assert np.array_equal(stream, c.enc.stream)
+    assert np.array_equal(offsets, c.enc.offsets)
+    assert np.array_equal(sub_len, c.enc.sub_len)
+
+
 # ----------------------------------------------------------------------------- decoder
 
 def _dict_decode(bits_arr, start, count, table):

@@ -1,0 +1,70 @@
+"""A synthetic model held on the device in compressed form.
+
+Glue for the benchmark and the full-size tests: it draws every tensor of a workload on the
+device and runs the compress stages on it through whatever binding it is given (`E`, the
+library's Python binding, passed in: this module imports neither the library nor the
+oracle, and holds none of the method's arithmetic)."""
+from __future__ import annotations
+
+import time
+
+import torch
+
+import workloads
+
+
+class DeviceModel:
+    """A synthetic model compressed on the device with the library's own offline stages."""
+
+    def __init__(self, wl, E, lut_bits: int, keep_q: bool = False, max_code_len: int = 0):
+        self.wl = wl
+        self.q = []              # quantised symbols per tensor (only with keep_q)
+        self.qparams = []
+        self.cbs = []
+        self.keep = []           # device buffers
+        descs = []
+        # per-tensor decode tables read from HBM: canonical ranges + the lookup table of the tensor's mode
+        lut_bytes = 1312 + (2048 if wl.bits == 8 else (17 << lut_bits))
+        total = sum((t.numel + 15) // 16 * 16 for t in wl.tensors)
+        self.out = torch.empty(total, dtype=torch.float16, device="cuda")
+        self.out_slices = []
+        self.n = 0
+        self.stream_bytes = 0    # ceil(total_bits / 8) per tensor
+        self.stream_buf_bytes = 0
+        self.index_bytes = 0
+        self.table_bytes = 0
+        self.max_len = 0
+        pos = 0
+        self.host_meta = []
+        self.compress_s = 0.0    # wall time of quantise + histogram + codebook + encode over all tensors
+        for spec in wl.tensors:
+            w = workloads.make_tensor(spec, "cuda").view(-1)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            q, qp = E.entro_quantize_tensor(w, wl.bits)
+            counts = E.entro_histogram(q, wl.bits)
+            cb = (E.entro_build_codebook_limited(counts.tolist(), max_code_len) if max_code_len
+                  else E.entro_build_codebook(counts.tolist()))
+            enc = E.entro_encode(q, cb, wl.chunk_symbols, stream_words=E.entro_stream_words(counts.tolist(), cb))
+            torch.cuda.synchronize()
+            self.compress_s += time.perf_counter() - t0
+            self.qparams.append((qp.scale, qp.zero_point))
+            self.cbs.append(cb)
+            if keep_q:
+                self.q.append(q)
+            del w, q
+            out = self.out[pos:pos + spec.numel]
+            pos += (spec.numel + 15) // 16 * 16
+            descs.append(E.make_desc(enc.stream, enc.index, spec.numel, wl.chunk_symbols, cb, qp.scale,
+                                     qp.zero_point, out))
+            self.keep.append(enc)
+            self.out_slices.append(out)
+            self.n += spec.numel
+            self.stream_bytes += (enc.total_bits + 7) // 8
+            self.stream_buf_bytes += enc.stream.numel() * 4
+            self.index_bytes += enc.index.numel()
+            self.table_bytes += lut_bytes
+            self.max_len = max(self.max_len, cb.max_len)
+        self.descs = E.desc_array(descs)
+        self.algorithmic_bytes = self.stream_bytes + self.index_bytes + self.table_bytes + 2 * self.n
+        self.bits_per_weight = 8.0 * self.stream_bytes / self.n
