@@ -278,9 +278,10 @@ typedef struct {
  * down to the smaller amount of weight data that is moved while tokens are generated, a
  * phase bound by memory bandwidth (Section 4, Table 3); here only the compressed stream
  * crosses HBM, once for all tokens of the batch.  descs_host[i].out_fp16_dev is not used and may be NULL.  All ntensors
- * products are independent and run in one launch.  The order of the fp32 additions is not
- * fixed (rows that span chunks are summed with atomics), so results can differ from run to
- * run in the last bits before the final rounding.
+ * products are independent and run in one launch, which also rounds and stores y: a row that
+ * lies inside one chunk is summed by one warp in a fixed order; a row that spans chunks gets
+ * the chunks' partial sums added with fp32 atomics (the last chunk to arrive rounds), so its
+ * result can differ from run to run in the last bits before the final rounding.
  * Limits: cols a multiple of 256, batch * cols at most 32768 (x of all tokens is staged in
  * shared memory), chunk_symbols a multiple of 256 (ENTRO_ERR_UNSUPPORTED otherwise); batch
  * outside 1 .. ENTRO_GEMV_MAX_BATCH or reserved != 0 is ENTRO_ERR_INVALID_ARG.
@@ -289,6 +290,29 @@ typedef struct {
  */
 entro_status entro_decode_dequant_gemv(const entro_tensor_desc *descs_host, const entro_gemv_io *io_host,
                                        int ntensors, void *cuda_stream);
+
+/*
+ * The same products prepared once and run many times: the token-generation loop decodes the
+ * same compressed weights for every token (Section 4, Table 3, token-generation rows), so
+ * everything that does not change from token to token is set up once.  entro_gemv_prepare
+ * validates the arguments as entro_decode_dequant_gemv does, allocates a device area of its
+ * own for the plan (descriptors, decode tables, fp32 sums of the rows that span chunks),
+ * fills it, and returns after cuda_stream has finished that work.  The compressed streams, x and y are NOT copied: the plan keeps the
+ * device pointers given in descs_host / io_host, and every run reads the streams and x and
+ * writes y there (the application refreshes x between runs).
+ * entro_gemv_run is one kernel launch on cuda_stream (asynchronous): decode, multiply, round
+ * and store y.  Runs of one plan must not overlap on the GPU (order them on one stream or
+ * with events); different plans may.  Malformed input is reported through
+ * entro_last_device_status; after such a report the plan's sums are undefined: release it
+ * and prepare again.
+ * entro_gemv_release waits for the device to finish with the plan's area and frees it
+ * (NULL is allowed).
+ */
+typedef struct entro_gemv_plan entro_gemv_plan;
+entro_status entro_gemv_prepare(const entro_tensor_desc *descs_host, const entro_gemv_io *io_host,
+                                int ntensors, void *cuda_stream, entro_gemv_plan **plan_out);
+entro_status entro_gemv_run(entro_gemv_plan *plan, void *cuda_stream);
+entro_status entro_gemv_release(entro_gemv_plan *plan);
 
 /*
  * Plain fp16 matrix-vector product y = fp16_rne(W x), W [rows, cols] row-major fp16 on the
@@ -358,6 +382,19 @@ entro_status entro_set_decode_config(int lut_bits, int warps_per_cta, int ctas_p
  */
 entro_status entro_profile_begin(int max_records);
 int entro_profile_read(float *ms_host, int cap);
+
+/*
+ * The checked build (compiled with -DENTRO_CHECKED: python -m paper_2505_02380_b200.build
+ * --checked makes libentro_checked.so) tests, before each access, every address that the
+ * decode kernel works out by hand: shared-memory offsets of table cells, ring words, index
+ * slots and staged x; place and extent of every bulk copy; every output store.  A violation
+ * is counted and the access left out; nothing traps and no wait is unbounded.  It stands
+ * in for a memory checker and runs several times slower.  entro_checked_build: 1 in that
+ * build, else 0.  entro_check_violations: waits for the device, then returns and clears the
+ * count on the current device (always 0 in the ordinary build, -1 on a CUDA error).
+ */
+int entro_checked_build(void);
+long long entro_check_violations(void);
 
 /* Kernels launched by this library on the calling thread's device since load (for
  * launch accounting in benchmarks). */

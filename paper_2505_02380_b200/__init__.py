@@ -15,7 +15,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libentro.so")
+# The checked build (libentro_checked.so, see build.py) is loaded instead when ENTRO_LIBRARY names it.
+LIB_PATH = os.environ.get("ENTRO_LIBRARY") or os.path.join(_HERE, "libentro.so")
 
 MAX_SYMBOLS = 256
 SUB_BLOCKS = 32
@@ -109,6 +110,9 @@ def lib():
         L.entro_decode_dequant_batched_host.argtypes = [C.POINTER(TensorDesc), C.POINTER(HostIO), i32, vp]
         L.entro_decode_symbols_batched.argtypes = [C.POINTER(TensorDesc), i32, i32, vp]
         L.entro_decode_dequant_gemv.argtypes = [C.POINTER(TensorDesc), C.POINTER(GemvIO), i32, vp]
+        L.entro_gemv_prepare.argtypes = [C.POINTER(TensorDesc), C.POINTER(GemvIO), i32, vp, C.POINTER(vp)]
+        L.entro_gemv_run.argtypes = [vp, vp]
+        L.entro_gemv_release.argtypes = [vp]
         L.entro_gemv_fp16.argtypes = [vp, u32, u32, vp, vp, vp]
         L.entro_decode_dequant_static.argtypes = [C.POINTER(TensorDesc), i32, vp, vp]
         L.entro_last_device_status.argtypes = [vp]
@@ -116,6 +120,10 @@ def lib():
         L.entro_profile_begin.argtypes = [i32]
         L.entro_profile_read.restype = i32
         L.entro_profile_read.argtypes = [C.POINTER(C.c_float), i32]
+        L.entro_checked_build.restype = i32
+        L.entro_checked_build.argtypes = []
+        L.entro_check_violations.restype = C.c_longlong
+        L.entro_check_violations.argtypes = []
         L.entro_kernel_launch_count.restype = u64
         L.entro_kernel_launch_count.argtypes = []
         L.entro_status_string.restype = C.c_char_p
@@ -130,8 +138,8 @@ def lib():
 EXPORTS = ["entro_quantize_tensor", "entro_quantize_blocks", "entro_histogram", "entro_build_codebook", "entro_build_codebook_limited", "entro_stream_words",
            "entro_encode_bound_words", "entro_index_bytes", "entro_encode", "entro_decode_dequant",
            "entro_decode_dequant_batched", "entro_decode_dequant_batched_host", "entro_decode_dequant_static",
-           "entro_decode_dequant_gemv", "entro_gemv_fp16", "entro_decode_symbols_batched", "entro_last_device_status",
-           "entro_set_decode_config", "entro_profile_begin", "entro_profile_read", "entro_kernel_launch_count",
+           "entro_decode_dequant_gemv", "entro_gemv_prepare", "entro_gemv_run", "entro_gemv_release", "entro_gemv_fp16", "entro_decode_symbols_batched", "entro_last_device_status",
+           "entro_set_decode_config", "entro_checked_build", "entro_check_violations", "entro_profile_begin", "entro_profile_read", "entro_kernel_launch_count",
            "entro_status_string"]
 
 
@@ -363,6 +371,51 @@ def entro_decode_dequant_gemv(descs, xs: Optional[Sequence[torch.Tensor]] = None
     return ys
 
 
+class GemvPlan:
+    """Handle of entro_gemv_prepare: keeps the descriptors, x and y alive for as long as the plan
+    holds their device pointers."""
+
+    def __init__(self, handle: int, keep):
+        self.handle, self._keep = handle, keep
+
+    def release(self) -> None:
+        if self.handle:
+            _check(lib().entro_gemv_release(self.handle), "entro_gemv_release")
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.release()
+        except Exception:
+            pass
+
+
+def entro_gemv_prepare(descs, xs: Optional[Sequence[torch.Tensor]] = None, shapes: Optional[Sequence] = None,
+                       ys: Optional[List[torch.Tensor]] = None, stream: Optional[torch.cuda.Stream] = None, io=None):
+    """Arguments as for entro_decode_dequant_gemv.  -> (GemvPlan, ys).  Every entro_gemv_run(plan)
+    reads xs (refreshed in place by the caller) and writes ys."""
+    if isinstance(descs, list):
+        descs = desc_array(descs)
+    n = len(descs)
+    if io is None:
+        if ys is None:
+            ys = [torch.empty((xs[i].shape[0], shapes[i][0]) if xs[i].dim() == 2 else shapes[i][0],
+                              dtype=torch.float16, device=xs[i].device) for i in range(n)]
+        io = make_gemv_io(xs, ys, shapes)
+    handle = C.c_void_p()
+    _check(lib().entro_gemv_prepare(descs, io, n, _stream(stream), C.byref(handle)), "entro_gemv_prepare")
+    return GemvPlan(handle.value, (descs, xs, ys, io)), ys
+
+
+def entro_gemv_run(plan: GemvPlan, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """One launch: decode + dequantise + multiply + round into the plan's ys.  Asynchronous."""
+    _check(lib().entro_gemv_run(plan.handle, _stream(stream)), "entro_gemv_run")
+
+
+def entro_gemv_release(plan: GemvPlan) -> None:
+    plan.release()
+
+
 def entro_gemv_fp16(w: torch.Tensor, x: torch.Tensor, y: Optional[torch.Tensor] = None,
                     stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
     """y = W x for an fp16 matrix W [rows, cols] on the device (fp32 accumulation).  Asynchronous."""
@@ -406,6 +459,19 @@ def entro_profile_read(cap: int = 65536) -> List[float]:
     if n < 0:
         raise EntroError(ERR_CUDA, "entro_profile_read")
     return [float(buf[i]) for i in range(n)]
+
+
+def entro_checked_build() -> bool:
+    return bool(lib().entro_checked_build())
+
+
+def entro_check_violations() -> int:
+    """Checked build: waits for the device, returns and clears the count of accesses the kernels'
+    own bounds checks refused.  Always 0 in the ordinary build."""
+    n = int(lib().entro_check_violations())
+    if n < 0:
+        raise EntroError(ERR_CUDA, "entro_check_violations")
+    return n
 
 
 def entro_kernel_launch_count() -> int:

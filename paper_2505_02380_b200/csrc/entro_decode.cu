@@ -32,6 +32,8 @@
 //     codes in K bits); one unreplicated copy of the exponent-indexed table serves the
 //     symbol-by-symbol repair of such windows.
 //   aux   canonical ranges per length, for whatever the tables do not resolve.
+#include <new>
+
 #include "entro_decode_chunk.cuh"
 
 namespace entro {
@@ -39,11 +41,43 @@ namespace {
 
 // ------------------------------------------------------------------ persistent kernel
 
+// The exponent-indexed table of a tensor into the first 64 KB of shared memory: cell-major
+// copies, word w holds cell w / copies.
+__device__ __forceinline__ void load_exp_table(const TensorTables* tt)
+{
+    const uint32_t shift = 9u - __ldg(&tt->aux.expm);       // log2 of the number of copies
+    if (shift >= 2u) {
+        // four or more copies: the four words of a 16-byte store belong to one cell
+        uint4* s4 = reinterpret_cast<uint4*>(smem);
+        for (uint32_t q = threadIdx.x; q < (uint32_t)kExpEntriesMax / 4u; q += blockDim.x) {
+            const uint32_t v = __ldg(tt->exp_lut() + ((4u * q) >> shift));
+            s4[q] = make_uint4(v, v, v, v);
+        }
+    } else {
+        uint32_t* s1 = reinterpret_cast<uint32_t*>(smem);
+        for (uint32_t w = threadIdx.x; w < (uint32_t)kExpEntriesMax; w += blockDim.x)
+            s1[w] = __ldg(tt->exp_lut() + (w >> shift));
+    }
+}
+
+// A CTA calls this once, after its last claim of a work item.  The last CTA of the grid to get
+// here puts the work counter and the count of finished CTAs back to zero.
+__device__ __forceinline__ void cta_finished(uint32_t* control)
+{
+    if (atomicAdd(control + 2, 1u) == gridDim.x - 1u) {
+        control[0] = 0;
+        control[2] = 0;
+    }
+}
+
 // item_start[t] = first work item of tensor t, item_start[ntensors] = number of items; an
 // item is up to tensors[t].item_chunks consecutive chunks of one tensor.
 // kSink says where the decoded values go.  With kSinkGemv they are not stored: gemv[t]
 // describes the matrix-vector products they enter (the fused decode + dequantise + GEMV of a
 // token step, one token or a small batch).
+// control: [0] the work counter, which must be 0 at the start and is 0 again at the end (the
+// last CTA to finish puts it back, so that a prepared launch can be repeated with nothing in
+// between), [1] the status word, [2] CTAs that have finished.
 template <int K, int kSink>
 __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __restrict__ tensors, int ntensors,
                                                          const uint32_t* __restrict__ item_start,
@@ -56,7 +90,10 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     constexpr bool kGemv = kBatch > 0;
     // layout: [tables][aux][tensor]([gemv descriptor][x])[per-warp rings][over-read pad][mbarriers][index slots][item + claim slots]
     if (smem_addr(smem) != kSmemBase) {   // the lookups' address arithmetic would be wrong: refuse to run
-        if (threadIdx.x == 0) atomicOr(control + 1, kStatInternal);
+        if (threadIdx.x == 0) {
+            atomicOr(control + 1, kStatInternal);
+            cta_finished(control);
+        }
         return;
     }
     DecodeAux* s_aux = aux_ptr<K>();
@@ -136,26 +173,13 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                 uint32_t* s3 = reinterpret_cast<uint32_t*>(smem + (17u << K));
                 for (uint32_t i = threadIdx.x; i < (uint32_t)kExpEntriesMin; i += blockDim.x) s3[i] = __ldg(tt->exp_small + i);
             } else {
-                // cell-major copies, 64 KB in all: word w holds cell w / copies
-                const uint32_t shift = 9u - __ldg(&tt->aux.expm);       // log2 of the number of copies
-                if (shift >= 2u) {
-                    // four or more copies: the four words of a 16-byte store belong to one cell
-                    uint4* s4 = reinterpret_cast<uint4*>(smem);
-                    for (uint32_t q = threadIdx.x; q < (uint32_t)kExpEntriesMax / 4u; q += blockDim.x) {
-                        const uint32_t v = __ldg(tt->exp_lut() + ((4u * q) >> shift));
-                        s4[q] = make_uint4(v, v, v, v);
-                    }
-                } else {
-                    uint32_t* s1 = reinterpret_cast<uint32_t*>(smem);
-                    for (uint32_t w = threadIdx.x; w < (uint32_t)kExpEntriesMax; w += blockDim.x)
-                        s1[w] = __ldg(tt->exp_lut() + (w >> shift));
-                }
+                load_exp_table(tt);
             }
             __syncthreads();
         }
         const DevTensor& T = *s_tensor;
-        const uint32_t chunks_per_item = T.item_chunks;
-        const uint32_t first = (item - __ldg(item_start + cur)) * chunks_per_item;
+        const uint32_t first = (item - __ldg(item_start + cur)) * T.item_chunks;
+        const uint32_t count = min(T.item_chunks, T.n_chunks - first);   // chunks of this item
 
         // The warps share out the item's chunks.  Each warp, per turn: start the bulk copy of
         // chunk i + 1 (its offsets arrived a turn ago), work out the lanes' positions in chunk
@@ -164,7 +188,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             uint32_t k = 0;
             if (lane == 0) k = atomicAdd(&s_claim[slot], 1u);
             k = __shfl_sync(0xffffffffu, k, 0);
-            return k < min(chunks_per_item, T.n_chunks - first) ? first + k : kNone;
+            return k < count ? first + k : kNone;
         };
         Ready r0;
         r0.c = kNone;
@@ -179,7 +203,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             __syncwarp();                           // every lane has read the slot before it is refilled
             c2 = r1.c == kNone ? kNone : claim();
             fetch_index(T, c2, other, lane);
-            decode_finish<K, kSink>(cx, status, r0, L, lane);
+            decode_finish<K, kSink>(cx, status, r0, L, lane, stage_bytes);
             if (r1.c == kNone) break;
             r0 = r1;
             sp = other;
@@ -195,6 +219,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     // A warp that gave up on a bulk copy lets it land (bounded) before its buffer goes away.
     const uint32_t issued = cx.state & 0x7fffffffu;
     if (cx.dead() && issued) (void)mbar_wait(cx.bar + 8u * ((issued - 1) & 1u), ((issued - 1) >> 1) & 1u);
+    if (threadIdx.x == 0) cta_finished(control);
 }
 
 struct Shape {
@@ -392,7 +417,6 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
                                    int sink = kSinkFp16)
 {
     const DecodeConfig cfg = config_for(decode_config(), descs, ntensors, ws->max_smem_optin);
-    ItemPlan plan = plan_items(cfg, descs, ntensors, ws->sm_count);
     int live = 0;
     for (int i = 0; i < ntensors; ++i) {
         entro_status st = validate_desc(descs[i]);
@@ -400,6 +424,7 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
         if (descs[i].n) live++;
     }
     if (live == 0) return ENTRO_OK;
+    ItemPlan plan = plan_items(cfg, descs, ntensors, ws->sm_count);
 
     const size_t tensors_bytes = (size_t)live * sizeof(DevTensor);
     const size_t items_bytes = (((size_t)live + 1) * 4 + 15) & ~(size_t)15;
@@ -579,17 +604,6 @@ extern "C" entro_status entro_decode_dequant_batched_host(const entro_tensor_des
 namespace entro {
 namespace {
 
-// y = fp16(y32) for every tensor of a fused call.
-__global__ void __launch_bounds__(256) gemv_finalize_kernel(const GemvTensor* __restrict__ g, int ntensors)
-{
-    for (int t = blockIdx.y; t < ntensors; t += gridDim.y) {
-        const GemvTensor G = g[t];
-        const uint32_t n = G.rows * G.batch;      // both are [batch][rows]
-        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
-            G.y[i] = __half_as_ushort(__float2half_rn(G.y32[i]));
-    }
-}
-
 // Plain fp16 matrix-vector product (the step that follows an unfused decode): one warp per
 // row, 16-byte loads, fp32 products and sums, x read through the read-only path.
 __global__ void __launch_bounds__(256) gemv_fp16_kernel(const uint16_t* __restrict__ w, uint32_t rows, uint32_t cols,
@@ -621,16 +635,27 @@ __global__ void __launch_bounds__(256) gemv_fp16_kernel(const uint16_t* __restri
 }  // namespace
 }  // namespace entro
 
-extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs_host, const entro_gemv_io* io_host,
-                                                  int ntensors, void* cuda_stream)
+namespace entro {
+namespace {
+
+// Sizes and places of everything a fused matrix-vector call keeps on the device:
+// [DevTensor x n][item_start][GemvTensor x n] (uploaded) [tables x n][fp32 sums][counts of pending parts].
+struct GemvLayout {
+    int n = 0;
+    uint32_t lanes_batch = 1;        // accumulators per lane: the largest batch rounded up to 1, 2, 4 or 8
+    uint32_t x_bytes = 0;            // shared memory for x of that many tokens
+    size_t tensors_at = 0, items_at = 0, gemv_at = 0, upload_bytes = 0;
+    size_t tables_at = 0, y32_at = 0, pending_at = 0, total_bytes = 0;
+};
+
+entro_status gemv_layout(const entro_tensor_desc* descs, const entro_gemv_io* io, int ntensors, GemvLayout& L)
 {
-    if (ntensors < 0 || (ntensors > 0 && (!descs_host || !io_host))) return ENTRO_ERR_INVALID_ARG;
-    if (ntensors == 0) return ENTRO_OK;
-    uint64_t total_rows = 0;
+    if (ntensors < 0 || (ntensors > 0 && (!descs || !io))) return ENTRO_ERR_INVALID_ARG;
+    uint64_t sum_rows = 0, sum_batch_rows = 0;
     uint32_t max_batch = 1;
     for (int i = 0; i < ntensors; ++i) {
-        const entro_tensor_desc& d = descs_host[i];
-        const entro_gemv_io& g = io_host[i];
+        const entro_tensor_desc& d = descs[i];
+        const entro_gemv_io& g = io[i];
         if (d.n == 0) return ENTRO_ERR_INVALID_ARG;
         entro_status st = validate_desc(d, false);
         if (st != ENTRO_OK) return st;
@@ -640,71 +665,170 @@ extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs
         if (g.batch < 1 || g.batch > ENTRO_GEMV_MAX_BATCH || g.reserved != 0) return ENTRO_ERR_INVALID_ARG;
         if ((uint64_t)g.rows * g.batch > 0xffffffffull) return ENTRO_ERR_UNSUPPORTED;
         if (g.cols % 256u || (uint64_t)g.cols * g.batch > kGemvMaxX || d.chunk_symbols % 256u) return ENTRO_ERR_UNSUPPORTED;
-        total_rows += (uint64_t)g.rows * g.batch;
+        sum_rows += g.rows;
+        sum_batch_rows += (uint64_t)g.rows * g.batch;
         if (g.batch > max_batch) max_batch = g.batch;
     }
-    // accumulators per lane: the batch rounded up to 1, 2, 4 or 8; x of that many tokens is staged
-    const uint32_t lanes_batch = max_batch <= 1 ? 1u : max_batch <= 2 ? 2u : max_batch <= 4 ? 4u : 8u;
-    uint32_t x_bytes = 0;
+    L.n = ntensors;
+    L.lanes_batch = max_batch <= 1 ? 1u : max_batch <= 2 ? 2u : max_batch <= 4 ? 4u : 8u;
+    L.x_bytes = 0;
     for (int i = 0; i < ntensors; ++i) {
-        const uint32_t need = (io_host[i].cols * lanes_batch * 2u + 127u) & ~127u;
-        if (need > x_bytes) x_bytes = need;
+        const uint32_t need = (io[i].cols * L.lanes_batch * 2u + 127u) & ~127u;
+        if (need > L.x_bytes) L.x_bytes = need;
     }
-    if (x_bytes > 2u * kGemvMaxX) return ENTRO_ERR_UNSUPPORTED;   // a wide matrix beside a larger batch elsewhere in the call
+    if (L.x_bytes > 2u * kGemvMaxX) return ENTRO_ERR_UNSUPPORTED;   // a wide matrix beside a larger batch elsewhere in the call
+    auto up16 = [](size_t v) { return (v + 15) & ~(size_t)15; };
+    size_t at = 0;
+    L.tensors_at = at, at += (size_t)ntensors * sizeof(DevTensor);
+    L.items_at = at, at += up16(((size_t)ntensors + 1) * 4);
+    L.gemv_at = at, at += (size_t)ntensors * sizeof(GemvTensor);
+    L.upload_bytes = at;
+    L.tables_at = at, at += (size_t)ntensors * sizeof(TensorTables);
+    L.y32_at = at, at += up16(sum_batch_rows * 4);
+    L.pending_at = at, at += up16(sum_rows * 4);
+    L.total_bytes = at;
+    return ENTRO_OK;
+}
+
+// Fills the upload area (host copy at `host`, to live at `dev` on the device); -> number of
+// work items, or 0 if there are too many.
+uint64_t gemv_fill(const GemvLayout& L, const DecodeConfig& cfg, int sm_count, const entro_tensor_desc* descs,
+                   const entro_gemv_io* io, char* host, char* dev)
+{
+    ItemPlan plan = plan_items(cfg, descs, L.n, sm_count);
+    DevTensor* ht = reinterpret_cast<DevTensor*>(host + L.tensors_at);
+    uint32_t* hitems = reinterpret_cast<uint32_t*>(host + L.items_at);
+    GemvTensor* hg = reinterpret_cast<GemvTensor*>(host + L.gemv_at);
+    float* y32 = reinterpret_cast<float*>(dev + L.y32_at);
+    uint32_t* pending = reinterpret_cast<uint32_t*>(dev + L.pending_at);
+    uint64_t items = 0, row0 = 0, brow0 = 0;
+    for (int i = 0; i < L.n; ++i) {
+        hitems[i] = (uint32_t)items;
+        items += fill_dev_tensor(descs[i], plan, ht[i]);
+        if (items > 0x7fffffffull) return 0;
+        hg[i].x = static_cast<const uint16_t*>(io[i].x_fp16_dev);
+        hg[i].y32 = y32 + brow0;
+        hg[i].y = static_cast<uint16_t*>(io[i].y_fp16_dev);
+        hg[i].rows = io[i].rows;
+        hg[i].cols = io[i].cols;
+        hg[i].batch = io[i].batch;
+        hg[i].pad = 0;
+        hg[i].pending = pending + row0;
+        row0 += io[i].rows;
+        brow0 += (uint64_t)io[i].rows * io[i].batch;
+    }
+    hitems[L.n] = (uint32_t)items;
+    return items;
+}
+
+}  // namespace
+}  // namespace entro
+
+extern "C" entro_status entro_decode_dequant_gemv(const entro_tensor_desc* descs_host, const entro_gemv_io* io_host,
+                                                  int ntensors, void* cuda_stream)
+{
+    GemvLayout L;
+    entro_status st = gemv_layout(descs_host, io_host, ntensors, L);
+    if (st != ENTRO_OK) return st;
+    if (ntensors == 0) return ENTRO_OK;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     Guard guard;
     Workspace* ws = workspace();
     if (!ws) return ENTRO_ERR_CUDA;
     const DecodeConfig cfg = decode_config();
-    ItemPlan plan = plan_items(cfg, descs_host, ntensors, ws->sm_count);
-
-    // workspace: [DevTensor x n][item_start][GemvTensor x n] (uploaded) [tables x n][y32]
-    const size_t tensors_bytes = (size_t)ntensors * sizeof(DevTensor);
-    const size_t items_bytes = (((size_t)ntensors + 1) * 4 + 15) & ~(size_t)15;
-    const size_t gemv_bytes = (size_t)ntensors * sizeof(GemvTensor);
-    const size_t upload_bytes = tensors_bytes + items_bytes + gemv_bytes;
-    const size_t tables_bytes = (size_t)ntensors * sizeof(TensorTables);
-    const size_t y32_bytes = (total_rows * 4 + 15) & ~(size_t)15;
-    if (!reserve_pinned(ws, upload_bytes)) return ENTRO_ERR_CUDA;
-    if (!reserve_device(ws, upload_bytes + tables_bytes + y32_bytes)) return ENTRO_ERR_CUDA;
+    if (!reserve_pinned(ws, L.upload_bytes)) return ENTRO_ERR_CUDA;
+    if (!reserve_device(ws, L.total_bytes)) return ENTRO_ERR_CUDA;
     char* base = static_cast<char*>(ws->dev);
-    char* hbase = static_cast<char*>(ws->pinned);
-    DevTensor* ht = reinterpret_cast<DevTensor*>(hbase);
-    uint32_t* hitems = reinterpret_cast<uint32_t*>(hbase + tensors_bytes);
-    GemvTensor* hg = reinterpret_cast<GemvTensor*>(hbase + tensors_bytes + items_bytes);
-    float* y32 = reinterpret_cast<float*>(base + upload_bytes + tables_bytes);
-    uint64_t items = 0, row0 = 0;
-    for (int i = 0; i < ntensors; ++i) {
-        hitems[i] = (uint32_t)items;
-        items += fill_dev_tensor(descs_host[i], plan, ht[i]);
-        if (items > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
-        hg[i].x = static_cast<const uint16_t*>(io_host[i].x_fp16_dev);
-        hg[i].y32 = y32 + row0;
-        hg[i].y = static_cast<uint16_t*>(io_host[i].y_fp16_dev);
-        hg[i].rows = io_host[i].rows;
-        hg[i].cols = io_host[i].cols;
-        hg[i].batch = io_host[i].batch;
-        hg[i].pad[0] = hg[i].pad[1] = hg[i].pad[2] = 0;
-        row0 += (uint64_t)io_host[i].rows * io_host[i].batch;
-    }
-    hitems[ntensors] = (uint32_t)items;
-    DevTensor* dt = reinterpret_cast<DevTensor*>(base);
-    uint32_t* ditems = reinterpret_cast<uint32_t*>(base + tensors_bytes);
-    GemvTensor* dg = reinterpret_cast<GemvTensor*>(base + tensors_bytes + items_bytes);
-    TensorTables* dtables = reinterpret_cast<TensorTables*>(base + upload_bytes);
-    ENTRO_CUDA(cudaMemcpyAsync(dt, ht, upload_bytes, cudaMemcpyHostToDevice, s));
+    const uint64_t items = gemv_fill(L, cfg, ws->sm_count, descs_host, io_host, static_cast<char*>(ws->pinned), base);
+    if (items == 0) return ENTRO_ERR_UNSUPPORTED;
+    DevTensor* dt = reinterpret_cast<DevTensor*>(base + L.tensors_at);
+    GemvTensor* dg = reinterpret_cast<GemvTensor*>(base + L.gemv_at);
+    TensorTables* dtables = reinterpret_cast<TensorTables*>(base + L.tables_at);
+    ENTRO_CUDA(cudaMemcpyAsync(base, ws->pinned, L.upload_bytes, cudaMemcpyHostToDevice, s));
     mark_pinned_in_use(ws, s);
     build_tables_kernel<<<dim3((unsigned)ntensors, table_slices(ntensors, ws->sm_count)), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control, dg);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
-    entro_status st = launch_decode_any(ws, cfg, dt, ntensors, ditems, (uint32_t)items, dtables, s, dg, kSinkGemv,
-                                        (int)lanes_batch, x_bytes);
+    return launch_decode_any(ws, cfg, dt, ntensors, reinterpret_cast<uint32_t*>(base + L.items_at), (uint32_t)items,
+                             dtables, s, dg, kSinkGemv, (int)L.lanes_batch, L.x_bytes);
+}
+
+// ------------------------------------------------------------------ prepared matrix-vector products
+
+struct entro_gemv_plan {
+    int device = -1;
+    GemvLayout L;
+    DecodeConfig cfg;
+    char* dev = nullptr;
+    uint32_t items = 0;
+};
+
+extern "C" entro_status entro_gemv_prepare(const entro_tensor_desc* descs_host, const entro_gemv_io* io_host,
+                                           int ntensors, void* cuda_stream, entro_gemv_plan** plan_out)
+{
+    if (!plan_out) return ENTRO_ERR_INVALID_ARG;
+    *plan_out = nullptr;
+    if (ntensors <= 0) return ENTRO_ERR_INVALID_ARG;
+    Guard guard;
+    Workspace* ws = workspace();
+    if (!ws) return ENTRO_ERR_CUDA;
+    const DecodeConfig cfg = decode_config();
+    GemvLayout L;
+    entro_status st = gemv_layout(descs_host, io_host, ntensors, L);
     if (st != ENTRO_OK) return st;
-    dim3 grid(16, (unsigned)(ntensors < 64 ? ntensors : 64));
-    gemv_finalize_kernel<<<grid, 256, 0, s>>>(dg, ntensors);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    entro_gemv_plan* plan = new (std::nothrow) entro_gemv_plan;
+    if (!plan) return ENTRO_ERR_CUDA;
+    plan->device = ws->device;
+    plan->L = L;
+    plan->cfg = cfg;
+    void* host = nullptr;
+    auto fail = [&](entro_status why) {
+        if (host) cudaFreeHost(host);
+        if (plan->dev) cudaFree(plan->dev);
+        delete plan;
+        return why;
+    };
+    if (cudaMalloc(reinterpret_cast<void**>(&plan->dev), L.total_bytes) != cudaSuccess) return fail(ENTRO_ERR_CUDA);
+    if (cudaMallocHost(&host, L.upload_bytes) != cudaSuccess) return fail(ENTRO_ERR_CUDA);
+    const uint64_t items = gemv_fill(L, cfg, ws->sm_count, descs_host, io_host, static_cast<char*>(host), plan->dev);
+    if (items == 0) return fail(ENTRO_ERR_UNSUPPORTED);
+    plan->items = (uint32_t)items;
+    if (cudaMemcpyAsync(plan->dev, host, L.upload_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return fail(ENTRO_ERR_CUDA);
+    build_tables_kernel<<<dim3((unsigned)ntensors, table_slices(ntensors, ws->sm_count)), 256, 0, s>>>(
+        reinterpret_cast<DevTensor*>(plan->dev + L.tensors_at), cfg.lut_bits,
+        reinterpret_cast<TensorTables*>(plan->dev + L.tables_at), ws->control,
+        reinterpret_cast<GemvTensor*>(plan->dev + L.gemv_at));
     count_launch();
-    ENTRO_CUDA(cudaGetLastError());
+    if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return fail(ENTRO_ERR_CUDA);
+    cudaFreeHost(host);
+    *plan_out = plan;
     return ENTRO_OK;
+}
+
+extern "C" entro_status entro_gemv_run(entro_gemv_plan* plan, void* cuda_stream)
+{
+    if (!plan || !plan->dev) return ENTRO_ERR_INVALID_ARG;
+    Guard guard;
+    Workspace* ws = workspace();
+    if (!ws) return ENTRO_ERR_CUDA;
+    if (ws->device != plan->device) return ENTRO_ERR_INVALID_ARG;
+    const GemvLayout& L = plan->L;
+    return launch_decode_any(ws, plan->cfg, reinterpret_cast<DevTensor*>(plan->dev + L.tensors_at), L.n,
+                             reinterpret_cast<uint32_t*>(plan->dev + L.items_at), plan->items,
+                             reinterpret_cast<TensorTables*>(plan->dev + L.tables_at), (cudaStream_t)cuda_stream,
+                             reinterpret_cast<GemvTensor*>(plan->dev + L.gemv_at), kSinkGemv, (int)L.lanes_batch,
+                             L.x_bytes);
+}
+
+extern "C" entro_status entro_gemv_release(entro_gemv_plan* plan)
+{
+    if (!plan) return ENTRO_OK;
+    Guard guard;
+    entro_status st = ENTRO_OK;
+    if (plan->dev && cudaFree(plan->dev) != cudaSuccess) st = ENTRO_ERR_CUDA;   // waits for kernels that still use it
+    delete plan;
+    return st;
 }
 
 extern "C" entro_status entro_gemv_fp16(const void* w_fp16_dev, uint32_t rows, uint32_t cols, const void* x_fp16_dev,
@@ -851,6 +975,29 @@ extern "C" entro_status entro_decode_dequant_static(const entro_tensor_desc* des
     if (status_dev)
         ENTRO_CUDA(cudaMemcpyAsync(status_dev, sc->control + 1, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
     return ENTRO_OK;
+}
+
+extern "C" int entro_checked_build(void)
+{
+#ifdef ENTRO_CHECKED
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+extern "C" long long entro_check_violations(void)
+{
+#ifdef ENTRO_CHECKED
+    Guard g;
+    unsigned int count = 0, zero = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    if (cudaMemcpyFromSymbol(&count, g_check_violations, sizeof(count)) != cudaSuccess) return -1;
+    if (cudaMemcpyToSymbol(g_check_violations, &zero, sizeof(zero)) != cudaSuccess) return -1;
+    return (long long)count;
+#else
+    return 0;
+#endif
 }
 
 extern "C" entro_status entro_set_decode_config(int lut_bits, int warps_per_cta, int ctas_per_sm, int chunks_per_item)

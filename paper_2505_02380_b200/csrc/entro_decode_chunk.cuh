@@ -101,6 +101,7 @@ __device__ __forceinline__ uint32_t ready_meta(uint32_t at, uint32_t bytes, uint
 
 __device__ __forceinline__ unsigned long long lds64(uint32_t addr)
 {
+    if (ENTRO_CHECK(smem_ok(addr, 8u))) return 0ull;
     unsigned long long v;
     asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(addr));
     return v;
@@ -111,6 +112,7 @@ __device__ __forceinline__ unsigned long long lds64(uint32_t addr)
 // held in registers while the copies are in flight.
 __device__ __forceinline__ void fetch_index(const DevTensor& T, uint32_t c, uint32_t slot, uint32_t lane)
 {
+    if (c != kNone && ENTRO_CHECK(c < T.n_chunks && smem_ok(slot, 16u) && smem_ok(slot + kSlotBytes - 16u, 16u))) c = kNone;
     if (c != kNone && lane < 20u) {
         // 4 bytes per lane: lanes 0..15 the sub-block lengths, lanes 16..19 the two offsets
         const char* src = lane < 16u ? reinterpret_cast<const char*>(T.sub_len + (uint64_t)c * kSubBlocks) + lane * 4u
@@ -120,9 +122,14 @@ __device__ __forceinline__ void fetch_index(const DevTensor& T, uint32_t c, uint
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
-__device__ __forceinline__ void issue_copy(const WarpCtx& cx, const DevTensor& T, Ready& r, uint64_t byte0, uint32_t lane)
+__device__ __forceinline__ void issue_copy(const WarpCtx& cx, const DevTensor& T, Ready& r, uint64_t byte0, uint32_t lane,
+                                           uint32_t stage_bytes)
 {
-    if (lane == 0)
+    // the copy lands inside this warp's ring, comes from inside the stream buffer, and both ends are 16-byte aligned
+    const bool bad = ENTRO_CHECK(r.at() + r.bytes() <= stage_bytes && smem_ok(cx.stage_addr + r.at(), 16u) &&
+                                 r.bytes() >= 16u && smem_ok(cx.stage_addr + r.at() + r.bytes() - 16u, 16u) &&
+                                 (byte0 & 15ull) == 0ull && byte0 + r.bytes() <= T.stream_words * 4ull);
+    if (lane == 0 && !bad)
         bulk_load(cx.stage_addr + r.at(), reinterpret_cast<const char*>(T.stream) + byte0, r.bytes(),
                   cx.bar + 8u * (r.ticket() & 1u));
     r.meta |= 1u << 28;
@@ -178,12 +185,28 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32
     }
     r.meta = ready_meta(at, bytes, cx.state, kStaged);
     cx.state++;
-    if (now) issue_copy(cx, T, r, byte0, lane);
+    if (now) issue_copy(cx, T, r, byte0, lane, stage_bytes);
     else if (lane == 0)   // no room yet: at least bring the bytes into L2 while the previous chunk is decoded
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const char*>(T.stream) + byte0),
                      "r"(bytes)
                      : "memory");
     return r;
+}
+
+// A chunk has added its part of a row that spans chunks to the row's fp32 sums.  The chunk
+// that brings the row's count of parts still to come to zero rounds the sums to fp16, and
+// leaves sums and count as the next call wants to find them (zero, and the full count).
+__device__ __forceinline__ void row_part_done(const GemvTensor* G, uint32_t row)
+{
+    __threadfence();                                   // this chunk's additions are visible before the count moves
+    const uint32_t before = atomicSub(G->pending + row, 1u);
+    if ((before & 0xffffu) != 1u) return;
+    __threadfence();
+    for (uint32_t b = 0; b < G->batch; ++b) {
+        const uint64_t at = (uint64_t)b * G->rows + row;
+        G->y[at] = __half_as_ushort(__float2half_rn(atomicExch(G->y32 + at, 0.f)));
+    }
+    G->pending[row] = (before >> 16) * 0x10001u;
 }
 
 // Any symbol count per lane, words fetched straight from global memory, one value at a
@@ -240,7 +263,7 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
                 if (i & 1u) reinterpret_cast<uint8_t*>(T.out)[(chunk_first + i) >> 1] = (uint8_t)(low | ((e >> 16) << 4));
                 else if (i + 1u == m) reinterpret_cast<uint8_t*>(T.out)[(chunk_first + i) >> 1] = (uint8_t)(e >> 16);
                 else low = (e >> 16) & 15u;
-            } else {
+            } else if (!ENTRO_CHECK(chunk_first + i < T.n)) {
                 out[i] = (uint16_t)(e >> 16);
             }
         }
@@ -254,12 +277,20 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
     }
     const uint64_t used = ((uint64_t)r.next << 5) - (uint64_t)r.nb - bit;
     if (used != my_bits) atomicOr(status, kStatCorrupt);
+    if (kB > 0) {
+        // every row the chunk touches has now got this chunk's part
+        __threadfence();
+        __syncwarp();
+        const uint32_t row0 = (uint32_t)(chunk_first / G->cols), row1 = (uint32_t)((chunk_first + m - 1u) / G->cols);
+        for (uint32_t row = row0 + lane; row <= row1; row += kSubBlocks) row_part_done(G, row);
+    }
 }
 
 // ------------------------------------------------------------------ what happens to decoded values
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr)
 {
+    if (ENTRO_CHECK(smem_ok(addr, 16u))) return make_uint4(0u, 0u, 0u, 0u);
     uint4 v;
     asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
@@ -272,11 +303,31 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
 struct OutCursor {
     const void* base;
     uint32_t off, end;
+#ifdef ENTRO_CHECKED
+    const char *lo, *hi;      // the output buffer of the tensor
+#endif
     __device__ __forceinline__ void start(void* lane_first, uint32_t steps, uint32_t stride)
     {
         base = lane_first;
         off = 0;
         end = steps * stride;
+    }
+    // Checked build: the tensor's output is [first, first + bytes); is a store of n bytes at p inside it?
+    __device__ __forceinline__ void bounds(const void* first, uint64_t bytes)
+    {
+#ifdef ENTRO_CHECKED
+        lo = static_cast<const char*>(first);
+        hi = lo + bytes;
+#endif
+    }
+    __device__ __forceinline__ bool outside(const void* p, uint32_t n) const
+    {
+#ifdef ENTRO_CHECKED
+        const char* c = static_cast<const char*>(p);
+        return ENTRO_CHECK(c >= lo && c + n <= hi && (reinterpret_cast<uintptr_t>(p) & (n - 1u)) == 0u);
+#else
+        return false;
+#endif
     }
     __device__ __forceinline__ bool more() const { return off != end; }
     __device__ __forceinline__ void* next(uint32_t stride)
@@ -293,7 +344,11 @@ struct OutCursor {
 struct EmitStore {
     OutCursor out;
     __device__ __forceinline__ bool more() const { return out.more(); }
-    __device__ __forceinline__ void operator()(uint4 v) { __stcs(static_cast<uint4*>(out.next(16u * kSubBlocks)), v); }
+    __device__ __forceinline__ void operator()(uint4 v)
+    {
+        uint4* p = static_cast<uint4*>(out.next(16u * kSubBlocks));
+        if (!out.outside(p, 16u)) __stcs(p, v);
+    }
     __device__ __forceinline__ void finish() {}
 };
 
@@ -304,8 +359,8 @@ struct EmitBytes {
     __device__ __forceinline__ bool more() const { return out.more(); }
     __device__ __forceinline__ void operator()(uint4 v)
     {
-        __stcs(static_cast<uint2*>(out.next(8u * kSubBlocks)),
-               make_uint2(__byte_perm(v.x, v.y, 0x6420), __byte_perm(v.z, v.w, 0x6420)));
+        uint2* p = static_cast<uint2*>(out.next(8u * kSubBlocks));
+        if (!out.outside(p, 8u)) __stcs(p, make_uint2(__byte_perm(v.x, v.y, 0x6420), __byte_perm(v.z, v.w, 0x6420)));
     }
 };
 
@@ -317,7 +372,8 @@ struct EmitNibbles {
     {
         const uint32_t a = __byte_perm(v.x, v.y, 0x6420), b = __byte_perm(v.z, v.w, 0x6420);   // s0..s3, s4..s7
         const uint32_t ta = a | (a >> 4), tb = b | (b >> 4);                                   // bytes 0 and 2 hold the pairs
-        __stcs(static_cast<uint32_t*>(out.next(4u * kSubBlocks)), __byte_perm(ta, tb, 0x6420));
+        uint32_t* p = static_cast<uint32_t*>(out.next(4u * kSubBlocks));
+        if (!out.outside(p, 4u)) __stcs(p, __byte_perm(ta, tb, 0x6420));
     }
 };
 
@@ -325,8 +381,9 @@ struct EmitNibbles {
 // cols a multiple of 256, so the 32 lanes of a step stay inside one row) and meet the 8
 // matching entries of x of every token, staged in shared memory as fp16 token after token
 // (tokens beyond the batch are zeros); products and sums in fp32, one accumulator per token.
-// When the row ends the warp adds its lanes up and adds the results to the row's fp32
-// accumulators.
+// When the row ends the warp adds its lanes up.  A row that began and ended inside this
+// chunk is complete: its sums are rounded to fp16 and stored.  A row that other chunks hold
+// parts of gets the sums added to its fp32 accumulators, and the last chunk to do so rounds.
 template <int B>
 struct EmitDot {
     uint32_t xaddr;       // shared-window address of x[0][col .. col + 8) for this lane's next group
@@ -335,23 +392,30 @@ struct EmitDot {
     uint32_t left;        // steps left in the current row
     uint32_t rs;          // steps per row (cols / 256)
     float acc[B];
-    float* yrow;          // fp32 accumulator of the current row, first token
-    uint32_t rows, batch;
+    const GemvTensor* G;  // in shared memory
+    uint32_t row;         // the current row
+    uint32_t began_before;   // 1: the current row began in an earlier chunk
     uint32_t lane;
     uint32_t todo;        // groups left in the lane's sub-block
     __device__ __forceinline__ bool more() const { return todo != 0u; }
 
-    __device__ __forceinline__ void flush()
+    __device__ __forceinline__ void flush(bool whole)
     {
 #pragma unroll
         for (int b = 0; b < B; ++b) {
             float v = acc[b];
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
-            if (lane == 0 && (uint32_t)b < batch) atomicAdd(yrow + (uint64_t)b * rows, v);
+            if (lane == 0 && (uint32_t)b < G->batch) {
+                const uint64_t at = (uint64_t)b * G->rows + row;
+                if (whole) G->y[at] = __half_as_ushort(__float2half_rn(v));
+                else atomicAdd(G->y32 + at, v);
+            }
             acc[b] = 0.f;
         }
-        ++yrow;
+        if (!whole && lane == 0) row_part_done(G, row);
+        ++row;
+        began_before = 0u;
         left = rs;
         xaddr = xlane;
     }
@@ -381,11 +445,11 @@ struct EmitDot {
         }
         xaddr += 512u;
         --todo;
-        if (--left == 0u) flush();
+        if (--left == 0u) flush(began_before == 0u);
     }
     __device__ __forceinline__ void finish()
     {
-        if (left != rs) flush();     // the chunk ended inside a row
+        if (left != rs) flush(false);     // the chunk ended inside a row
     }
 };
 
@@ -450,6 +514,7 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
             }
         }
         emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
+        if (ENTRO_CHECK(smem_ok(r.next, 4u))) break;      // the next word the reader would pull in
     }
     return cur_bit_addr(r);
 }
@@ -534,7 +599,8 @@ __device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status
 }
 
 template <int K, int kSink>
-__device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Ready& r, Lane L, uint32_t lane)
+__device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Ready& r, Lane L, uint32_t lane,
+                                              uint32_t stage_bytes)
 {
     constexpr int kBatch = kGemvBatchOf<kSink>;
     constexpr bool kGemv = kBatch > 0;
@@ -542,7 +608,7 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
     const DevTensor& T = *tensor_ptr<K>();
     const GemvTensor* G = kGemv ? gemv_ptr<K>() : nullptr;
     if (L.kind == kStaged) {
-        if (!r.issued()) issue_copy(cx, T, r, (T.offsets[r.c] >> 3) & ~15ull, lane);
+        if (!r.issued()) issue_copy(cx, T, r, (T.offsets[r.c] >> 3) & ~15ull, lane, stage_bytes);
         bool ok = mbar_wait(cx.bar + 8u * (r.ticket() & 1u), (r.ticket() >> 1) & 1u);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) {
@@ -575,24 +641,27 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         em.xstride = G->cols * 2u;
 #pragma unroll
         for (int b = 0; b < (kGemv ? kBatch : 1); ++b) em.acc[b] = 0.f;
-        em.yrow = G->y32 + row0;
-        em.rows = G->rows;
-        em.batch = G->batch;
+        em.G = G;
+        em.row = row0;
+        em.began_before = k0 != 0u;
         em.todo = sub >> 3;
         stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
         em.finish();
     } else if (kSink == kSinkBytes) {
         EmitBytes em;
         em.out.start(reinterpret_cast<uint8_t*>(T.out) + (uint64_t)r.c * T.chunk_symbols + lane * 8u, sub >> 3, 8u * kSubBlocks);
+        em.out.bounds(T.out, T.n);
         stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
     } else if (kSink == kSinkNibbles) {
         EmitNibbles em;
         em.out.start(reinterpret_cast<uint8_t*>(T.out) + (((uint64_t)r.c * T.chunk_symbols) >> 1) + lane * 4u, sub >> 3,
                      4u * kSubBlocks);
+        em.out.bounds(T.out, (T.n + 1u) >> 1);
         stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
     } else {
         EmitStore em;
         em.out.start(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u, sub >> 3, 16u * kSubBlocks);
+        em.out.bounds(T.out, T.n * 2u);
         stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
         em.finish();
     }

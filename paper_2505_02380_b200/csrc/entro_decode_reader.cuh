@@ -113,6 +113,7 @@ __device__ __forceinline__ uint32_t exp_lookup(LutKey key, uint32_t inv_window)
 {
     const uint32_t fb = __float_as_uint(__uint2float_rz(inv_window));
     const uint32_t a = ((fb >> 12) & key.mask) | key.lane;
+    if (ENTRO_CHECK(a < 4u * (uint32_t)kExpEntriesMax && (a & 3u) == 0u)) return kEscLen;
     return *reinterpret_cast<const uint32_t*>(smem + a);
 }
 
@@ -168,11 +169,27 @@ __device__ __forceinline__ uint32_t cur_bit_addr(const Cur& c) { return (c.next 
 // in, predicated.
 // If the group does not stand the caller repairs it from rewind_group, which needs only
 // pos, next and s.
+// Checked build: the cell's byte offset must lie inside the 64 KB of the table, else the
+// violation is counted and cell 0 is read instead.
+#ifdef ENTRO_CHECKED
+#define ENTRO_CELL_CHECK_AT(counter)                 \
+    "setp.gt.u32 q, a, 65532;\n\t"                    \
+    "@q red.global.add.u32 [" counter "], 1;\n\t"     \
+    "@q mov.b32 a, 0;\n\t"
+#define ENTRO_CELL_CHECK ENTRO_CELL_CHECK_AT("%10")
+#define ENTRO_CHECK_REGS ".reg .pred q;\n\t"
+#define ENTRO_CHECK_ARG , "l"(&g_check_violations)
+#else
+#define ENTRO_CELL_CHECK_AT(counter)
+#define ENTRO_CELL_CHECK
+#define ENTRO_CHECK_REGS
+#define ENTRO_CHECK_ARG
+#endif
 #define ENTRO_LOOKUP(dst, win)                       \
     "cvt.rz.f32.u32 f, " win ";\n\t"                  \
     "mov.b32 a, f;\n\t"                               \
     "shr.u32 a, a, 12;\n\t"                           \
-    "lop3.b32 a, a, %9, %8, 0xEA;\n\t"                \
+    "lop3.b32 a, a, %9, %8, 0xEA;\n\t" ENTRO_CELL_CHECK \
     "ld.shared.b32 " dst ", [a+1024];\n\t"
 #define ENTRO_OPEN                                   \
     "shf.l.wrap.b32 h, %1, %0, %2;\n\t"
@@ -192,7 +209,7 @@ __device__ __forceinline__ void group4(Cur& c, LutKey key, uint32_t& pk0, uint32
 {
     asm volatile(
         "{\n\t"
-        ".reg .pred p;\n\t"
+        ".reg .pred p;\n\t" ENTRO_CHECK_REGS
         ".reg .b32 t, w, a, h, e0, e1, e2, e3;\n\t"
         ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("e0", "h")
         "shf.l.wrap.b32 w, 0, h, e0;\n\t" ENTRO_LOOKUP("e1", "w")
@@ -204,7 +221,7 @@ __device__ __forceinline__ void group4(Cur& c, LutKey key, uint32_t& pk0, uint32
         "prmt.b32 %4, e0, e1, 0x7632;\n\t"
         "prmt.b32 %5, e2, e3, 0x7632;\n\t" ENTRO_MOVE_ON "}"
         : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk0), "=&r"(pk1), "=&r"(s), "+r"(c.w2)
-        : "r"(key.lane), "r"(key.mask));
+        : "r"(key.lane), "r"(key.mask) ENTRO_CHECK_ARG);
 }
 
 __device__ __forceinline__ void group2(Cur& c, LutKey key, uint32_t& pk0, uint32_t& s)
@@ -212,7 +229,7 @@ __device__ __forceinline__ void group2(Cur& c, LutKey key, uint32_t& pk0, uint32
     __attribute__((unused)) uint32_t unused;   // operand slot of the second pair, which a group of two does not have
     asm volatile(
         "{\n\t"
-        ".reg .pred p;\n\t"
+        ".reg .pred p;\n\t" ENTRO_CHECK_REGS
         ".reg .b32 t, w, a, h, e0, e1;\n\t"
         ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("e0", "h")
         "shf.l.wrap.b32 w, 0, h, e0;\n\t" ENTRO_LOOKUP("e1", "w")
@@ -220,7 +237,7 @@ __device__ __forceinline__ void group2(Cur& c, LutKey key, uint32_t& pk0, uint32
         "prmt.b32 %4, e0, e1, 0x7632;\n\t"
         "mov.b32 %5, 0;\n\t" ENTRO_MOVE_ON "}"
         : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk0), "=&r"(unused), "=&r"(s), "+r"(c.w2)
-        : "r"(key.lane), "r"(key.mask));
+        : "r"(key.lane), "r"(key.mask) ENTRO_CHECK_ARG);
 }
 // Three lookups, for the streams whose groups of four would too often need 32 bits or more.
 // Eight symbols go out as 3 + 3 + 2, so the pairs of values straddle the groups: with kTail
@@ -232,7 +249,7 @@ __device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint
     if (!kTail)
         asm volatile(
             "{\n\t"
-            ".reg .pred p;\n\t"
+            ".reg .pred p;\n\t" ENTRO_CHECK_REGS
             ".reg .b32 t, w, a, h, e0, e1;\n\t"
             ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("e0", "h")
             "shf.l.wrap.b32 w, 0, h, e0;\n\t" ENTRO_LOOKUP("e1", "w")
@@ -241,11 +258,11 @@ __device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint
             "add.u32 %6, %6, %5;\n\t"
             "prmt.b32 %4, e0, e1, 0x7632;\n\t" ENTRO_MOVE_ON "}"
             : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s), "+r"(c.w2)
-            : "r"(key.lane), "r"(key.mask));
+            : "r"(key.lane), "r"(key.mask) ENTRO_CHECK_ARG);
     else
         asm volatile(
             "{\n\t"
-            ".reg .pred p;\n\t"
+            ".reg .pred p;\n\t" ENTRO_CHECK_REGS
             ".reg .b32 t, w, a, h, e1, e2;\n\t"
             ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP("%4", "h")
             "shf.l.wrap.b32 w, 0, h, %4;\n\t" ENTRO_LOOKUP("e1", "w")
@@ -254,7 +271,7 @@ __device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint
             "add.u32 %6, %6, e2;\n\t"
             "prmt.b32 %5, e1, e2, 0x7632;\n\t" ENTRO_MOVE_ON "}"
             : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(first), "=&r"(second), "=&r"(s), "+r"(c.w2)
-            : "r"(key.lane), "r"(key.mask));
+            : "r"(key.lane), "r"(key.mask) ENTRO_CHECK_ARG);
 }
 // Eight lookups on one view, for streams of so few bits per symbol (at most 2) that eight
 // codes almost always fit 32 bits: 4-bit alphabets beyond the reach of the eight-symbol table.
@@ -262,7 +279,7 @@ __device__ __forceinline__ void group3(Cur& c, LutKey key, uint32_t& first, uint
     "cvt.rz.f32.u32 f, " win ";\n\t"                  \
     "mov.b32 a, f;\n\t"                               \
     "shr.u32 a, a, 12;\n\t"                           \
-    "lop3.b32 a, a, %11, %10, 0xEA;\n\t"              \
+    "lop3.b32 a, a, %11, %10, 0xEA;\n\t" ENTRO_CELL_CHECK_AT("%12") \
     "ld.shared.b32 " dst ", [a+1024];\n\t"
 #define ENTRO_NEXT8(e)                               \
     "add.u32 %6, %6, " e ";\n\t"                      \
@@ -271,7 +288,7 @@ __device__ __forceinline__ void group8(Cur& c, LutKey key, uint4& pk, uint32_t& 
 {
     asm volatile(
         "{\n\t"
-        ".reg .pred p;\n\t"
+        ".reg .pred p;\n\t" ENTRO_CHECK_REGS
         ".reg .b32 t, w, a, h, e0, e1, e2, e3, e4, e5, e6, e7;\n\t"
         ".reg .f32 f;\n\t" ENTRO_OPEN ENTRO_LOOKUP8("e0", "h")
         "shf.l.wrap.b32 w, 0, h, e0;\n\t" ENTRO_LOOKUP8("e1", "w")
@@ -286,11 +303,15 @@ __device__ __forceinline__ void group8(Cur& c, LutKey key, uint4& pk, uint32_t& 
         "prmt.b32 %9, e6, e7, 0x7632;\n\t" ENTRO_MOVE_ON "}"
         : "+r"(c.w0), "+r"(c.w1), "+r"(c.pos), "+r"(c.next), "=&r"(pk.x), "=&r"(pk.y), "=&r"(s), "+r"(c.w2), "=&r"(pk.z),
           "=&r"(pk.w)
-        : "r"(key.lane), "r"(key.mask));
+        : "r"(key.lane), "r"(key.mask) ENTRO_CHECK_ARG);
 }
 #undef ENTRO_LOOKUP8
 #undef ENTRO_NEXT8
 #undef ENTRO_LOOKUP
+#undef ENTRO_CELL_CHECK
+#undef ENTRO_CELL_CHECK_AT
+#undef ENTRO_CHECK_REGS
+#undef ENTRO_CHECK_ARG
 #undef ENTRO_OPEN
 #undef ENTRO_MOVE_ON
 

@@ -49,10 +49,17 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
     TensorTables& out = tables[t];
     const uint32_t first = blockIdx.y * 256u + (uint32_t)tid, stride = gridDim.y * 256u;   // this thread's entries
     if (t == 0 && first == 0) control[0] = 0;   // work counter of the decode kernel that follows
-    if (gemv) {                                 // and the fp32 sums of the fused matrix-vector products
-        float* y32 = gemv[t].y32;
-        const uint32_t n = gemv[t].rows * gemv[t].batch;
-        for (uint32_t i = first; i < n; i += stride) y32[i] = 0.f;
+    if (gemv) {
+        // the fused matrix-vector products: fp32 sums of the rows that span chunks start at zero,
+        // and every row is told how many chunks hold a part of it
+        const GemvTensor& G = gemv[t];
+        const uint32_t n = G.rows * G.batch;
+        for (uint32_t i = first; i < n; i += stride) G.y32[i] = 0.f;
+        for (uint32_t r = first; r < G.rows; r += stride) {
+            const uint64_t a = (uint64_t)r * G.cols, b = a + G.cols - 1u;
+            const uint32_t parts = (uint32_t)(b / T.chunk_symbols - a / T.chunk_symbols) + 1u;
+            G.pending[r] = parts * 0x10001u;
+        }
     }
     if (tid <= ENTRO_MAX_CODE_LEN) count[tid] = 0;
     len[tid] = (uint32_t)tid < T.nsym ? T.len[tid] : 0;

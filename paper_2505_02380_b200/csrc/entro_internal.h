@@ -44,11 +44,12 @@ static_assert(sizeof(DevTensor) % 16 == 0, "DevTensor is copied as 16-byte vecto
 // The matrix-vector side of one tensor for the fused decode + GEMV kernel.
 struct GemvTensor {
     const uint16_t* x;    // [batch][cols] fp16 values
-    float* y32;           // [batch][rows] fp32 accumulators (workspace), zeroed by the table build
+    float* y32;           // [batch][rows] fp32 accumulators of the rows that span chunks (workspace); zero between calls
     uint16_t* y;          // [batch][rows] fp16 results
     uint32_t rows, cols;
     uint32_t batch;       // tokens, 1 .. ENTRO_GEMV_MAX_BATCH
-    uint32_t pad[3];
+    uint32_t pad;
+    uint32_t* pending;    // [rows] chunks that hold part of the row: expected << 16 | still to come
 };
 static_assert(sizeof(GemvTensor) == 48, "GemvTensor is read as three 16-byte vectors");
 constexpr uint32_t kGemvMaxX = 32768;         // fp16 values of x (all tokens) staged in shared memory

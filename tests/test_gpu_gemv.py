@@ -39,6 +39,29 @@ from helpers import assert_status_ok, codebook_from_oracle, expected_out, to_dev
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["call", "plan"])
+def gemv(request):
+    """The fused products two ways: the one-shot call, and a plan prepared once and run twice
+    (first on other vectors, then, with x refreshed in place, on the ones the test gave: the
+    second run must not see anything the first one left in the plan's sums)."""
+    if request.param == "call":
+        return E.entro_decode_dequant_gemv
+
+    def via_plan(descs, xs, shapes):
+        xs = list(xs)
+        first = [torch.roll(x, 1, dims=-1) * 0.5 for x in xs]
+        bufs = [f.clone() for f in first]
+        plan, ys = E.entro_gemv_prepare(descs, bufs, shapes)
+        E.entro_gemv_run(plan)
+        for b, x in zip(bufs, xs):
+            b.copy_(x)
+        E.entro_gemv_run(plan)
+        torch.cuda.synchronize()
+        E.entro_gemv_release(plan)
+        return ys
+    return via_plan
+
+
 def _f16(bits_u16):
     return bits_u16.view(np.float16).astype(np.float64)
 
@@ -109,10 +132,10 @@ def _check_exact(y_gpu_u16, w_hat_u16, rows, cols, x_f16):
 
 @pytest.mark.parametrize("bits,chunk,rows,cols", [(4, 8192, 64, 512), (8, 4096, 64, 512), (4, 8192, 3, 1280),
                                                   (8, 4096, 37, 768), (4, 8192, 33, 4096), (4, 1024, 16, 256)])
-def test_fused_gemv_small(bits, chunk, rows, cols):
+def test_fused_gemv_small(gemv, bits, chunk, rows, cols):
     c, desc = _compressed(rows, cols, bits, chunk, 7000 + rows + cols)
     x = workloads.make_vector(cols, 11).cuda()
-    (y,) = E.entro_decode_dequant_gemv([desc], [x], [(rows, cols)])
+    (y,) = gemv([desc], [x], [(rows, cols)])
     torch.cuda.synchronize()
     assert_status_ok()
     _check(y.cpu().numpy().view(np.uint16), expected_out(c), rows, cols, x.cpu().numpy().view(np.uint16), chunk)
@@ -138,12 +161,12 @@ def test_unit_vector_reads_a_column_bit_exactly(bits, chunk):
 @pytest.mark.parametrize("bits,chunk,rows,cols,batch", [(4, 8192, 64, 512, 2), (8, 4096, 64, 512, 3), (4, 8192, 3, 1280, 4),
                                                         (8, 4096, 37, 768, 5), (4, 8192, 33, 4096, 8), (4, 1024, 16, 256, 7),
                                                         (8, 4096, 9, 14336, 2), (4, 8192, 40, 2048, 1)])
-def test_fused_gemv_small_batch(bits, chunk, rows, cols, batch):
+def test_fused_gemv_small_batch(gemv, bits, chunk, rows, cols, batch):
     """Every token of a batch is an independent product with the same weights: each row of
     the [batch, rows] result is checked against the oracle's product for that token."""
     c, desc = _compressed(rows, cols, bits, chunk, 7500 + rows + cols + batch)
     x = torch.stack([workloads.make_vector(cols, 300 + 17 * b) for b in range(batch)]).cuda()
-    (y,) = E.entro_decode_dequant_gemv([desc], [x], [(rows, cols)])
+    (y,) = gemv([desc], [x], [(rows, cols)])
     torch.cuda.synchronize()
     assert_status_ok()
     assert tuple(y.shape) == (batch, rows)
@@ -170,7 +193,7 @@ def test_batch_of_unit_vectors_reads_columns_bit_exactly():
     assert_status_ok()
 
 
-def test_one_call_with_different_batches_per_tensor():
+def test_one_call_with_different_batches_per_tensor(gemv):
     shapes, batches = [(32, 512), (8, 2048), (24, 256)], [3, 1, 8]
     cs, descs, xs = [], [], []
     for k, ((rows, cols), batch) in enumerate(zip(shapes, batches)):
@@ -179,7 +202,7 @@ def test_one_call_with_different_batches_per_tensor():
         descs.append(desc)
         x = torch.stack([workloads.make_vector(cols, 900 + 10 * k + b) for b in range(batch)]).cuda()
         xs.append(x if batch > 1 else x[0].contiguous())
-    ys = E.entro_decode_dequant_gemv(descs, xs, shapes)
+    ys = gemv(descs, xs, shapes)
     torch.cuda.synchronize()
     assert_status_ok()
     for c, (rows, cols), batch, x, y in zip(cs, shapes, batches, xs, ys):
@@ -207,12 +230,12 @@ def _mistral_layer():
     return wl, descs, shapes, refs, keep
 
 
-def test_mistral_shaped_layer_fused_and_unfused():
+def test_mistral_shaped_layer_fused_and_unfused(gemv):
     """The seven projections of one mistral-shaped layer (4-bit symbols, 8192-symbol chunks)
     in ONE fused call, against the oracle; and the plain fp16 GEMV on the decoded weights."""
     wl, descs, shapes, refs, _ = _mistral_layer()
     xs = [workloads.make_vector(cols, 100 + k).cuda() for k, (rows, cols) in enumerate(shapes)]
-    ys = E.entro_decode_dequant_gemv(descs, xs, shapes)
+    ys = gemv(descs, xs, shapes)
     torch.cuda.synchronize()
     assert_status_ok()
     for (rows, cols), y, x, ref in zip(shapes, ys, xs, refs):
@@ -223,7 +246,7 @@ def test_mistral_shaped_layer_fused_and_unfused():
         _check(y2.cpu().numpy().view(np.uint16), ref, rows, cols, x.cpu().numpy().view(np.uint16), wl.chunk_symbols)
 
 
-def test_mistral_shaped_layer_exact_sums_bit_for_bit():
+def test_mistral_shaped_layer_exact_sums_bit_for_bit(gemv):
     """Config 5 at its own shapes: the seven projections of a mistral-shaped layer (4-bit symbols,
     8192-symbol chunks; 4096 x 14336 down_proj rows span two or three chunks and are combined
     with atomics), one token and batches of 2, 4 and 8, with x chosen so that fp32 sums are exact
@@ -236,7 +259,7 @@ def test_mistral_shaped_layer_exact_sums_bit_for_bit():
         xs_np = [np.stack([_exact_x(shapes[k][1], wl.chunk_symbols, 50 * batch + 7 * k + b) for b in range(batch)])
                  for k in pick]
         xs = [torch.from_numpy(x if batch > 1 else x[0]).cuda() for x in xs_np]
-        ys = E.entro_decode_dequant_gemv([descs[k] for k in pick], xs, [shapes[k] for k in pick])
+        ys = gemv([descs[k] for k in pick], xs, [shapes[k] for k in pick])
         torch.cuda.synchronize()
         assert_status_ok()
         for k, x_np, y in zip(pick, xs_np, ys):
@@ -247,18 +270,36 @@ def test_mistral_shaped_layer_exact_sums_bit_for_bit():
 
 @pytest.mark.parametrize("bits,chunk,rows,cols,batch", [(8, 4096, 96, 14336, 1), (8, 4096, 96, 14336, 2), (8, 4096, 128, 4096, 4),
                                                         (4, 8192, 40, 2048, 8), (8, 1024, 33, 1280, 3), (4, 8192, 7, 14336, 1)])
-def test_exact_sums_bit_for_bit_other_shapes(bits, chunk, rows, cols, batch):
+def test_exact_sums_bit_for_bit_other_shapes(gemv, bits, chunk, rows, cols, batch):
     """The same at 8-bit symbols with 4096-symbol chunks (a 14336-column row spans four or five
     chunks), small chunks, and a tensor whose last chunk is ragged."""
     c, desc = _compressed(rows, cols, bits, chunk, 7800 + rows + cols)
     x_np = np.stack([_exact_x(cols, chunk, 900 + b) for b in range(batch)])
     x = torch.from_numpy(x_np if batch > 1 else x_np[0]).cuda()
-    (y,) = E.entro_decode_dequant_gemv([desc], [x], [(rows, cols)])
+    (y,) = gemv([desc], [x], [(rows, cols)])
     torch.cuda.synchronize()
     assert_status_ok()
     y_np = y.cpu().numpy().view(np.uint16).reshape(batch, rows)
     for b in range(batch):
         _check_exact(y_np[b], expected_out(c), rows, cols, x_np[b])
+
+
+def test_plan_argument_errors_and_release():
+    c, desc = _compressed(8, 512, 4, 8192, 7310)
+    x = torch.zeros(512, dtype=torch.float16, device="cuda")
+    with pytest.raises(E.EntroError) as e:
+        E.entro_gemv_prepare([desc], [x], [(16, 512)])                 # rows * cols != n
+    assert e.value.status == E.ERR_INVALID_ARG
+    L = E.lib()
+    assert L.entro_gemv_run(None, None) == E.ERR_INVALID_ARG
+    assert L.entro_gemv_release(None) == E.OK
+    plan, (y,) = E.entro_gemv_prepare([desc], [x], [(8, 512)])
+    E.entro_gemv_run(plan)
+    torch.cuda.synchronize()
+    assert_status_ok()
+    assert not y.cpu().numpy().any()                                    # W . 0 = 0
+    E.entro_gemv_release(plan)
+    E.entro_gemv_release(plan)                                          # a released handle is inert in the binding
 
 
 def test_gemv_argument_errors():

@@ -62,6 +62,40 @@ def test_static_entry_point_matches_batched_on_two_calls_in_a_row():
     _run_and_compare(second, 9100)
 
 
+def test_static_entry_point_with_chunks_larger_than_a_warps_ring():
+    """Flat 8-bit symbols in 8192-symbol chunks: a chunk is about 8 KB, more than the 5 KB of
+    shared memory a warp has in the usual launch shape.  Both entry points then launch fewer
+    warps with larger rings; their outputs must agree bit for bit and be the dequantised
+    symbols."""
+    chunk = 8192
+    rng = np.random.default_rng(9400)
+    keep, descs_a, descs_b, outs_a, outs_b, refs = [], [], [], [], [], []
+    for n in (5 * chunk + 31, 2 * chunk):
+        q = rng.integers(0, 256, n).astype(np.uint8)
+        ln = oracle.huffman_lengths(np.bincount(q, minlength=256).tolist())
+        cd = oracle.canonical_codes(ln)
+        enc = oracle.encode(q, ln, cd, chunk)
+        assert int(enc.offsets[1]) // 8 > 6000
+        s, ix = to_dev_stream(enc.stream), to_dev_index(enc)
+        cb = E.Codebook.from_lengths(ln.tolist(), cd.tolist())
+        a = torch.zeros(n, dtype=torch.float16, device="cuda")
+        b = torch.zeros(n, dtype=torch.float16, device="cuda")
+        keep += [s, ix]
+        descs_a.append(E.make_desc(s, ix, n, chunk, cb, 0.03125, 128, a))
+        descs_b.append(E.make_desc(s, ix, n, chunk, cb, 0.03125, 128, b))
+        outs_a.append(a)
+        outs_b.append(b)
+        refs.append(oracle.dequant(q, 0.03125, 128))
+    status = torch.full((1,), 77, dtype=torch.int32, device="cuda")
+    E.entro_decode_dequant_batched(descs_a)
+    E.entro_decode_dequant_static(descs_b, status)
+    torch.cuda.synchronize()
+    assert E.entro_last_device_status() == E.OK and int(status.item()) == 0
+    for a, b, ref in zip(outs_a, outs_b, refs):
+        assert np.array_equal(b.cpu().numpy().view(np.uint16), a.cpu().numpy().view(np.uint16))
+        assert np.array_equal(b.cpu().numpy().view(np.uint16), ref)
+
+
 def test_static_entry_point_reports_corruption_in_the_callers_word():
     n, chunk = 150_000, 4096
     c = oracle.compress(workloads.make_values(n, 0.02, 9200).numpy(), 8, chunk)
