@@ -407,9 +407,32 @@ def measure_other(E, name, steps, peak):
                         "frac": achieved / peak[0], "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS, "kernel_ms": k_ms,
                         "kernel_ms_min": float(np.min(kernel_ms))}}
     if in_l2:
+        # the timed calls above repeat one call, which finds descriptors and tables in place (one launch);
+        # two alternating calls (same tensor, two output buffers) rebuild them every time
+        import ctypes as C
+        out2 = torch.empty_like(model.out)
+        alt = (E.TensorDesc * len(model.descs))()
+        for i, d in enumerate(model.descs):
+            C.memmove(C.byref(alt[i]), C.byref(d), C.sizeof(E.TensorDesc))
+            alt[i].out_fp16_dev = out2.data_ptr() + (d.out_fp16_dev - model.out.data_ptr())
+        for _ in range(3):
+            E.entro_decode_dequant_batched(model.descs)
+            E.entro_decode_dequant_batched(alt)
+        torch.cuda.synchronize()
+        ev0.record()
+        for _ in range(steps):
+            E.entro_decode_dequant_batched(model.descs)
+            E.entro_decode_dequant_batched(alt)
+        ev1.record()
+        torch.cuda.synchronize()
+        assert E.entro_last_device_status() == E.OK and torch.equal(out2, model.out)
         out["us_per_call"] = 1e3 * step_ms
-        out["note"] = ("latency-bound: the whole tensor (%.1f MB of traffic) stays in L2 and the call is a handful of "
-                       "microseconds of launches; the roofline fraction is not a roofline point" % (model.algorithmic_bytes / 1e6))
+        out["us_per_call_tables_rebuilt"] = 1e3 * ev0.elapsed_time(ev1) / (2 * steps)
+        out["note"] = ("latency-bound: the whole tensor (%.1f MB of traffic) stays in L2 and a call is a handful of "
+                       "microseconds of launches, so the roofline fraction is not a roofline point.  us_per_call: the "
+                       "same call repeated (descriptors and tables found in place, one launch); "
+                       "us_per_call_tables_rebuilt: descriptor upload + table build + decode every call"
+                       % (model.algorithmic_bytes / 1e6))
     del model
     torch.cuda.empty_cache()
     return out

@@ -223,6 +223,12 @@ entro_status entro_decode_dequant(const uint32_t *stream_dev, uint64_t stream_wo
  * The same for a whole model in one pass: all tensors' chunks form one work list that a
  * persistent kernel consumes (the paper balances load by dealing many segments to each
  * thread, Section 3).  descs_host is read before the call returns.  Asynchronous.
+ * A call is: upload of the descriptors, construction of the per-tensor decode tables, the
+ * decode launch.  For calls of at most ENTRO_STATIC_MAX_TENSORS descriptors the library
+ * remembers the call: if the next call that uses its device area is the same call again
+ * (byte-identical descriptors, same launch shape), descriptors and tables are found in
+ * place and the call is the decode launch alone (a tensor decoded again and again, e.g. a
+ * layer materialised on demand).
  */
 entro_status entro_decode_dequant_batched(const entro_tensor_desc *descs_host, int ntensors,
                                           void *cuda_stream);

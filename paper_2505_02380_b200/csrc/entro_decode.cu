@@ -32,6 +32,7 @@
 //     codes in K bits); one unreplicated copy of the exponent-indexed table serves the
 //     symbol-by-symbol repair of such windows.
 //   aux   canonical ranges per length, for whatever the tables do not resolve.
+#include <cstring>
 #include <new>
 
 #include "entro_decode_chunk.cuh"
@@ -424,6 +425,23 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
         if (descs[i].n) live++;
     }
     if (live == 0) return ENTRO_OK;
+
+    // A repeat of the last call (few tensors, the very same descriptors, launch shape and
+    // sink, nothing else in the device area since): descriptors and tables are still in place,
+    // and the work counter is back at zero, so the decode launch is all there is to do.  (Tables
+    // are constants of a compressed tensor; only the choice of the decode mode looks at the
+    // device, at the stream's bit rate, and every mode decodes every stream.)
+    const bool few = ntensors <= Workspace::kKeptTensors;
+    if (few && ws->kept && ws->kept_ntensors == ntensors && ws->kept_sink == sink &&
+        memcmp(&ws->kept_cfg, &cfg, sizeof(cfg)) == 0 &&
+        memcmp(ws->kept_descs, descs, (size_t)ntensors * sizeof(entro_tensor_desc)) == 0) {
+        char* kept_base = static_cast<char*>(ws->dev);
+        const size_t kept_tensors_bytes = (size_t)ws->kept_live * sizeof(DevTensor);
+        const size_t kept_upload = kept_tensors_bytes + ((((size_t)ws->kept_live + 1) * 4 + 15) & ~(size_t)15);
+        return launch_decode_any(ws, cfg, reinterpret_cast<DevTensor*>(kept_base), ws->kept_live,
+                                 reinterpret_cast<uint32_t*>(kept_base + kept_tensors_bytes), ws->kept_items,
+                                 reinterpret_cast<TensorTables*>(kept_base + kept_upload), s, nullptr, sink);
+    }
     ItemPlan plan = plan_items(cfg, descs, ntensors, ws->sm_count);
 
     const size_t tensors_bytes = (size_t)live * sizeof(DevTensor);
@@ -456,7 +474,17 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     build_tables_kernel<<<dim3((unsigned)live, table_slices(live, ws->sm_count)), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control, nullptr);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
-    return launch_decode_any(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, s, nullptr, sink);
+    const entro_status st = launch_decode_any(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, s, nullptr, sink);
+    if (few && st == ENTRO_OK) {
+        ws->kept = true;
+        ws->kept_ntensors = ntensors;
+        ws->kept_live = live;
+        ws->kept_sink = sink;
+        ws->kept_items = (uint32_t)items;
+        ws->kept_cfg = cfg;
+        memcpy(ws->kept_descs, descs, (size_t)ntensors * sizeof(entro_tensor_desc));
+    }
+    return st;
 }
 
 }  // namespace entro

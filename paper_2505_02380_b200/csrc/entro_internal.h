@@ -121,6 +121,16 @@ struct Workspace {
     static constexpr int kCopyGroups = 48;
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_in[kCopyGroups] = {}, ev_dec[kCopyGroups] = {}, ev_edge = nullptr;
+    // What the device area holds if the last call that filled it was a batched decode of few
+    // tensors: the call's descriptors (host copy) and what its launch needs.  A repeat of that
+    // call finds descriptors and tables already in place and is one launch.  reserve_device
+    // (every call that fills the area goes through it) forgets it.
+    static constexpr int kKeptTensors = ENTRO_STATIC_MAX_TENSORS;
+    bool kept = false;
+    int kept_ntensors = 0, kept_live = 0, kept_sink = 0;
+    uint32_t kept_items = 0;
+    DecodeConfig kept_cfg;
+    entro_tensor_desc kept_descs[kKeptTensors];
     // optional timing of the decode kernel (entro_profile_begin / entro_profile_read)
     cudaEvent_t* prof_start = nullptr;
     cudaEvent_t* prof_stop = nullptr;

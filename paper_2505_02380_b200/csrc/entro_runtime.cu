@@ -38,6 +38,7 @@ Workspace* workspace()
 
 bool reserve_device(Workspace* ws, size_t bytes)
 {
+    ws->kept = false;      // the caller is about to overwrite the area
     if (bytes <= ws->dev_bytes) return true;
     if (ws->dev) {
         // cudaFree waits for work that may still use the old area.

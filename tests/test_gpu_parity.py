@@ -346,6 +346,41 @@ def _fib_counts(k, nsym):
     return fib[:k] + [0] * (nsym - k)
 
 
+def test_repeated_call_on_few_tensors_reuses_what_is_in_place():
+    """A batched decode of few tensors leaves descriptors and tables on the device; the same call
+    again is then only the decode launch.  Repeats, other tensors in between, and another user of
+    the library's device area in between (an encode) must all give the oracle's output."""
+    cases = []
+    for k, (bits, chunk, n) in enumerate([(8, 4096, 5 * 4096 + 77), (4, 8192, 3 * 8192), (8, 4096, 300_000)]):
+        w_np, _ = _values(n, 0.02, 6100 + k)
+        c = oracle.compress(w_np, bits, chunk)
+        s, ix = to_dev_stream(c.enc.stream), to_dev_index(c.enc)
+        out = torch.zeros(n, dtype=torch.float16, device="cuda")
+        cases.append((c, s, ix, out, E.make_desc(s, ix, n, chunk, codebook_from_oracle(c), c.qp.scale, c.qp.zero_point, out)))
+
+    def run(which):
+        descs = E.desc_array([cases[i][4] for i in which])
+        for i in which:
+            cases[i][3].zero_()
+        E.entro_decode_dequant_batched(descs)
+        torch.cuda.synchronize()
+        assert_status_ok()
+        for i in which:
+            assert np.array_equal(cases[i][3].cpu().numpy().view(np.uint16), expected_out(cases[i][0])), (which, i)
+
+    launches = E.entro_kernel_launch_count()
+    run([0, 1])
+    first = E.entro_kernel_launch_count() - launches
+    run([0, 1])                                            # the repeat
+    assert E.entro_kernel_launch_count() - launches == first + 1
+    run([2])                                               # other tensors
+    run([0, 1])
+    q = torch.from_numpy(cases[0][0].q).cuda()
+    E.entro_encode(q, codebook_from_oracle(cases[0][0]), 4096)       # writes the library's device area
+    run([0, 1])
+    run([0, 1])
+
+
 @pytest.mark.parametrize("k,nsym", [(31, 256), (33, 256), (16, 16), (12, 16)])
 def test_decode_long_codes(k, nsym):
     """Fibonacci histograms give code lengths up to k - 1 (32 at most): the lookup table's
