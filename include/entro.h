@@ -206,6 +206,48 @@ entro_status entro_encode(const uint8_t *q_dev, uint64_t n, const entro_codebook
                           void *cuda_stream);
 
 /*
+ * The offline stages for many tensors with one synchronisation per stage instead of several
+ * per tensor (a whole model is compressed in a fraction of a second).  Results are those of
+ * the per-tensor calls, bit for bit.
+ *
+ * entro_quantize_histogram_batched: for every job, the range of the tensor, (s, z) from it
+ * (computed on the device with the arithmetic stated at entro_quantize_tensor), the symbols
+ * q_dev, and their frequencies, counted in the pass that writes them.  qp_host[j] and
+ * counts_host[j * ENTRO_MAX_SYMBOLS .. + 2^bits) are filled on return (counts beyond 2^bits
+ * are 0).  ENTRO_ERR_NONFINITE if a tensor holds a NaN or an infinity (that tensor's q_dev is
+ * not written, its counts are 0; the other tensors are complete).
+ *
+ * entro_encode_batched: entro_encode for every job; total_bits_host[j] on return.
+ * ENTRO_ERR_BUFFER_TOO_SMALL if a stream does not fit its buffer (that stream is left
+ * zeroed), ENTRO_ERR_INVALID_ARG if a symbol has no code; the other tensors are complete.
+ */
+typedef struct {
+    const void *w_fp16_dev;   /* n fp16 weights, 16-byte aligned */
+    uint64_t n;
+    int32_t bits;             /* 4 or 8 */
+    int32_t mode;             /* entro_mode */
+    uint8_t *q_dev;           /* n bytes, 16-byte aligned */
+} entro_quantize_job;
+
+typedef struct {
+    const uint8_t *q_dev;     /* n symbols, 16-byte aligned */
+    uint64_t n;
+    const entro_codebook *cb_host;
+    uint32_t chunk_symbols;
+    uint32_t reserved;        /* 0 */
+    uint32_t *stream_dev;     /* 16-byte aligned */
+    uint64_t stream_cap_words;
+    void *index_dev;          /* 8-byte aligned */
+    uint64_t index_cap_bytes;
+} entro_encode_job;
+
+entro_status entro_quantize_histogram_batched(const entro_quantize_job *jobs_host, int njobs,
+                                              entro_qparams *qp_host, uint64_t *counts_host,
+                                              void *cuda_stream);
+entro_status entro_encode_batched(const entro_encode_job *jobs_host, int njobs, uint64_t *total_bits_host,
+                                  void *cuda_stream);
+
+/*
  * Parallel decode fused with dequantisation (Section 3, "Segmentation for parallel
  * Huffman decoding": every segment decodes independently from its known boundary; Eq. 1
  * inverted): out[i] = fp16_rne( s *_fp32 (float)(q[i] - z) ), q the decoded symbols in

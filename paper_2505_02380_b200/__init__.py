@@ -77,6 +77,17 @@ class GemvIO(C.Structure):
                 ("batch", C.c_uint32), ("reserved", C.c_uint32)]
 
 
+class QuantizeJob(C.Structure):
+    _fields_ = [("w_fp16_dev", C.c_void_p), ("n", C.c_uint64), ("bits", C.c_int32), ("mode", C.c_int32),
+                ("q_dev", C.c_void_p)]
+
+
+class EncodeJob(C.Structure):
+    _fields_ = [("q_dev", C.c_void_p), ("n", C.c_uint64), ("cb_host", C.POINTER(Codebook)), ("chunk_symbols", C.c_uint32),
+                ("reserved", C.c_uint32), ("stream_dev", C.c_void_p), ("stream_cap_words", C.c_uint64),
+                ("index_dev", C.c_void_p), ("index_cap_bytes", C.c_uint64)]
+
+
 class HostIO(C.Structure):
     _fields_ = [("stream_host", C.c_void_p), ("index_host", C.c_void_p), ("out_fp16_host", C.c_void_p)]
 
@@ -105,6 +116,9 @@ def lib():
         L.entro_index_bytes.restype = u64
         L.entro_index_bytes.argtypes = [u64, u32]
         L.entro_encode.argtypes = [vp, u64, C.POINTER(Codebook), u32, vp, u64, vp, u64, C.POINTER(C.c_uint64), vp]
+        L.entro_quantize_histogram_batched.argtypes = [C.POINTER(QuantizeJob), i32, C.POINTER(QParams),
+                                                       C.POINTER(C.c_uint64), vp]
+        L.entro_encode_batched.argtypes = [C.POINTER(EncodeJob), i32, C.POINTER(C.c_uint64), vp]
         L.entro_decode_dequant.argtypes = [vp, u64, vp, u64, u32, C.POINTER(Codebook), C.c_float, C.c_int32, vp, vp]
         L.entro_decode_dequant_batched.argtypes = [C.POINTER(TensorDesc), i32, vp]
         L.entro_decode_dequant_batched_host.argtypes = [C.POINTER(TensorDesc), C.POINTER(HostIO), i32, vp]
@@ -136,7 +150,8 @@ def lib():
 
 # Every symbol include/entro.h declares.
 EXPORTS = ["entro_quantize_tensor", "entro_quantize_blocks", "entro_histogram", "entro_build_codebook", "entro_build_codebook_limited", "entro_stream_words",
-           "entro_encode_bound_words", "entro_index_bytes", "entro_encode", "entro_decode_dequant",
+           "entro_encode_bound_words", "entro_index_bytes", "entro_encode", "entro_quantize_histogram_batched",
+           "entro_encode_batched", "entro_decode_dequant",
            "entro_decode_dequant_batched", "entro_decode_dequant_batched_host", "entro_decode_dequant_static",
            "entro_decode_dequant_gemv", "entro_gemv_prepare", "entro_gemv_run", "entro_gemv_release", "entro_gemv_fp16", "entro_decode_symbols_batched", "entro_last_device_status",
            "entro_set_decode_config", "entro_checked_build", "entro_check_violations", "entro_profile_begin", "entro_profile_read", "entro_kernel_launch_count",
@@ -257,6 +272,67 @@ def entro_encode(q: torch.Tensor, cb: Codebook, chunk_symbols: int, stream_words
     _check(lib().entro_encode(_dev(q, torch.uint8), n, C.byref(cb), chunk_symbols, sbuf.data_ptr(), cap,
                               ibuf.data_ptr(), ibytes, C.byref(total), _stream(stream)), "entro_encode")
     return Encoded(sbuf, ibuf, int(total.value), n, chunk_symbols)
+
+
+def entro_quantize_histogram_batched(ws: Sequence[torch.Tensor], bits: int, mode: int = MODE_AUTO,
+                                     stream: Optional[torch.cuda.Stream] = None,
+                                     qs: Optional[Sequence[torch.Tensor]] = None):
+    """Quantise every fp16 device tensor of ws and count its symbols, one synchronisation for all.
+    qs: the uint8 device tensors that receive the symbols (new ones if not given).
+    -> (qs, qps: list of QParams, counts: uint64 array [len(ws), 256])"""
+    n = len(ws)
+    if qs is None:
+        qs = [torch.empty(w.numel(), dtype=torch.uint8, device=w.device) for w in ws]
+    jobs = (QuantizeJob * n)()
+    for j, (w, q) in enumerate(zip(ws, qs)):
+        jobs[j] = QuantizeJob(_dev(w, torch.float16), w.numel(), bits, mode, q.data_ptr())
+    qps = (QParams * n)()
+    counts = np.zeros((n, MAX_SYMBOLS), dtype=np.uint64)
+    _check(lib().entro_quantize_histogram_batched(jobs, n, qps, counts.ctypes.data_as(C.POINTER(C.c_uint64)),
+                                                  _stream(stream)), "entro_quantize_histogram_batched")
+    return qs, list(qps), counts
+
+
+def entro_encode_batched(qs: Sequence[torch.Tensor], cbs: Sequence[Codebook], chunk_symbols: int,
+                         stream_words: Sequence[int], stream: Optional[torch.cuda.Stream] = None,
+                         bufs: Optional[Sequence] = None) -> List[Encoded]:
+    """entro_encode for every (q, codebook), one synchronisation for all.  stream_words[j]: capacity
+    of tensor j's stream buffer (entro_stream_words of its counts).  bufs[j] = (int32 stream tensor of
+    stream_words[j] words, uint8 index tensor of entro_index_bytes bytes) if the caller brings the
+    buffers (for instance slices of two large allocations)."""
+    n = len(qs)
+    jobs = (EncodeJob * n)()
+    given = bufs is not None
+    bufs = list(bufs) if given else []
+    for j, (q, cb) in enumerate(zip(qs, cbs)):
+        ibytes = entro_index_bytes(q.numel(), chunk_symbols)
+        if ibytes == 0:
+            raise EntroError(ERR_INVALID_ARG, "entro_index_bytes")
+        if given:
+            sbuf, ibuf = bufs[j]
+            assert sbuf.numel() == int(stream_words[j]) and ibuf.numel() == ibytes
+        else:
+            sbuf = torch.empty(int(stream_words[j]), dtype=torch.int32, device=q.device)
+            ibuf = torch.empty(ibytes, dtype=torch.uint8, device=q.device)
+            bufs.append((sbuf, ibuf))
+        jobs[j] = EncodeJob(_dev(q, torch.uint8), q.numel(), C.pointer(cb), chunk_symbols, 0, _dev(sbuf, torch.int32),
+                            sbuf.numel(), _dev(ibuf, torch.uint8), ibytes)
+    totals = (C.c_uint64 * n)()
+    _check(lib().entro_encode_batched(jobs, n, totals, _stream(stream)), "entro_encode_batched")
+    return [Encoded(sbuf, ibuf, int(totals[j]), qs[j].numel(), chunk_symbols) for j, (sbuf, ibuf) in enumerate(bufs)]
+
+
+def entro_stream_words_np(counts_row: np.ndarray, cb: Codebook) -> int:
+    """entro_stream_words on a row of the counts array of entro_quantize_histogram_batched."""
+    return int(lib().entro_stream_words(counts_row.ctypes.data_as(C.POINTER(C.c_uint64)), C.byref(cb)))
+
+
+def entro_build_codebook_np(counts_row: np.ndarray, nsym: int) -> Codebook:
+    """entro_build_codebook on a row of that counts array (no conversion to a list)."""
+    cb = Codebook()
+    _check(lib().entro_build_codebook(counts_row.ctypes.data_as(C.POINTER(C.c_uint64)), nsym, C.byref(cb)),
+           "entro_build_codebook")
+    return cb
 
 
 def entro_decode_dequant(stream_words: torch.Tensor, index: torch.Tensor, n: int, chunk_symbols: int, cb: Codebook,

@@ -116,8 +116,20 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const uint8_t* __restric
                                                         const Code* __restrict__ cb,
                                                         const unsigned long long* __restrict__ offsets,
                                                         const uint16_t* __restrict__ sub_len,
-                                                        uint32_t* __restrict__ stream)
+                                                        uint32_t* __restrict__ stream, uint64_t stream_words,
+                                                        unsigned long long* __restrict__ report)
 {
+    // report (batched calls): [0] total bits, [1] != 0 if they do not fit stream_words words (then
+    // nothing is written)
+    if (report) {
+        const unsigned long long total = offsets[n_chunks];
+        const bool fits = (total + 31) / 32 <= stream_words;
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            report[0] = total;
+            report[1] = fits ? 0ull : 1ull;
+        }
+        if (!fits) return;
+    }
     __shared__ uint32_t s_code[ENTRO_MAX_SYMBOLS];
     __shared__ uint8_t s_len[ENTRO_MAX_SYMBOLS];
     for (int i = threadIdx.x; i < ENTRO_MAX_SYMBOLS; i += kThreads) {
@@ -227,10 +239,89 @@ extern "C" entro_status entro_encode(const uint8_t* q_dev, uint64_t n, const ent
     if (words + ENTRO_STREAM_SLACK_WORDS > stream_cap_words) return ENTRO_ERR_BUFFER_TOO_SMALL;
 
     ENTRO_CUDA(cudaMemsetAsync(stream_dev, 0, stream_cap_words * sizeof(uint32_t), s));
-    pack_kernel<<<grid, kThreads, 0, s>>>(q_dev, n, chunk_symbols, nc, dev_code, offsets, sub_len, stream_dev);
+    pack_kernel<<<grid, kThreads, 0, s>>>(q_dev, n, chunk_symbols, nc, dev_code, offsets, sub_len, stream_dev, 0, nullptr);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     ENTRO_CUDA(cudaStreamSynchronize(s));
     *total_bits_host = h.total;
     return ENTRO_OK;
+}
+
+// The same for many tensors with one synchronisation at the end: per tensor the three passes
+// are queued back to back, the pack pass itself refuses to write a stream that would not fit,
+// and totals and error flags of all tensors come back in one copy.
+extern "C" entro_status entro_encode_batched(const entro_encode_job* jobs, int njobs, uint64_t* total_bits_host,
+                                             void* cuda_stream)
+{
+    if (njobs < 0 || (njobs > 0 && (!jobs || !total_bits_host))) return ENTRO_ERR_INVALID_ARG;
+    if (njobs == 0) return ENTRO_OK;
+    uint32_t max_nc = 0;
+    for (int j = 0; j < njobs; ++j) {
+        const entro_encode_job& job = jobs[j];
+        if (!job.q_dev || !job.cb_host || !job.stream_dev || !job.index_dev || job.n == 0) return ENTRO_ERR_INVALID_ARG;
+        if (job.chunk_symbols < kSubBlocks || job.chunk_symbols % kSubBlocks || job.chunk_symbols > ENTRO_MAX_CHUNK_SYMBOLS)
+            return ENTRO_ERR_INVALID_ARG;
+        if (!aligned(job.q_dev, 16) || !aligned(job.stream_dev, 16) || !aligned(job.index_dev, 8)) return ENTRO_ERR_INVALID_ARG;
+        if (!codebook_lengths_valid(job.cb_host)) return ENTRO_ERR_INVALID_ARG;
+        const uint64_t nc64 = num_chunks(job.n, job.chunk_symbols);
+        if (nc64 > 0x7fffffffull) return ENTRO_ERR_UNSUPPORTED;
+        if (entro_index_bytes(job.n, job.chunk_symbols) > job.index_cap_bytes) return ENTRO_ERR_BUFFER_TOO_SMALL;
+        if (job.stream_cap_words <= ENTRO_STREAM_SLACK_WORDS) return ENTRO_ERR_BUFFER_TOO_SMALL;
+        if ((uint32_t)nc64 > max_nc) max_nc = (uint32_t)nc64;
+    }
+    Guard g;
+    Workspace* ws = workspace();
+    if (!ws) return ENTRO_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // device area: [Code x njobs][report x njobs: total, overflow][bad-symbol flag x njobs][chunk bits of the tensor in flight]
+    const size_t code_bytes = (sizeof(Code) + 15) & ~(size_t)15;
+    const size_t codes_bytes = code_bytes * (size_t)njobs;
+    const size_t report_bytes = (size_t)njobs * 16;
+    const size_t flags_bytes = ((size_t)njobs * 4 + 15) & ~(size_t)15;
+    if (!reserve_device(ws, codes_bytes + report_bytes + flags_bytes + (size_t)max_nc * 8 + 16)) return ENTRO_ERR_CUDA;
+    if (!reserve_pinned(ws, codes_bytes + report_bytes + flags_bytes)) return ENTRO_ERR_CUDA;
+    char* base = static_cast<char*>(ws->dev);
+    char* host = static_cast<char*>(ws->pinned);
+    for (int j = 0; j < njobs; ++j) {
+        Code* hc = reinterpret_cast<Code*>(host + code_bytes * (size_t)j);
+        const entro_codebook* cb = jobs[j].cb_host;
+        for (int k = 0; k < ENTRO_MAX_SYMBOLS; ++k) {
+            hc->code[k] = k < cb->nsym ? cb->code[k] : 0;
+            hc->len[k] = k < cb->nsym ? cb->len[k] : 0;
+        }
+    }
+    unsigned long long* report = reinterpret_cast<unsigned long long*>(base + codes_bytes);
+    uint32_t* flags = reinterpret_cast<uint32_t*>(base + codes_bytes + report_bytes);
+    unsigned long long* chunk_bits = reinterpret_cast<unsigned long long*>(base + codes_bytes + report_bytes + flags_bytes);
+    ENTRO_CUDA(cudaMemcpyAsync(base, host, codes_bytes, cudaMemcpyHostToDevice, s));
+    ENTRO_CUDA(cudaMemsetAsync(report, 0, report_bytes + flags_bytes, s));
+    for (int j = 0; j < njobs; ++j) {
+        const entro_encode_job& job = jobs[j];
+        const uint32_t nc = (uint32_t)num_chunks(job.n, job.chunk_symbols);
+        const Code* dev_code = reinterpret_cast<const Code*>(base + code_bytes * (size_t)j);
+        unsigned long long* offsets = static_cast<unsigned long long*>(job.index_dev);
+        uint16_t* sub_len = reinterpret_cast<uint16_t*>(offsets + nc + 1);
+        int grid = (int)((nc + kWarps - 1) / kWarps);
+        const int cap = ws->sm_count * 8;
+        if (grid > cap) grid = cap;
+        sub_lengths_kernel<<<grid, kThreads, 0, s>>>(job.q_dev, job.n, job.chunk_symbols, nc, dev_code, sub_len, chunk_bits, flags + j);
+        chunk_offsets_kernel<<<1, 1024, 0, s>>>(chunk_bits, nc, offsets);
+        ENTRO_CUDA(cudaMemsetAsync(job.stream_dev, 0, job.stream_cap_words * sizeof(uint32_t), s));
+        pack_kernel<<<grid, kThreads, 0, s>>>(job.q_dev, job.n, job.chunk_symbols, nc, dev_code, offsets, sub_len, job.stream_dev,
+                                              job.stream_cap_words - ENTRO_STREAM_SLACK_WORDS, report + 2 * (size_t)j);
+        count_launch(3);
+    }
+    ENTRO_CUDA(cudaGetLastError());
+    char* host_report = host + codes_bytes;                 // behind the codes, which the device may still be reading
+    ENTRO_CUDA(cudaMemcpyAsync(host_report, report, report_bytes + flags_bytes, cudaMemcpyDeviceToHost, s));
+    ENTRO_CUDA(cudaStreamSynchronize(s));
+    const unsigned long long* hr = reinterpret_cast<const unsigned long long*>(host_report);
+    const uint32_t* hf = reinterpret_cast<const uint32_t*>(host_report + report_bytes);
+    entro_status st = ENTRO_OK;
+    for (int j = 0; j < njobs; ++j) {
+        total_bits_host[j] = hr[2 * j];
+        if (hf[j]) st = ENTRO_ERR_INVALID_ARG;                       // a symbol without a code
+        else if (hr[2 * j + 1] && st == ENTRO_OK) st = ENTRO_ERR_BUFFER_TOO_SMALL;
+    }
+    return st;
 }

@@ -129,6 +129,125 @@ __global__ void __launch_bounds__(kThreads) quantise_kernel(const uint16_t* __re
     }
 }
 
+// (s, z) of one tensor on the device, by the arithmetic of the host code in
+// entro_quantize_tensor (IEEE fp32, one rounding per operation), so that a batch of tensors
+// needs no round trip to the host between the range pass and the quantise pass.
+struct DevQParams {
+    float scale;
+    int32_t zero_point;
+    int32_t mode;
+    uint32_t nonfinite;
+    float lo, hi;
+    uint32_t pad[2];
+};
+
+__device__ __forceinline__ void derive_params(const Range* range, int qmax, int mode, DevQParams* out)
+{
+    float lo = range->lo, hi = range->hi;
+    if (lo == 0.0f) lo = 0.0f;   // -0 and +0 are the same bound
+    if (hi == 0.0f) hi = 0.0f;
+    int resolved = mode;
+    if (resolved == ENTRO_MODE_AUTO) resolved = (lo >= 0.0f) ? ENTRO_MODE_UNSIGNED : ENTRO_MODE_ASYMMETRIC;
+    float s;
+    int z = 0;
+    if (resolved == ENTRO_MODE_UNSIGNED) {
+        s = __fdiv_rn(hi, (float)qmax);
+        if (!(s > 0.0f)) s = 1.0f;
+    } else {
+        s = __fdiv_rn(__fsub_rn(hi, lo), (float)qmax);
+        if (!(s > 0.0f)) s = 1.0f;
+        float zr = rintf(__fdiv_rn(-lo, s));
+        zr = zr < 0.0f ? 0.0f : (zr > (float)qmax ? (float)qmax : zr);
+        z = (int)zr;
+    }
+    out->scale = s;
+    out->zero_point = z;
+    out->mode = resolved;
+    out->nonfinite = range->nonfinite;
+    out->lo = lo;
+    out->hi = hi;
+    out->pad[0] = out->pad[1] = 0;
+}
+
+// Pass 2 of a batch: fold the partials, then derive the parameters in the same launch.
+__global__ void __launch_bounds__(kThreads) range_final_params_kernel(const Range* __restrict__ partial, int count,
+                                                                      int qmax, int mode, DevQParams* __restrict__ out)
+{
+    float lo = INFINITY, hi = -INFINITY;
+    uint32_t bad = 0;
+    for (int i = threadIdx.x; i < count; i += kThreads) {
+        lo = fminf(lo, partial[i].lo);
+        hi = fmaxf(hi, partial[i].hi);
+        bad |= partial[i].nonfinite;
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+        bad |= __shfl_xor_sync(0xffffffffu, bad, d);
+    }
+    __shared__ Range s[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) s[threadIdx.x >> 5] = {lo, hi, bad, 0};
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Range r = s[0];
+        for (int k = 1; k < kThreads / 32; ++k) {
+            r.lo = fminf(r.lo, s[k].lo);
+            r.hi = fmaxf(r.hi, s[k].hi);
+            r.nonfinite |= s[k].nonfinite;
+        }
+        derive_params(&r, qmax, mode, out);
+    }
+}
+
+// Quantise and count in one pass over the weights: q as quantise_kernel writes it, counts as
+// histogram_kernel counts them.  Nothing is written for a tensor that holds a NaN or an infinity.
+__global__ void __launch_bounds__(kThreads) quantise_count_kernel(const uint16_t* __restrict__ w, uint64_t n,
+                                                                  const DevQParams* __restrict__ p, int qmax,
+                                                                  uint8_t* __restrict__ q,
+                                                                  unsigned long long* __restrict__ counts)
+{
+    if (p->nonfinite) return;
+    __shared__ uint32_t hist[kThreads / 32][ENTRO_MAX_SYMBOLS];
+    for (int i = threadIdx.x; i < (kThreads / 32) * ENTRO_MAX_SYMBOLS; i += kThreads) (&hist[0][0])[i] = 0;
+    __syncthreads();
+    uint32_t* mine = hist[threadIdx.x >> 5];
+    const float s = p->scale;
+    const int z = p->zero_point;
+    const uint64_t nvec = n / 8;
+    const uint4* wv = reinterpret_cast<const uint4*>(w);
+    uint2* qv = reinterpret_cast<uint2*>(q);
+    for (uint64_t i = blockIdx.x * (uint64_t)kThreads + threadIdx.x; i < nvec; i += (uint64_t)gridDim.x * kThreads) {
+        uint4 v = __ldg(wv + i);
+        uint32_t u[4] = {v.x, v.y, v.z, v.w};
+        uint32_t b[8];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            b[2 * k] = quantise_one((uint16_t)(u[k] & 0xffffu), s, z, qmax);
+            b[2 * k + 1] = quantise_one((uint16_t)(u[k] >> 16), s, z, qmax);
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) atomicAdd(&mine[b[k]], 1u);
+        uint2 o;
+        o.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+        o.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
+        qv[i] = o;
+    }
+    if (blockIdx.x == 0) {
+        for (uint64_t i = nvec * 8 + threadIdx.x; i < n; i += kThreads) {
+            const uint32_t sym = quantise_one(w[i], s, z, qmax);
+            q[i] = (uint8_t)sym;
+            atomicAdd(&mine[sym], 1u);
+        }
+    }
+    __syncthreads();
+    for (uint32_t k = threadIdx.x; k <= (uint32_t)qmax; k += kThreads) {
+        unsigned long long t = 0;
+        for (int wi = 0; wi < kThreads / 32; ++wi) t += hist[wi][k];
+        if (t) atomicAdd(&counts[k], t);
+    }
+}
+
 // Block-based grid: one warp per block of `block` consecutive weights.  The warp finds the
 // block's range, every lane derives the same (s, z) from it with the arithmetic of the
 // per-tensor call (IEEE fp32, one rounding per operation), then the block is quantised.
@@ -294,6 +413,69 @@ extern "C" entro_status entro_quantize_tensor(const void* w_fp16_dev, uint64_t n
     ENTRO_CUDA(cudaGetLastError());
     ENTRO_CUDA(cudaStreamSynchronize(s));
     return ENTRO_OK;
+}
+
+extern "C" entro_status entro_quantize_histogram_batched(const entro_quantize_job* jobs, int njobs,
+                                                         entro_qparams* qp_host, uint64_t* counts_host,
+                                                         void* cuda_stream)
+{
+    if (njobs < 0 || (njobs > 0 && (!jobs || !qp_host || !counts_host))) return ENTRO_ERR_INVALID_ARG;
+    if (njobs == 0) return ENTRO_OK;
+    for (int j = 0; j < njobs; ++j) {
+        const entro_quantize_job& job = jobs[j];
+        if (!job.w_fp16_dev || !job.q_dev || job.n == 0 || (job.bits != 4 && job.bits != 8)) return ENTRO_ERR_INVALID_ARG;
+        if (job.mode != ENTRO_MODE_AUTO && job.mode != ENTRO_MODE_UNSIGNED && job.mode != ENTRO_MODE_ASYMMETRIC)
+            return ENTRO_ERR_INVALID_ARG;
+        if (!aligned(job.w_fp16_dev, 16) || !aligned(job.q_dev, 16)) return ENTRO_ERR_INVALID_ARG;
+    }
+    Guard g;
+    Workspace* ws = workspace();
+    if (!ws) return ENTRO_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // device area: [partial ranges of the tensor in flight][parameters x njobs][counts x njobs x 256]
+    const int max_grid = ws->sm_count * 8;
+    const size_t partial_bytes = (size_t)max_grid * sizeof(Range);
+    const size_t params_bytes = (size_t)njobs * sizeof(DevQParams);
+    const size_t counts_bytes = (size_t)njobs * ENTRO_MAX_SYMBOLS * sizeof(unsigned long long);
+    if (!reserve_device(ws, partial_bytes + params_bytes + counts_bytes)) return ENTRO_ERR_CUDA;
+    if (!reserve_pinned(ws, params_bytes + counts_bytes)) return ENTRO_ERR_CUDA;
+    char* base = static_cast<char*>(ws->dev);
+    Range* partial = reinterpret_cast<Range*>(base);
+    DevQParams* params = reinterpret_cast<DevQParams*>(base + partial_bytes);
+    unsigned long long* counts = reinterpret_cast<unsigned long long*>(base + partial_bytes + params_bytes);
+    ENTRO_CUDA(cudaMemsetAsync(counts, 0, counts_bytes, s));
+    for (int j = 0; j < njobs; ++j) {
+        const entro_quantize_job& job = jobs[j];
+        const uint16_t* w = static_cast<const uint16_t*>(job.w_fp16_dev);
+        const int qmax = (1 << job.bits) - 1;
+        int grid = grid_for(job.n / 8 + 1, ws->sm_count, 8);
+        // at most 2^31 symbols per block keeps the 32-bit shared counters exact
+        if ((uint64_t)grid < (job.n >> 31) + 1) grid = (int)((job.n >> 31) + 1);
+        if (grid > max_grid) return ENTRO_ERR_UNSUPPORTED;
+        range_partial_kernel<<<grid, kThreads, 0, s>>>(w, job.n, partial);
+        range_final_params_kernel<<<1, kThreads, 0, s>>>(partial, grid, qmax, job.mode, params + j);
+        quantise_count_kernel<<<grid, kThreads, 0, s>>>(w, job.n, params + j, qmax, job.q_dev,
+                                                        counts + (size_t)j * ENTRO_MAX_SYMBOLS);
+        count_launch(3);
+    }
+    ENTRO_CUDA(cudaGetLastError());
+    char* host = static_cast<char*>(ws->pinned);
+    ENTRO_CUDA(cudaMemcpyAsync(host, params, params_bytes + counts_bytes, cudaMemcpyDeviceToHost, s));
+    ENTRO_CUDA(cudaStreamSynchronize(s));
+    const DevQParams* hp = reinterpret_cast<const DevQParams*>(host);
+    const unsigned long long* hc = reinterpret_cast<const unsigned long long*>(host + params_bytes);
+    entro_status st = ENTRO_OK;
+    for (int j = 0; j < njobs; ++j) {
+        qp_host[j].bits = jobs[j].bits;
+        qp_host[j].mode = hp[j].mode;
+        qp_host[j].scale = hp[j].scale;
+        qp_host[j].zero_point = hp[j].zero_point;
+        qp_host[j].lo = hp[j].lo;
+        qp_host[j].hi = hp[j].hi;
+        for (int k = 0; k < ENTRO_MAX_SYMBOLS; ++k) counts_host[(size_t)j * ENTRO_MAX_SYMBOLS + k] = hc[(size_t)j * ENTRO_MAX_SYMBOLS + k];
+        if (hp[j].nonfinite) st = ENTRO_ERR_NONFINITE;
+    }
+    return st;
 }
 
 extern "C" entro_status entro_quantize_blocks(const void* w_fp16_dev, uint64_t n, int bits, entro_mode mode,

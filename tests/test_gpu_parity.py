@@ -136,6 +136,47 @@ def test_format_stated_in_the_header_is_the_format_the_library_uses(bits, chunk,
     assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.dequant(q_np, qp.scale, qp.zero_point))
 
 
+def test_batched_offline_stages_equal_the_per_tensor_calls_and_the_oracle():
+    """entro_quantize_histogram_batched / entro_encode_batched: parameters (computed on the device),
+    symbols, counts, streams and indices of every tensor equal the per-tensor calls' and the oracle's."""
+    specs = [(8, 300_000 + 7, "matrix"), (8, 4096, "gain"), (8, 1, "matrix"), (8, 5 * 4096, "matrix"), (8, 33, "gain")]
+    for bits, chunk in ((8, 4096), (4, 8192)):
+        vals = [_values(n, 0.02 + 0.003 * k, 8800 + 10 * bits + k, kind) for k, (_, n, kind) in enumerate(specs)]
+        qs, qps, counts = E.entro_quantize_histogram_batched([v[1] for v in vals], bits)
+        cbs, words = [], []
+        for j, (w_np, w_dev) in enumerate(vals):
+            c = oracle.compress(w_np, bits, chunk)
+            q1, qp1 = E.entro_quantize_tensor(w_dev, bits)
+            assert (np.float32(qps[j].scale).tobytes(), qps[j].zero_point, qps[j].mode) == \
+                   (np.float32(c.qp.scale).tobytes(), c.qp.zero_point, c.qp.mode) == \
+                   (np.float32(qp1.scale).tobytes(), qp1.zero_point, qp1.mode), j
+            assert np.array_equal(qs[j].cpu().numpy(), c.q) and torch.equal(qs[j], q1), j
+            assert np.array_equal(counts[j, :1 << bits], c.counts) and not counts[j, 1 << bits:].any(), j
+            cb = E.entro_build_codebook_np(counts[j], 1 << bits)
+            assert np.array_equal(cb.lengths(), c.lengths)
+            cbs.append(cb)
+            words.append(E.entro_stream_words_np(counts[j], cb))
+            vals[j] = (c, w_dev)
+        encs = E.entro_encode_batched(qs, cbs, chunk, words)
+        for j, enc in enumerate(encs):
+            c = vals[j][0]
+            assert enc.total_bits == c.enc.total_bits, j
+            assert np.array_equal(enc.stream_np(), c.enc.stream), j
+            assert np.array_equal(enc.offsets(), c.enc.offsets) and np.array_equal(enc.sub_len(), c.enc.sub_len), j
+        # a stream buffer that is too small is reported and left zeroed; the others are complete
+        short = list(words)
+        short[0] = E.STREAM_SLACK_WORDS + 2
+        with pytest.raises(E.EntroError) as e:
+            E.entro_encode_batched(qs, cbs, chunk, short)
+        assert e.value.status == E.ERR_BUFFER_TOO_SMALL
+    # a tensor with an infinity is reported; the other tensors of the batch are complete
+    w_bad = vals[0][1].clone()
+    w_bad[5] = float("inf")
+    with pytest.raises(E.EntroError) as e:
+        E.entro_quantize_histogram_batched([vals[3][1], w_bad], 8)
+    assert e.value.status == E.ERR_NONFINITE
+
+
 def test_encode_errors():
     q = torch.tensor([0, 1, 2, 3] * 100, dtype=torch.uint8).cuda()
     cb = E.entro_build_codebook([5, 5, 5, 0])              # symbol 3 has no code

@@ -36,23 +36,41 @@ class DeviceModel:
         self.max_len = 0
         pos = 0
         self.host_meta = []
-        self.compress_s = 0.0    # wall time of quantise + histogram + codebook + encode over all tensors
-        for spec in wl.tensors:
-            w = workloads.make_tensor(spec, "cuda").view(-1)
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            q, qp = E.entro_quantize_tensor(w, wl.bits)
-            counts = E.entro_histogram(q, wl.bits)
-            cb = (E.entro_build_codebook_limited(counts.tolist(), max_code_len) if max_code_len
-                  else E.entro_build_codebook(counts.tolist()))
-            enc = E.entro_encode(q, cb, wl.chunk_symbols, stream_words=E.entro_stream_words(counts.tolist(), cb))
-            torch.cuda.synchronize()
-            self.compress_s += time.perf_counter() - t0
+        self.compress_s = 0.0    # wall time of quantise + histogram + codebooks + encode over all tensors
+        # every tensor is drawn first (the fp16 model is resident, as it would be after training), then the
+        # offline stages run over all of them with one synchronisation per stage
+        ws = [workloads.make_tensor(spec, "cuda").view(-1) for spec in wl.tensors]
+
+        def carve(sizes, dtype, unit):
+            """One allocation cut into 16-byte aligned slices of the given sizes (in elements of `unit` bytes)."""
+            per = 16 // unit
+            padded = [(n + per - 1) // per * per for n in sizes]
+            arena = torch.empty(sum(padded), dtype=dtype, device="cuda")
+            out, at = [], 0
+            for n, m in zip(sizes, padded):
+                out.append(arena[at:at + n])
+                at += m
+            return out
+
+        q_bufs = carve([t.numel for t in wl.tensors], torch.uint8, 1)
+        index_bufs = carve([E.entro_index_bytes(t.numel, wl.chunk_symbols) for t in wl.tensors], torch.uint8, 1)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        qs, qps, counts = E.entro_quantize_histogram_batched(ws, wl.bits, qs=q_bufs)
+        nsym = 1 << wl.bits
+        cbs = [E.entro_build_codebook_limited(counts[j, :nsym].tolist(), max_code_len) if max_code_len
+               else E.entro_build_codebook_np(counts[j], nsym) for j in range(len(ws))]
+        words = [E.entro_stream_words_np(counts[j], cb) for j, cb in enumerate(cbs)]
+        stream_bufs = carve(words, torch.int32, 4)
+        encs = E.entro_encode_batched(qs, cbs, wl.chunk_symbols, words, bufs=list(zip(stream_bufs, index_bufs)))
+        torch.cuda.synchronize()
+        self.compress_s = time.perf_counter() - t0
+        del ws
+        for spec, q, qp, cb, enc in zip(wl.tensors, qs, qps, cbs, encs):
             self.qparams.append((qp.scale, qp.zero_point))
             self.cbs.append(cb)
             if keep_q:
                 self.q.append(q)
-            del w, q
             out = self.out[pos:pos + spec.numel]
             pos += (spec.numel + 15) // 16 * 16
             descs.append(E.make_desc(enc.stream, enc.index, spec.numel, wl.chunk_symbols, cb, qp.scale,
@@ -65,6 +83,7 @@ class DeviceModel:
             self.index_bytes += enc.index.numel()
             self.table_bytes += lut_bytes
             self.max_len = max(self.max_len, cb.max_len)
+        del qs
         self.descs = E.desc_array(descs)
         self.algorithmic_bytes = self.stream_bytes + self.index_bytes + self.table_bytes + 2 * self.n
         self.bits_per_weight = 8.0 * self.stream_bytes / self.n
