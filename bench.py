@@ -544,7 +544,7 @@ def measure(E, wl, args, world, local_rank, rank, peak, with_e2e, with_cpu):
                      "traffic": (NCU_DRAM_BYTES_PER_WEIGHT.get(wl.bits) * model.n
                                  if NCU_DRAM_BYTES_PER_WEIGHT.get(wl.bits) else None),
                      "traffic_note": "bytes per launch: ncu DRAM read+write on the 1-layer case, scaled by weights"},
-        "compress": {"seconds": model.compress_s, "weights_per_s": model.n / model.compress_s,
+        "compress": {"seconds": model.compress_s, "weights_per_s": model.n / model.compress_s, **model.compress_stages,
                      "what": "entro_quantize_histogram_batched + codebooks (host) + entro_encode_batched over the whole "
                              "resident fp16 model, wall clock, one synchronise per stage; outside the timed steps"},
         "model": model,

@@ -54,17 +54,26 @@ class DeviceModel:
 
         q_bufs = carve([t.numel for t in wl.tensors], torch.uint8, 1)
         index_bufs = carve([E.entro_index_bytes(t.numel, wl.chunk_symbols) for t in wl.tensors], torch.uint8, 1)
+        nsym = 1 << wl.bits
+        # one small tensor through both calls first: kernels are loaded on their first launch
+        tiny = ws[0][:4096].contiguous()
+        tq, _, tc = E.entro_quantize_histogram_batched([tiny], wl.bits)
+        tcb = E.entro_build_codebook_np(tc[0], nsym)
+        E.entro_encode_batched(tq, [tcb], wl.chunk_symbols, [E.entro_stream_words_np(tc[0], tcb)])
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         qs, qps, counts = E.entro_quantize_histogram_batched(ws, wl.bits, qs=q_bufs)
-        nsym = 1 << wl.bits
+        t1 = time.perf_counter()
         cbs = [E.entro_build_codebook_limited(counts[j, :nsym].tolist(), max_code_len) if max_code_len
                else E.entro_build_codebook_np(counts[j], nsym) for j in range(len(ws))]
         words = [E.entro_stream_words_np(counts[j], cb) for j, cb in enumerate(cbs)]
         stream_bufs = carve(words, torch.int32, 4)
+        t2 = time.perf_counter()
         encs = E.entro_encode_batched(qs, cbs, wl.chunk_symbols, words, bufs=list(zip(stream_bufs, index_bufs)))
         torch.cuda.synchronize()
         self.compress_s = time.perf_counter() - t0
+        self.compress_stages = {"quantise_and_count_s": t1 - t0, "codebooks_and_stream_buffer_s": t2 - t1,
+                                "encode_s": self.compress_s - (t2 - t0)}
         del ws
         for spec, q, qp, cb, enc in zip(wl.tensors, qs, qps, cbs, encs):
             self.qparams.append((qp.scale, qp.zero_point))
