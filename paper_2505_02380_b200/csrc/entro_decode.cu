@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
 {
     constexpr int kBatch = kGemvBatchOf<kSink>;
     constexpr bool kGemv = kBatch > 0;
-    // layout: [tables][aux][tensor]([gemv descriptor][x])[per-warp rings][over-read pad][mbarriers][index slots][item + claim slots]
+    // layout: [tables][aux][tensor]([gemv descriptor][x])[per-warp rings][over-read pad][mbarriers][index slots][item slots]
     if (smem_addr(smem) != kSmemBase) {   // the lookups' address arithmetic would be wrong: refuse to run
         if (threadIdx.x == 0) {
             atomicOr(control + 1, kStatInternal);
@@ -105,7 +105,6 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     const uint32_t after = kRings + warps * stage_bytes + kOverRead;          // offset in smem, a multiple of 16
     const uint32_t slots = after + warps * 16u;
     volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(smem + slots + warps * 2u * kSlotBytes);   // [2]
-    uint32_t* s_claim = const_cast<uint32_t*>(s_item) + 2;                                                     // [2]
     uint32_t* status = control + 1;
 
     WarpCtx cx;
@@ -124,7 +123,6 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     const uint32_t total_items = item_start[ntensors];
     if (threadIdx.x == 0) {
         s_item[0] = atomicAdd(control, 1u);
-        s_claim[0] = 0;
     }
     __syncthreads();
     int cur = -1;
@@ -182,28 +180,33 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
         const uint32_t first = (item - __ldg(item_start + cur)) * T.item_chunks;
         const uint32_t count = min(T.item_chunks, T.n_chunks - first);   // chunks of this item
 
-        // The warps share out the item's chunks.  Each warp, per turn: start the bulk copy of
-        // chunk i + 1 (its offsets arrived a turn ago), work out the lanes' positions in chunk
-        // i, ask for the index entries of chunk i + 2 in the slot that frees, decode chunk i.
-        auto claim = [&]() -> uint32_t {
-            uint32_t k = 0;
-            if (lane == 0) k = atomicAdd(&s_claim[slot], 1u);
-            k = __shfl_sync(0xffffffffu, k, 0);
-            return k < count ? first + k : kNone;
+        // The warps deal out the item's chunks among themselves, warp w taking chunks w, w + warps,
+        // ... of the item (the chunks of one tensor cost about the same, so nobody waits long at the
+        // item's end).  Each warp, per turn: start the bulk copy of chunk i + 1 (its offsets arrived
+        // a turn ago), work out the lanes' positions in chunk i, ask for the index entries of chunk
+        // i + 2 in the slot that frees, decode chunk i.
+        uint32_t upcoming = first + warp;           // the warp's next chunk whose index entries have not been asked for
+        const uint32_t item_end = first + count;
+        auto next_chunk = [&]() -> uint32_t {
+            const uint32_t c = upcoming < item_end ? upcoming : kNone;
+            upcoming += warps;
+            return c;
         };
         Ready r0;
         r0.c = kNone;
         r0.meta = ready_meta(0, 0, 0, kSkip);
+        const uint32_t turns = s_aux->turns;
+        const uint32_t both_slots = 2u * cx.idx_addr + kSlotBytes;   // the sum of the two slots' addresses
         uint32_t sp = cx.idx_addr;                  // slot of the chunk fetched last
-        uint32_t c2 = claim();
-        fetch_index(T, c2, sp, lane);
+        uint32_t c2 = next_chunk();
+        fetch_index(s_aux, T, c2, sp, lane);
         while (true) {
-            Ready r1 = prepare(cx, T, stage_bytes, status, c2, sp, r0, lane);
-            const uint32_t other = cx.idx_addr + (sp == cx.idx_addr ? kSlotBytes : 0u);
+            Ready r1 = prepare(cx, T, turns, stage_bytes, status, c2, sp, r0, lane);
+            const uint32_t other = both_slots - sp;
             const Lane L = decode_start<K>(cx, status, r0, other, lane);
             __syncwarp();                           // every lane has read the slot before it is refilled
-            c2 = r1.c == kNone ? kNone : claim();
-            fetch_index(T, c2, other, lane);
+            c2 = r1.c == kNone ? kNone : next_chunk();
+            fetch_index(s_aux, T, c2, other, lane);
             decode_finish<K, kSink>(cx, status, r0, L, lane, stage_bytes);
             if (r1.c == kNone) break;
             r0 = r1;
@@ -212,9 +215,8 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
         asm volatile("cp.async.wait_all;" ::: "memory");
         if (threadIdx.x == 0) {
             s_item[slot ^ 1u] = next_item;
-            s_claim[slot ^ 1u] = 0;
         }
-        __syncthreads();   // tables may be replaced; s_item / s_claim [slot ^ 1] are now visible
+        __syncthreads();   // tables may be replaced; s_item[slot ^ 1] is now visible
         slot ^= 1u;
     }
     // A warp that gave up on a bulk copy lets it land (bounded) before its buffer goes away.

@@ -82,21 +82,23 @@ constexpr uint32_t kSlotBytes = 80;
 
 enum : uint32_t { kStaged = 0, kGeneral = 1, kSkip = 2 };
 
-// Chunk whose bytes have been asked for.  meta packs what the staging needs: ring offset /
-// 16 (12 bits), bytes / 16 (12 bits), ticket modulo 4 (2 bits), kind (2 bits), copy issued
-// (1 bit).  Everything else is re-read from the chunk's index slot when it is decoded.
+// Chunk whose bytes have been asked for.  meta packs what the staging needs so that every field
+// comes out by one or two operations: bits 0..1 kind, bit 2 copy issued, bits 4..15 the ring
+// offset (a multiple of 16, in place), bits 16..17 the ticket modulo 4, bits 20..31 the byte
+// count (a multiple of 16, at most 65520) shifted up by 16.  Everything else is re-read from the
+// chunk's index slot when it is decoded.
 struct Ready {
     uint32_t c;                // or kNone
     uint32_t meta;
-    __device__ __forceinline__ uint32_t at() const { return (meta & 0xfffu) << 4; }
-    __device__ __forceinline__ uint32_t bytes() const { return ((meta >> 12) & 0xfffu) << 4; }
-    __device__ __forceinline__ uint32_t ticket() const { return (meta >> 24) & 3u; }
-    __device__ __forceinline__ uint32_t kind() const { return (meta >> 26) & 3u; }
-    __device__ __forceinline__ bool issued() const { return (meta >> 28) & 1u; }
+    __device__ __forceinline__ uint32_t at() const { return meta & 0xfff0u; }
+    __device__ __forceinline__ uint32_t bytes() const { return (meta >> 16) & 0xfff0u; }
+    __device__ __forceinline__ uint32_t ticket() const { return (meta >> 16) & 3u; }
+    __device__ __forceinline__ uint32_t kind() const { return meta & 3u; }
+    __device__ __forceinline__ bool issued() const { return (meta & 4u) != 0u; }
 };
 __device__ __forceinline__ uint32_t ready_meta(uint32_t at, uint32_t bytes, uint32_t ticket, uint32_t kind)
 {
-    return (at >> 4) | ((bytes >> 4) << 12) | ((ticket & 3u) << 24) | (kind << 26);
+    return at | kind | ((bytes | (ticket & 3u)) << 16);
 }
 
 __device__ __forceinline__ unsigned long long lds64(uint32_t addr)
@@ -110,13 +112,13 @@ __device__ __forceinline__ unsigned long long lds64(uint32_t addr)
 // Ask for chunk c's index entries to be copied into the slot at shared address `slot`
 // (lanes 0..15 two sub-block lengths each, lanes 16 and 17 one offset each).  Nothing is
 // held in registers while the copies are in flight.
-__device__ __forceinline__ void fetch_index(const DevTensor& T, uint32_t c, uint32_t slot, uint32_t lane)
+__device__ __forceinline__ void fetch_index(const DecodeAux* aux, const DevTensor& T, uint32_t c, uint32_t slot, uint32_t lane)
 {
     if (c != kNone && ENTRO_CHECK(c < T.n_chunks && smem_ok(slot, 16u) && smem_ok(slot + kSlotBytes - 16u, 16u))) c = kNone;
     if (c != kNone && lane < 20u) {
-        // 4 bytes per lane: lanes 0..15 the sub-block lengths, lanes 16..19 the two offsets
-        const char* src = lane < 16u ? reinterpret_cast<const char*>(T.sub_len + (uint64_t)c * kSubBlocks) + lane * 4u
-                                     : reinterpret_cast<const char*>(T.offsets + c) + (lane - 16u) * 4u;
+        // 4 bytes per lane: lanes 0..15 the sub-block lengths (64 bytes per chunk), lanes 16..19 the two offsets (8 per chunk)
+        unsigned long long src;
+        asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(src) : "r"(c), "r"(lane < 16u ? 64u : 8u), "l"(aux->index_src[lane]));
         asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(slot + lane * 4u), "l"(src) : "memory");
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -132,7 +134,7 @@ __device__ __forceinline__ void issue_copy(const WarpCtx& cx, const DevTensor& T
     if (lane == 0 && !bad)
         bulk_load(cx.stage_addr + r.at(), reinterpret_cast<const char*>(T.stream) + byte0, r.bytes(),
                   cx.bar + 8u * (r.ticket() & 1u));
-    r.meta |= 1u << 28;
+    r.meta |= 4u;
 }
 
 // Bytes of the stream that decoding a chunk touches: from the 16-byte boundary below its
@@ -146,8 +148,8 @@ __device__ __forceinline__ void chunk_bytes(uint64_t off0, uint64_t off1, uint64
 // Chunk c's offsets have arrived in `slot`: check them, find a place in the ring next to
 // `prev` (the chunk decoded before this one, still undecoded), and start the bulk copy if
 // that place is free already.  All lanes compute the same values.
-__device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32_t stage_bytes, uint32_t* status,
-                                         uint32_t c, uint32_t slot, const Ready& prev, uint32_t lane)
+__device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32_t turns, uint32_t stage_bytes,
+                                         uint32_t* status, uint32_t c, uint32_t slot, const Ready& prev, uint32_t lane)
 {
     Ready r;
     r.c = c;
@@ -156,17 +158,16 @@ __device__ __forceinline__ Ready prepare(WarpCtx& cx, const DevTensor& T, uint32
     __syncwarp();
     if (c == kNone) return r;
     const uint64_t off0 = lds64(slot + 64u), off1 = lds64(slot + 72u);
-    uint64_t byte0, byte1;
-    chunk_bytes(off0, off1, byte0, byte1);
-    // (off1 < off0 wraps to a huge difference; off1 <= last_bit keeps byte1 inside the buffer)
+    // (off1 < off0 wraps to a huge difference; off1 <= last_bit keeps the copied bytes inside the buffer)
     if (off1 - off0 > 32ull * 65535ull || off1 > T.last_bit) {
         if (lane == 0) atomicOr(status, kStatCorrupt);
         return r;
     }
-    const uint32_t sub = T.chunk_symbols / kSubBlocks;
-    const bool full = c < T.full_chunks;
-    const uint32_t bytes = (uint32_t)(byte1 - byte0);
-    if (!full || (sub & 7u) || bytes > stage_bytes || cx.dead()) {
+    // the bytes decoding touches (chunk_bytes), their count in 32-bit arithmetic: the chunk is short
+    const uint64_t byte0 = (off0 >> 3) & ~15ull;
+    const uint32_t bytes = (((uint32_t)(off1 >> 3) + 13u + 15u) & ~15u) - (uint32_t)byte0;
+    // a full chunk of whole groups of 8 per lane whose bytes fit the ring is staged
+    if (c >= T.full_chunks || turns == 0u || bytes > stage_bytes || cx.dead()) {
         r.meta = ready_meta(0, 0, 0, kGeneral);
         return r;
     }
@@ -243,7 +244,7 @@ __device__ __forceinline__ void decode_chunk_general(const DecodeAux* aux, uint3
         for (uint32_t i = g * 8u; i < end; ++i) {
             gwin_refill(r);
             uint32_t e = kEscLen;
-            if (!oct) e = exp_lookup(lut_key(aux->expm, lane), ~r.hi);
+            if (!oct) e = exp_lookup(lut_key(aux, lane), ~r.hi);
             if ((e & 0xffffu) > 32u) e = decode_by_range(aux, r.hi, status);
             const uint32_t n = e & 0xffffu;
             r.hi = __funnelshift_lc(r.lo, r.hi, n);
@@ -543,15 +544,14 @@ template <int K, class Emit>
 __device__ __forceinline__ uint32_t rows_any(const DecodeAux* aux, uint32_t start, uint32_t* status, Emit& emit,
                                              uint32_t lane)
 {
-    if (aux->oct) return rows_oct<K>(start, status, emit);
-    const LutKey key = lut_key(aux->expm, lane);
-    switch (aux->group) {
-        case 16u: return rows_single<K, 16>(start, status, key, emit);
-        case 8u: return rows_single<K, 8>(start, status, key, emit);
-        case 4u: return rows_single<K, 4>(start, status, key, emit);
-        case 3u: return rows_single<K, 3>(start, status, key, emit);
-        default: return rows_single<K, 2>(start, status, key, emit);
-    }
+    const uint32_t mode = aux->mode;
+    if (mode == 0u) return rows_oct<K>(start, status, emit);
+    const LutKey key = lut_key(aux, lane);
+    if (mode == 8u) return rows_single<K, 8>(start, status, key, emit);
+    if (mode == 4u) return rows_single<K, 4>(start, status, key, emit);
+    if (mode == 3u) return rows_single<K, 3>(start, status, key, emit);
+    if (mode == 16u) return rows_single<K, 16>(start, status, key, emit);
+    return rows_single<K, 2>(start, status, key, emit);
 }
 
 // What decode_start leaves for decode_finish: where this lane begins and must end.
@@ -572,12 +572,15 @@ __device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status
     if (L.kind == kSkip) return L;
     const uint32_t pair = lds32(slot + (lane >> 1) * 4u);
     const uint32_t bits = (lane & 1u) ? pair >> 16 : pair & 0xffffu;
+    // inclusive prefix sum over the lanes: a shuffle says by itself whether its source lane exists
     uint32_t incl = bits;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= (uint32_t)d) incl += t;
-    }
+#define ENTRO_SCAN_STEP(d)                                     \
+    "shfl.sync.up.b32 t|p, %0, " #d ", 0, 0xffffffff;\n\t"      \
+    "@p add.u32 %0, %0, t;\n\t"
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t" ENTRO_SCAN_STEP(1) ENTRO_SCAN_STEP(2) ENTRO_SCAN_STEP(4)
+                     ENTRO_SCAN_STEP(8) ENTRO_SCAN_STEP(16) "}"
+                 : "+r"(incl));
+#undef ENTRO_SCAN_STEP
     const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
     // (prepare has checked that the chunk is shorter than 2^21 bits: the low words decide)
     const uint32_t off0 = lds32(slot + 64u), off1 = lds32(slot + 72u);
@@ -591,8 +594,8 @@ __device__ __forceinline__ Lane decode_start(const WarpCtx& cx, uint32_t* status
         L.start = excl;
         L.end = bits;
     } else {
-        const uint32_t byte0_bits = off0 & ~127u;              // bit offset of the copied bytes' start, modulo 2^32
-        L.start = (cx.stage_addr + r.at()) * 8u + (off0 - byte0_bits) + excl;
+        // (off0 & 127: the chunk's first bit behind the 16-byte boundary the copy started at)
+        L.start = (cx.stage_addr + r.at()) * 8u + (off0 & 127u) + excl;
         L.end = L.start + bits;
     }
     return L;
@@ -625,7 +628,7 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         decode_chunk_general<kBatch>(aux_ptr<K>(), status, T, G, kSink, r.c, L.start, L.end, lane);
         return;
     }
-    const uint32_t sub = T.chunk_symbols / kSubBlocks;
+    const uint32_t turns = aux_ptr<K>()->turns;     // groups of 8 symbols per lane (staged chunks have whole groups only)
     uint32_t stood;            // where the lane stands after its sub-block
     if (kGemv) {
         // the chunk starts gs0 steps of 256 weights into the matrix; a row is rs steps long
@@ -644,23 +647,23 @@ __device__ __forceinline__ void decode_finish(WarpCtx& cx, uint32_t* status, Rea
         em.G = G;
         em.row = row0;
         em.began_before = k0 != 0u;
-        em.todo = sub >> 3;
+        em.todo = turns;
         stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
         em.finish();
     } else if (kSink == kSinkBytes) {
         EmitBytes em;
-        em.out.start(reinterpret_cast<uint8_t*>(T.out) + (uint64_t)r.c * T.chunk_symbols + lane * 8u, sub >> 3, 8u * kSubBlocks);
+        em.out.start(reinterpret_cast<uint8_t*>(T.out) + (uint64_t)r.c * T.chunk_symbols + lane * 8u, turns, 8u * kSubBlocks);
         em.out.bounds(T.out, T.n);
         stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
     } else if (kSink == kSinkNibbles) {
         EmitNibbles em;
-        em.out.start(reinterpret_cast<uint8_t*>(T.out) + (((uint64_t)r.c * T.chunk_symbols) >> 1) + lane * 4u, sub >> 3,
+        em.out.start(reinterpret_cast<uint8_t*>(T.out) + (((uint64_t)r.c * T.chunk_symbols) >> 1) + lane * 4u, turns,
                      4u * kSubBlocks);
         em.out.bounds(T.out, (T.n + 1u) >> 1);
         stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
     } else {
         EmitStore em;
-        em.out.start(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u, sub >> 3, 16u * kSubBlocks);
+        em.out.start(T.out + (uint64_t)r.c * T.chunk_symbols + lane * 8u, turns, 16u * kSubBlocks);
         em.out.bounds(T.out, T.n * 2u);
         stood = rows_any<K>(aux_ptr<K>(), L.start, status, em, lane);
         em.finish();

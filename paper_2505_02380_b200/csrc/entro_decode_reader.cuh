@@ -100,11 +100,11 @@ __device__ __forceinline__ void gwin_refill(GlobalWin& r)
 struct LutKey {
     uint32_t mask, lane;
 };
-__device__ __forceinline__ LutKey lut_key(uint32_t expm, uint32_t lane)
+__device__ __forceinline__ LutKey lut_key(const DecodeAux* aux, uint32_t lane)
 {
     LutKey k;
-    k.mask = ((32u << expm) - 1u) << (11u - expm);
-    k.lane = (lane & ((32u >> (expm - 4u)) - 1u)) * 4u;
+    k.mask = aux->key_mask;
+    k.lane = (lane & aux->key_lane_mask) * 4u;
     return k;
 }
 

@@ -156,6 +156,17 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
         aux.expm = m;
     }
     __syncthreads();
+    if (tid == 0) {
+        const uint32_t m = aux.expm;
+        aux.key_mask = ((32u << m) - 1u) << (11u - m);
+        aux.key_lane_mask = (32u >> (m - 4u)) - 1u;
+        aux.turns = (T.chunk_symbols % (8u * kSubBlocks)) == 0u ? T.chunk_symbols / (8u * kSubBlocks) : 0u;
+        aux.mode = aux.oct ? 0u : aux.group;
+    }
+    if (tid < 20)
+        aux.index_src[tid] = tid < 16 ? reinterpret_cast<unsigned long long>(T.sub_len) + 4ull * tid
+                                      : reinterpret_cast<unsigned long long>(T.offsets) + 4ull * (tid - 16);
+    __syncthreads();
     const float d = (float)(tid - T.zero_point);
     aux.val[tid] = T.raw_symbols ? (uint16_t)tid : __half_as_ushort(__float2half_rn(__fmul_rn(T.scale, d)));
     __syncthreads();

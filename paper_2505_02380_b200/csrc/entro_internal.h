@@ -65,6 +65,13 @@ struct DecodeAux {
     uint32_t oct;      // 1: eight symbols per lookup (alphabets of <= 16 symbols)
     uint32_t group;    // one-symbol lookups per group: 2, 3, 4; 8 = two groups of four under one check; 16 = eight on one view
     uint32_t expm;     // mantissa bits of this tensor's exponent-indexed table
+    // worked out once per tensor so that a warp does not repeat it for every chunk:
+    uint32_t key_mask;       // the bits of (float bits >> 12) that select a cell of the exponent-indexed table
+    uint32_t key_lane_mask;  // lanes that share a copy of that table: copy = lane & this
+    uint32_t turns;          // groups of 8 symbols per lane and full chunk (chunk_symbols / 256), 0 if chunks cannot be staged
+    uint32_t mode;           // what the decode loop switches on: 0 = eight symbols per lookup, else `group`
+    unsigned long long index_src[20];   // lane l's 4 bytes of chunk 0's index entries: lanes 0..15 two sub-block lengths
+                                        // each, lanes 16..19 the halves of offsets[c], offsets[c + 1]
 };
 static_assert(sizeof(DecodeAux) % 16 == 0, "DecodeAux is copied as 16-byte vectors");
 
