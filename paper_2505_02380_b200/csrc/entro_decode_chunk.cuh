@@ -23,21 +23,29 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  : "memory");
 }
 
-// Bounded wait for phase `parity` of the barrier; false if the bound ran out.  Each try may
-// suspend the thread for up to the hinted time, so waiting costs few issue slots.
+// One try at phase `parity` of the barrier; may suspend the thread for up to the hinted time.
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity), "r"(20000u)
+        : "memory");
+    return done != 0u;
+}
+
+// Bounded wait for phase `parity` of the barrier; false if the bound ran out.  The bytes have
+// nearly always arrived long before they are asked for, so the first try stands by itself and
+// the loop is off the usual path.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
-    for (uint32_t tries = 0; tries < kWaitTries; ++tries) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity), "r"(20000u)
-            : "memory");
-        if (done) return true;
-    }
+    if (__builtin_expect(mbar_try(bar, parity), 1)) return true;
+#pragma unroll 1
+    for (uint32_t tries = 1; tries < kWaitTries; ++tries)
+        if (mbar_try(bar, parity)) return true;
     return false;
 }
 
