@@ -209,6 +209,9 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             fetch_index(s_aux, T, c2, other, lane);
             decode_finish<K, kSink>(cx, status, r0, L, lane, stage_bytes);
             if (r1.c == kNone) break;
+            // the ring is free now: a copy that had to wait for it starts here, a turn's worth of
+            // bookkeeping before its bytes are asked for (its offset is still in the chunk's slot)
+            if (r1.kind() == kStaged && !r1.issued()) issue_copy(cx, T, r1, (lds64(sp + 64u) >> 3) & ~15ull, lane, stage_bytes);
             r0 = r1;
             sp = other;
         }
