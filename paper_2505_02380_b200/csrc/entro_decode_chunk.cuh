@@ -351,7 +351,9 @@ struct OutCursor {
 // Plain decode: the 8 values of this lane's next group go to the output tensor.  A lane's
 // consecutive groups are 32 groups apart, so one call per lane writes 512 contiguous bytes.
 struct EmitStore {
+    static constexpr bool kTwice = true;    // a group may be written, found wrong, and written again
     OutCursor out;
+    __device__ __forceinline__ void back(uint32_t groups) { out.off -= groups * 16u * kSubBlocks; }
     __device__ __forceinline__ bool more() const { return out.more(); }
     __device__ __forceinline__ void operator()(uint4 v)
     {
@@ -364,6 +366,7 @@ struct EmitStore {
 // Integer output (the form the paper's decoder produces): the tables hold the symbols
 // themselves in their 16-bit value fields; a group of 8 leaves as 8 bytes ...
 struct EmitBytes {
+    static constexpr bool kTwice = false;
     OutCursor out;
     __device__ __forceinline__ bool more() const { return out.more(); }
     __device__ __forceinline__ void operator()(uint4 v)
@@ -375,6 +378,7 @@ struct EmitBytes {
 
 // ... or, for 4-bit symbols, as 4 bytes of two nibbles each, the earlier symbol low.
 struct EmitNibbles {
+    static constexpr bool kTwice = false;
     OutCursor out;
     __device__ __forceinline__ bool more() const { return out.more(); }
     __device__ __forceinline__ void operator()(uint4 v)
@@ -395,6 +399,7 @@ struct EmitNibbles {
 // parts of gets the sums added to its fp32 accumulators, and the last chunk to do so rounds.
 template <int B>
 struct EmitDot {
+    static constexpr bool kTwice = false;   // its values are added up: nothing wrong may pass
     uint32_t xaddr;       // shared-window address of x[0][col .. col + 8) for this lane's next group
     uint32_t xlane;       // the same at the start of a row
     uint32_t xstride;     // bytes from one token's x to the next
@@ -528,6 +533,52 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
     return cur_bit_addr(r);
 }
 
+// 8-bit alphabets whose groups of four almost never fail, turns per chunk that come in N's,
+// values that are stored: 8 N symbols, 2 N groups of four, under one check.  Each eight leave
+// as soon as they are decoded (their registers are free for the next eight); if any of the
+// groups failed, all are done again one group at a time and written again.
+template <int K, int N, class Emit>
+__device__ __forceinline__ uint32_t rows_multi(uint32_t start, uint32_t* status, LutKey key, Emit& emit)
+{
+    Cur r;
+    cur_init(r, start);
+    while (emit.more()) {
+        uint32_t pk[4], s[2 * N], any = 0;
+#pragma unroll
+        for (int h = 0; h < N; ++h) {
+            group4(r, key, pk[0], pk[1], s[2 * h]);
+            group4(r, key, pk[2], pk[3], s[2 * h + 1]);
+            any |= s[2 * h] | s[2 * h + 1];
+            if (h + 1 < N) emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
+        }
+        if (__builtin_expect((any & 0xffe0u) != 0u, 0)) {
+            // back over all groups: the position moved by the sum of the s, the words by one per flip of bit 5
+            uint32_t p = r.pos, steps = 0;
+#pragma unroll
+            for (int g = 2 * N - 1; g >= 0; --g) {
+                const uint32_t before = p - s[g];
+                steps += ((before ^ p) >> 5) & 1u;
+                p = before;
+            }
+            cur_init(r, (r.next - kCurBytes - 4u * steps) * 8u + (p & 31u));
+            emit.back(N - 1);
+#pragma unroll 1
+            for (int h = 0; h < N; ++h) {
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    uint32_t sg;
+                    group4(r, key, pk[2 * g], pk[2 * g + 1], sg);
+                    if (__builtin_expect((sg & 0xffe0u) != 0u, 0)) repair_quad<K>(r, status, key, sg, pk[2 * g], pk[2 * g + 1]);
+                }
+                if (h + 1 < N) emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
+            }
+        }
+        emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
+        if (ENTRO_CHECK(smem_ok(r.next, 4u))) break;      // the next word the reader would pull in
+    }
+    return cur_bit_addr(r);
+}
+
 // 4-bit alphabets: eight symbols per lookup.
 template <int K, class Emit>
 __device__ __forceinline__ uint32_t rows_oct(uint32_t start, uint32_t* status, Emit& emit)
@@ -555,7 +606,9 @@ __device__ __forceinline__ uint32_t rows_any(const DecodeAux* aux, uint32_t star
     const uint32_t mode = aux->mode;
     if (mode == 0u) return rows_oct<K>(start, status, emit);
     const LutKey key = lut_key(aux, lane);
-    if (mode == 8u) return rows_single<K, 8>(start, status, key, emit);
+    if constexpr (Emit::kTwice)
+        if (mode == 9u) return rows_multi<K, 2>(start, status, key, emit);
+    if (mode == 8u || mode == 9u) return rows_single<K, 8>(start, status, key, emit);
     if (mode == 4u) return rows_single<K, 4>(start, status, key, emit);
     if (mode == 3u) return rows_single<K, 3>(start, status, key, emit);
     if (mode == 16u) return rows_single<K, 16>(start, status, key, emit);
