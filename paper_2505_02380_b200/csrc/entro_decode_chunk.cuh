@@ -467,10 +467,11 @@ struct EmitDot {
     }
 };
 
-// 8-bit alphabets, eight symbols per turn.  G = 2, 3 (as 3 + 3 + 2), 4: groups of that many
-// lookups, each checked.  G = 8: two groups of four under one check, for streams whose groups
-// of four almost never fail; if either failed, both are done again one by one.  G = 16: all
-// eight lookups on one view (at most 2 bit per symbol), done again as two fours if it fails.
+// 8-bit alphabets, eight symbols per turn.  G = 2, 3 (as 3 + 3 + 2): groups of that many
+// lookups, each checked.  G = 8: two groups of four under one check (the modes 4, 8 and 9 of
+// the table build); if only the second failed it is repaired by itself, else both are done
+// again one by one.  G = 16: all eight lookups on one view (at most 2 bit per symbol), done
+// again as two fours if it fails.
 template <int K, int G, class Emit>
 __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status, LutKey key, Emit& emit)
 {
@@ -478,7 +479,7 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
     cur_init(r, start);
     while (emit.more()) {
         uint32_t pk[4];
-        bool again = G == 4;
+        bool again = false;
         if (G == 16) {
             uint4 v;
             uint32_t s;
@@ -494,14 +495,19 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
             group4(r, key, pk[0], pk[1], s0);
             group4(r, key, pk[2], pk[3], s1);
             if (__builtin_expect(((s0 | s1) & 0xffe0u) != 0u, 0)) {
-                // back over both: the position moved by s0 + s1, the words by one per flip of bit 5
-                const uint32_t p1 = r.pos - s1, p0 = p1 - s0;
-                const uint32_t steps = (((p0 ^ p1) >> 5) & 1u) + (((p1 ^ r.pos) >> 5) & 1u);
-                cur_init(r, (r.next - kCurBytes - 4u * steps) * 8u + (p0 & 31u));
-                again = true;
+                if ((s0 & 0xffe0u) == 0u) {
+                    // the first four stand: only the second four are repaired
+                    repair_quad<K>(r, status, key, s1, pk[2], pk[3]);
+                } else {
+                    // back over both: the position moved by s0 + s1, the words by one per flip of bit 5
+                    const uint32_t p1 = r.pos - s1, p0 = p1 - s0;
+                    const uint32_t steps = (((p0 ^ p1) >> 5) & 1u) + (((p1 ^ r.pos) >> 5) & 1u);
+                    cur_init(r, (r.next - kCurBytes - 4u * steps) * 8u + (p0 & 31u));
+                    again = true;
+                }
             }
         }
-        if (G == 4 || G == 8 || G == 16) {
+        if (G == 8 || G == 16) {
             if (again) {
 #pragma unroll
                 for (int g = 0; g < 2; ++g) {
@@ -511,14 +517,28 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
                 }
             }
         } else if (G == 3) {
-            uint32_t s, a2, b0;
-            group3<false>(r, key, pk[0], a2, s);
-            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_triple<K, false>(r, status, key, s, pk[0], a2);
-            group3<true>(r, key, b0, pk[2], s);
-            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_triple<K, true>(r, status, key, s, b0, pk[2]);
+            // 3 + 3 + 2 under one check; what failed first is repaired, what came after it is done again
+            uint32_t sa, sb, sc, a2, b0;
+            group3<false>(r, key, pk[0], a2, sa);
+            group3<true>(r, key, b0, pk[2], sb);
+            group2(r, key, pk[3], sc);
+            if (__builtin_expect(((sa | sb | sc) & 0xffe0u) != 0u, 0)) {
+                const bool fa = (sa & 0xffe0u) != 0u;
+                bool fb = (sb & 0xffe0u) != 0u;
+                if (fa | fb) {
+                    unwind_group(r, sc);
+                    if (fa) {
+                        unwind_group(r, sb);
+                        repair_triple<K, false>(r, status, key, sa, pk[0], a2);
+                        group3<true>(r, key, b0, pk[2], sb);
+                        fb = (sb & 0xffe0u) != 0u;
+                    }
+                    if (fb) repair_triple<K, true>(r, status, key, sb, b0, pk[2]);
+                    group2(r, key, pk[3], sc);
+                }
+                if ((sc & 0xffe0u) != 0u) repair_pair<K>(r, status, key, sc, pk[3]);
+            }
             pk[1] = __byte_perm(a2, b0, 0x7632);
-            group2(r, key, pk[3], s);
-            if (__builtin_expect((s & 0xffe0u) != 0u, 0)) repair_pair<K>(r, status, key, s, pk[3]);
         } else {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
@@ -608,8 +628,7 @@ __device__ __forceinline__ uint32_t rows_any(const DecodeAux* aux, uint32_t star
     const LutKey key = lut_key(aux, lane);
     if constexpr (Emit::kTwice)
         if (mode == 9u) return rows_multi<K, 2>(start, status, key, emit);
-    if (mode == 8u || mode == 9u) return rows_single<K, 8>(start, status, key, emit);
-    if (mode == 4u) return rows_single<K, 4>(start, status, key, emit);
+    if (mode == 8u || mode == 9u || mode == 4u) return rows_single<K, 8>(start, status, key, emit);
     if (mode == 3u) return rows_single<K, 3>(start, status, key, emit);
     if (mode == 16u) return rows_single<K, 16>(start, status, key, emit);
     return rows_single<K, 2>(start, status, key, emit);

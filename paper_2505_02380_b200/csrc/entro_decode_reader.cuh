@@ -344,6 +344,15 @@ __device__ __forceinline__ uint32_t rewind_group(const Cur& c, uint32_t s)
     return (c.next - kCurBytes - 4u * crossed) * 8u + (before & 31u);
 }
 
+// Takes the reader's position and word address back over a group that moved it on by s (the
+// words themselves stay as they are: whoever repairs from here opens them anew).
+__device__ __forceinline__ void unwind_group(Cur& c, uint32_t s)
+{
+    const uint32_t before = c.pos - s;
+    c.next -= 4u * (((before ^ c.pos) >> 5) & 1u);
+    c.pos = before;
+}
+
 // Repair of a group of two symbols that did not stand (kept inline: a call here would park
 // the caller's registers in local memory, which misses the small L1 left beside 228 KB of
 // shared memory): the symbols one by one, any code length, with the general reader.

@@ -252,6 +252,27 @@ def test_decode_every_group_size(sigma_levels, foreign):
     assert_status_ok()
 
 
+@pytest.mark.parametrize("sigma_levels", [1.6, 9.0, 24.0])
+def test_groups_under_one_check_are_repaired_wherever_they_fail(sigma_levels):
+    """Several groups of lookups share one check; when it fails, what failed first is repaired
+    and what came after it is done again (3 + 3 + 2 lookups, two fours), or everything is
+    written again (sixteen symbols of a narrow histogram).  A million symbols at widths near
+    the upper end of each mode's range make every position of a group fail hundreds of
+    times: groups that need 32 bits or more, and codes beyond the table's reach."""
+    chunk, n = 4096, 256 * 4096
+    rng = np.random.default_rng(int(sigma_levels * 10))
+    q = np.clip(np.rint(rng.normal(128.0, sigma_levels, n)), 0, 255).astype(np.uint8)
+    q[rng.integers(0, n, n // 400)] = rng.integers(0, 256, n // 400).astype(np.uint8)   # rare symbols, long codes
+    ln = oracle.huffman_lengths(np.bincount(q, minlength=256).tolist())
+    cd = oracle.canonical_codes(ln)
+    enc = oracle.encode(q, ln, cd, chunk)
+    out = E.entro_decode_dequant(to_dev_stream(enc.stream), to_dev_index(enc), n, chunk,
+                                 E.Codebook.from_lengths(ln.tolist(), cd.tolist()), 0.0078125, 128)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), oracle.dequant(q, 0.0078125, 128))
+    assert_status_ok()
+
+
 @pytest.mark.parametrize("chunk", [8192, 16384])
 def test_chunks_larger_than_a_warps_ring(chunk):
     """At 8 bit per symbol a chunk of 8192 or 16384 symbols does not fit the 5 KB of shared
