@@ -29,7 +29,7 @@ OK, ERR_INVALID_ARG, ERR_BUFFER_TOO_SMALL, ERR_NONFINITE, ERR_CODE_TOO_LONG, ERR
     ERR_UNSUPPORTED, ERR_TOO_MANY_TENSORS = range(9)
 STATIC_MAX_TENSORS = 8
 GEMV_MAX_BATCH = 8
-DEFAULT_DECODE_CONFIG = (12, 32, 1, 1024)   # lut_bits, warps_per_cta, ctas_per_sm, chunks_per_item
+DEFAULT_DECODE_CONFIG = (12, 32, 1, 1792)   # lut_bits, warps_per_cta, ctas_per_sm, chunks_per_item
 
 
 class EntroError(RuntimeError):

@@ -380,6 +380,10 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, ItemPlan& plan, DevTensor& 
     uint32_t per_item = (plan.graded && (plan.seen + nc) * 100 > plan.total * 88) ? plan.tail : plan.base;
     if (d.chunk_symbols > 4096u) per_item = (uint32_t)((uint64_t)per_item * 4096u / d.chunk_symbols);
     if (per_item < 32u) per_item = 32u;
+    // the tensor's items of equal size (a short last item leaves most of a CTA's warps idle),
+    // whole rounds of the 32 warps
+    const uint64_t pieces = (nc + per_item - 1) / per_item;
+    if (pieces > 1) per_item = (uint32_t)(((nc + pieces - 1) / pieces + 31u) / 32u * 32u);
     t.item_chunks = per_item;
     plan.seen += nc;
     t.raw_symbols = 0;

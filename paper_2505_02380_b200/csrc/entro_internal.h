@@ -93,7 +93,7 @@ struct DecodeConfig {
     int lut_bits = 12;
     int warps_per_cta = 32;
     int ctas_per_sm = 1;
-    int chunks_per_item = 1024;
+    int chunks_per_item = 1792;
 };
 
 // Where the decode kernel sends the decoded values.
