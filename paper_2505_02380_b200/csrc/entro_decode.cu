@@ -71,6 +71,25 @@ __device__ __forceinline__ void cta_finished(uint32_t* control)
     }
 }
 
+// Tensor of a work item: the last t with item_start[t] <= item, found by a whole warp, each
+// lane reading one of 32 evenly spaced entries per round (two dependent reads for up to 1024
+// tensors, where a binary search by one thread takes ten).  All lanes return the same t.
+__device__ __forceinline__ uint32_t tensor_of_item(const uint32_t* __restrict__ item_start, uint32_t ntensors, uint32_t item,
+                                                   uint32_t lane)
+{
+    uint32_t lo = 0, n = ntensors;
+    while (n > 1u) {
+        const uint32_t step = (n + 31u) >> 5;
+        const uint32_t at = lo + lane * step;
+        const uint32_t v = at < lo + n ? __ldg(item_start + at) : 0xffffffffu;
+        const uint32_t k = (uint32_t)__popc(__ballot_sync(0xffffffffu, v <= item));   // >= 1: item_start[lo] <= item
+        const uint32_t end = lo + n;
+        lo += (k - 1u) * step;
+        n = min(step, end - lo);
+    }
+    return lo;
+}
+
 // item_start[t] = first work item of tensor t, item_start[ntensors] = number of items; an
 // item is up to tensors[t].item_chunks consecutive chunks of one tensor.
 // kSink says where the decoded values go.  With kSinkGemv they are not stored: gemv[t]
@@ -104,7 +123,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     const uint32_t kRings = rings_at;          // rings_offset<K>(kGemv, bytes of staged x)
     const uint32_t after = kRings + warps * stage_bytes + kOverRead;          // offset in smem, a multiple of 16
     const uint32_t slots = after + warps * 16u;
-    volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(smem + slots + warps * 2u * kSlotBytes);   // [2]
+    volatile uint32_t* s_item = reinterpret_cast<volatile uint32_t*>(smem + slots + warps * 2u * kSlotBytes);   // [4]
     uint32_t* status = control + 1;
 
     WarpCtx cx;
@@ -120,27 +139,39 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
+    // s_item[slot] = the item's number within its tensor, s_item[2 + slot] = the tensor, or kNone
+    // when the items have run out.  Warp 0 puts the next item on record, tensor included, before
+    // the barrier that ends the current one, so nobody reads global memory behind that barrier
+    // to find out where to go on.
     const uint32_t total_items = item_start[ntensors];
-    if (threadIdx.x == 0) {
-        s_item[0] = atomicAdd(control, 1u);
+    auto put_on_record = [&](uint32_t item, uint32_t where) {      // warp 0, all lanes, the same item
+        uint32_t t = kNone, rel = 0;
+        if (item < total_items) {
+            t = tensor_of_item(item_start, (uint32_t)ntensors, item, lane);
+            rel = item - __ldg(item_start + t);
+        }
+        if (lane == 0) {
+            s_item[where] = rel;
+            s_item[2u + where] = t;
+        }
+    };
+    if (warp == 0) {
+        uint32_t item0 = 0;
+        if (lane == 0) item0 = atomicAdd(control, 1u);
+        put_on_record(__shfl_sync(0xffffffffu, item0, 0), 0u);
     }
     __syncthreads();
     int cur = -1;
     uint32_t slot = 0;
     while (true) {
-        const uint32_t item = s_item[slot];
-        if (item >= total_items) break;
+        const uint32_t item_tensor = s_item[2u + slot];
+        if (item_tensor == kNone) break;
+        const uint32_t item_rel = s_item[slot];
         // claim the next item early; the answer of the global counter is not waited for here
         // but put on record when this item is done, before the barrier that ends it
         uint32_t next_item = 0;
         if (threadIdx.x == 0) next_item = atomicAdd(control, 1u);
-        // tensor of this item: last t with item_start[t] <= item
-        int lo = 0, hi = ntensors - 1;
-        while (lo < hi) {
-            int mid = (lo + hi + 1) >> 1;
-            if (__ldg(item_start + mid) <= item) lo = mid;
-            else hi = mid - 1;
-        }
+        const int lo = (int)item_tensor;
         if (lo != cur) {
             cur = lo;
             const TensorTables* tt = tables + cur;
@@ -177,7 +208,7 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             __syncthreads();
         }
         const DevTensor& T = *s_tensor;
-        const uint32_t first = (item - __ldg(item_start + cur)) * T.item_chunks;
+        const uint32_t first = item_rel * T.item_chunks;
         const uint32_t count = min(T.item_chunks, T.n_chunks - first);   // chunks of this item
 
         // The warps deal out the item's chunks among themselves, warp w taking chunks w, w + warps,
@@ -216,10 +247,8 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
             sp = other;
         }
         asm volatile("cp.async.wait_all;" ::: "memory");
-        if (threadIdx.x == 0) {
-            s_item[slot ^ 1u] = next_item;
-        }
-        __syncthreads();   // tables may be replaced; s_item[slot ^ 1] is now visible
+        if (warp == 0) put_on_record(__shfl_sync(0xffffffffu, next_item, 0), slot ^ 1u);
+        __syncthreads();   // tables may be replaced; the next item's record is now visible
         slot ^= 1u;
     }
     // A warp that gave up on a bulk copy lets it land (bounded) before its buffer goes away.

@@ -366,8 +366,9 @@ struct EmitStore {
 // Integer output (the form the paper's decoder produces): the tables hold the symbols
 // themselves in their 16-bit value fields; a group of 8 leaves as 8 bytes ...
 struct EmitBytes {
-    static constexpr bool kTwice = false;
+    static constexpr bool kTwice = true;
     OutCursor out;
+    __device__ __forceinline__ void back(uint32_t groups) { out.off -= groups * 8u * kSubBlocks; }
     __device__ __forceinline__ bool more() const { return out.more(); }
     __device__ __forceinline__ void operator()(uint4 v)
     {
