@@ -42,17 +42,47 @@ namespace {
 
 // ------------------------------------------------------------------ persistent kernel
 
+// n 16-byte words from global to shared memory by the whole CTA, four reads in flight per
+// thread before the first store (one round trip to L2 per four words instead of one per word).
+__device__ __forceinline__ void copy_in(uint4* dst, const uint4* __restrict__ src, uint32_t n)
+{
+    for (uint32_t base = threadIdx.x; base < n; base += 4u * blockDim.x) {
+        uint4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t i = base + (uint32_t)k * blockDim.x;
+            v[k] = i < n ? __ldg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t i = base + (uint32_t)k * blockDim.x;
+            if (i < n) dst[i] = v[k];
+        }
+    }
+}
+
 // The exponent-indexed table of a tensor into the first 64 KB of shared memory: cell-major
 // copies, word w holds cell w / copies.
-__device__ __forceinline__ void load_exp_table(const TensorTables* tt)
+__device__ __forceinline__ void load_exp_table(const TensorTables* tt, uint32_t expm)
 {
-    const uint32_t shift = 9u - __ldg(&tt->aux.expm);       // log2 of the number of copies
+    const uint32_t shift = 9u - expm;                        // log2 of the number of copies
     if (shift >= 2u) {
-        // four or more copies: the four words of a 16-byte store belong to one cell
+        // four or more copies: the four words of a 16-byte store belong to one cell.  Four reads
+        // are in flight per thread before the first store (one round trip to L2 instead of four).
         uint4* s4 = reinterpret_cast<uint4*>(smem);
-        for (uint32_t q = threadIdx.x; q < (uint32_t)kExpEntriesMax / 4u; q += blockDim.x) {
-            const uint32_t v = __ldg(tt->exp_lut() + ((4u * q) >> shift));
-            s4[q] = make_uint4(v, v, v, v);
+        constexpr uint32_t kQuads = (uint32_t)kExpEntriesMax / 4u;
+        for (uint32_t base = threadIdx.x; base < kQuads; base += 4u * blockDim.x) {
+            uint32_t v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t q = base + (uint32_t)k * blockDim.x;
+                v[k] = q < kQuads ? __ldg(tt->exp_lut() + ((4u * q) >> shift)) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t q = base + (uint32_t)k * blockDim.x;
+                if (q < kQuads) s4[q] = make_uint4(v[k], v[k], v[k], v[k]);
+            }
         }
     } else {
         uint32_t* s1 = reinterpret_cast<uint32_t*>(smem);
@@ -175,6 +205,8 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
         if (lo != cur) {
             cur = lo;
             const TensorTables* tt = tables + cur;
+            // (both flags are read at once and first: the table's reads start one round trip after the switch)
+            const uint32_t is_oct = __ldg(&tt->aux.oct), expm = __ldg(&tt->aux.expm);
             const uint4* ga = reinterpret_cast<const uint4*>(&tt->aux);
             uint4* sa = reinterpret_cast<uint4*>(s_aux);
             for (uint32_t i = threadIdx.x; i < sizeof(DecodeAux) / 16; i += blockDim.x) sa[i] = __ldg(ga + i);
@@ -193,17 +225,15 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                 for (uint32_t i = threadIdx.x; i < want; i += blockDim.x)
                     sx[i] = i < have ? __ldg(gx + i) : make_uint4(0u, 0u, 0u, 0u);
             }
-            if (__ldg(&tt->aux.oct)) {
-                const uint4* g1 = tt->oct_val;
-                uint4* s1 = reinterpret_cast<uint4*>(smem);
-                for (uint32_t i = threadIdx.x; i < (1u << K); i += blockDim.x) s1[i] = __ldg(g1 + i);
+            if (is_oct) {
+                copy_in(reinterpret_cast<uint4*>(smem), tt->oct_val, 1u << K);
                 const uint4* g2 = reinterpret_cast<const uint4*>(tt->oct_len);
                 uint4* s2 = reinterpret_cast<uint4*>(smem + (16u << K));
                 for (uint32_t i = threadIdx.x; i < (1u << K) / 16; i += blockDim.x) s2[i] = __ldg(g2 + i);
                 uint32_t* s3 = reinterpret_cast<uint32_t*>(smem + (17u << K));
                 for (uint32_t i = threadIdx.x; i < (uint32_t)kExpEntriesMin; i += blockDim.x) s3[i] = __ldg(tt->exp_small + i);
             } else {
-                load_exp_table(tt);
+                load_exp_table(tt, expm);
             }
             __syncthreads();
         }
@@ -379,7 +409,7 @@ ItemPlan plan_items(const DecodeConfig& cfg, const entro_tensor_desc* descs, int
             ++live;
         }
     const uint64_t ctas = (uint64_t)sm_count * cfg.ctas_per_sm;
-    uint64_t want = (p.total + ctas * 4 - 1) / (ctas * 4);
+    uint64_t want = (p.total + ctas * 5 - 1) / (ctas * 5);
     want = (want + cfg.warps_per_cta - 1) / cfg.warps_per_cta * cfg.warps_per_cta;
     if (want < (uint64_t)cfg.warps_per_cta) want = cfg.warps_per_cta;
     p.base = want < (uint64_t)cfg.chunks_per_item ? (uint32_t)want : (uint32_t)cfg.chunks_per_item;
