@@ -558,7 +558,9 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
 // values that are stored: 8 N symbols, 2 N groups of four, under one check.  Each eight leave
 // as soon as they are decoded (their registers are free for the next eight); if any of the
 // groups failed, all are done again one group at a time and written again.
-template <int K, int N, class Emit>
+// kWide: every eight are one group of eight lookups on one view (streams of at most 2 bit per
+// symbol) instead of two groups of four; a failure is repaired in fours all the same.
+template <int K, int N, bool kWide, class Emit>
 __device__ __forceinline__ uint32_t rows_multi(uint32_t start, uint32_t* status, LutKey key, Emit& emit)
 {
     Cur r;
@@ -567,8 +569,15 @@ __device__ __forceinline__ uint32_t rows_multi(uint32_t start, uint32_t* status,
         uint32_t pk[4], s[2 * N], any = 0;
 #pragma unroll
         for (int h = 0; h < N; ++h) {
-            group4(r, key, pk[0], pk[1], s[2 * h]);
-            group4(r, key, pk[2], pk[3], s[2 * h + 1]);
+            if (kWide) {
+                uint4 v;
+                group8(r, key, v, s[2 * h]);
+                pk[0] = v.x, pk[1] = v.y, pk[2] = v.z, pk[3] = v.w;
+                s[2 * h + 1] = 0u;
+            } else {
+                group4(r, key, pk[0], pk[1], s[2 * h]);
+                group4(r, key, pk[2], pk[3], s[2 * h + 1]);
+            }
             any |= s[2 * h] | s[2 * h + 1];
             if (h + 1 < N) emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
         }
@@ -627,11 +636,14 @@ __device__ __forceinline__ uint32_t rows_any(const DecodeAux* aux, uint32_t star
     const uint32_t mode = aux->mode;
     if (mode == 0u) return rows_oct<K>(start, status, emit);
     const LutKey key = lut_key(aux, lane);
-    if constexpr (Emit::kTwice)
-        if (mode == 9u) return rows_multi<K, 2>(start, status, key, emit);
+    if constexpr (Emit::kTwice) {
+        if (mode == 9u) return rows_multi<K, 2, false>(start, status, key, emit);
+        if (mode == 17u) return rows_multi<K, 2, true>(start, status, key, emit);
+        if (mode == 18u) return rows_multi<K, 4, true>(start, status, key, emit);
+    }
     if (mode == 8u || mode == 9u || mode == 4u) return rows_single<K, 8>(start, status, key, emit);
     if (mode == 3u) return rows_single<K, 3>(start, status, key, emit);
-    if (mode == 16u) return rows_single<K, 16>(start, status, key, emit);
+    if (mode == 16u || mode == 17u || mode == 18u) return rows_single<K, 16>(start, status, key, emit);
     return rows_single<K, 2>(start, status, key, emit);
 }
 

@@ -161,8 +161,10 @@ __global__ void __launch_bounds__(256) build_tables_kernel(const DevTensor* __re
         aux.key_mask = ((32u << m) - 1u) << (11u - m);
         aux.key_lane_mask = (32u >> (m - 4u)) - 1u;
         aux.turns = (T.chunk_symbols % (8u * kSubBlocks)) == 0u ? T.chunk_symbols / (8u * kSubBlocks) : 0u;
-        // (9: groups as in 8, and the turns per chunk come in pairs)
-        aux.mode = aux.oct ? 0u : (aux.group == 8u && aux.turns != 0u && aux.turns % 2u == 0u) ? 9u : aux.group;
+        // (9 and 17: groups as in 8 and 16, and the turns per chunk come in pairs; 18: as 16, in fours)
+        const bool pairs = aux.turns != 0u && aux.turns % 2u == 0u;
+        aux.mode = aux.oct ? 0u : (pairs && (aux.group == 8u || aux.group == 16u)) ? aux.group + 1u : aux.group;
+        if (aux.mode == 17u && aux.turns % 4u == 0u) aux.mode = 18u;
     }
     if (tid < 20)
         aux.index_src[tid] = tid < 16 ? reinterpret_cast<unsigned long long>(T.sub_len) + 4ull * tid

@@ -69,7 +69,7 @@ struct DecodeAux {
     uint32_t key_mask;       // the bits of (float bits >> 12) that select a cell of the exponent-indexed table
     uint32_t key_lane_mask;  // lanes that share a copy of that table: copy = lane & this
     uint32_t turns;          // groups of 8 symbols per lane and full chunk (chunk_symbols / 256), 0 if chunks cannot be staged
-    uint32_t mode;           // what the decode loop switches on: 0 = eight symbols per lookup, 9 = group 8 with an even number of turns per chunk, else `group`
+    uint32_t mode;           // what the decode loop switches on: 0 = eight symbols per lookup, 9 / 17 = group 8 / 16 with an even number of turns per chunk, 18 = group 16 with turns in fours, else `group`
     unsigned long long index_src[20];   // lane l's 4 bytes of chunk 0's index entries: lanes 0..15 two sub-block lengths
                                         // each, lanes 16..19 the halves of offsets[c], offsets[c + 1]
 };

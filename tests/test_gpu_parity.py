@@ -252,11 +252,11 @@ def test_decode_every_group_size(sigma_levels, foreign):
     assert_status_ok()
 
 
-@pytest.mark.parametrize("sigma_levels", [1.6, 9.0, 24.0])
+@pytest.mark.parametrize("sigma_levels", [0.45, 1.6, 9.0, 24.0])
 def test_groups_under_one_check_are_repaired_wherever_they_fail(sigma_levels):
     """Several groups of lookups share one check; when it fails, what failed first is repaired
     and what came after it is done again (3 + 3 + 2 lookups, two fours), or everything is
-    written again (sixteen symbols of a narrow histogram).  A million symbols at widths near
+    written again (sixteen or thirty-two symbols of a narrow histogram).  A million symbols at widths near
     the upper end of each mode's range make every position of a group fail hundreds of
     times: groups that need 32 bits or more, and codes beyond the table's reach."""
     chunk, n = 4096, 256 * 4096
