@@ -134,7 +134,8 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
                                                          const TensorTables* __restrict__ tables,
                                                          uint32_t stage_bytes,
                                                          uint32_t* __restrict__ control,
-                                                         const GemvTensor* __restrict__ gemv, uint32_t rings_at)
+                                                         const GemvTensor* __restrict__ gemv, uint32_t rings_at,
+                                                         uint32_t striped)
 {
     constexpr int kBatch = kGemvBatchOf<kSink>;
     constexpr bool kGemv = kBatch > 0;
@@ -174,8 +175,15 @@ __global__ void __launch_bounds__(1024, 1) decode_kernel(const DevTensor* __rest
     // the barrier that ends the current one, so nobody reads global memory behind that barrier
     // to find out where to go on.
     const uint32_t total_items = item_start[ntensors];
+    // The first `striped` items (a multiple of the grid size, all of full size) are claimed in
+    // an order that hands a CTA consecutive items of the list, hence mostly of one tensor, as long
+    // as the CTAs keep pace: claim i is item (i mod grid) * rows + i / grid.  The table is then
+    // reloaded a few times per CTA instead of once per item.  The graded items at the end keep
+    // their order, so the CTAs still finish together.
+    const uint32_t stripe_rows = striped / gridDim.x;
     auto put_on_record = [&](uint32_t item, uint32_t where) {      // warp 0, all lanes, the same item
         uint32_t t = kNone, rel = 0;
+        if (item < striped) item = (item % gridDim.x) * stripe_rows + item / gridDim.x;
         if (item < total_items) {
             t = tensor_of_item(item_start, (uint32_t)ntensors, item, lane);
             rel = item - __ldg(item_start + t);
@@ -330,7 +338,8 @@ entro_status launch_decode(Workspace* ws, const DecodeConfig& cfg, const DevTens
     const bool timed = ws->prof_used < ws->prof_cap;
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_start[ws->prof_used], s));
     decode_kernel<K, kSink><<<grid, cfg.warps_per_cta * 32, sh.smem, s>>>(
-        tensors, ntensors, item_start, tables, sh.stage_bytes, ws->control, gemv, rings_offset<K>(kGemv, x_bytes));
+        tensors, ntensors, item_start, tables, sh.stage_bytes, ws->control, gemv, rings_offset<K>(kGemv, x_bytes),
+        ws->big_items / grid * grid);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
     if (timed) ENTRO_CUDA(cudaEventRecord(ws->prof_stop[ws->prof_used++], s));
@@ -397,6 +406,9 @@ struct ItemPlan {
     uint64_t seen = 0;         // chunks of the tensors planned so far
     uint32_t base = 0, tail = 0;
     bool graded = false;
+    uint64_t items = 0;        // work items of the tensors planned so far
+    uint64_t big_items = 0;    // of those, the ones before the first tensor with graded (small) items
+    bool tail_seen = false;
 };
 
 ItemPlan plan_items(const DecodeConfig& cfg, const entro_tensor_desc* descs, int ntensors, int sm_count)
@@ -449,7 +461,12 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, ItemPlan& plan, DevTensor& 
     t.full_chunks = (uint32_t)(d.n / d.chunk_symbols);
     t.pad[0] = t.pad[1] = 0;
     for (int j = 0; j < ENTRO_MAX_SYMBOLS; ++j) t.len[j] = j < d.cb.nsym ? d.cb.len[j] : 0;
-    return (nc + t.item_chunks - 1) / t.item_chunks;
+    const uint64_t n_items = (nc + t.item_chunks - 1) / t.item_chunks;
+    const bool small = plan.graded && (plan.seen * 100 > plan.total * 88);     // (seen already includes this tensor)
+    plan.items += n_items;
+    if (small) plan.tail_seen = true;
+    if (!plan.tail_seen) plan.big_items = plan.items;
+    return n_items;
 }
 
 }  // namespace
@@ -542,7 +559,17 @@ entro_status decode_batched_locked(Workspace* ws, const entro_tensor_desc* descs
     build_tables_kernel<<<dim3((unsigned)live, table_slices(live, ws->sm_count)), 256, 0, s>>>(dt, cfg.lut_bits, dtables, ws->control, nullptr);
     count_launch();
     ENTRO_CUDA(cudaGetLastError());
+    // Striped claims pay where decoding is bound by instructions (8-bit alphabets: fewer table
+    // reloads); a launch of 4-bit alphabets runs near the HBM peak and loses by them (148 places
+    // written at once instead of neighbouring ones: 2.50 against 2.465 ms on the mistral-shaped model).
+    uint64_t wide_symbols = 0, all_symbols = 0;
+    for (int i = 0; i < ntensors; ++i) {
+        all_symbols += descs[i].n;
+        if (descs[i].cb.nsym > 16) wide_symbols += descs[i].n;
+    }
+    ws->big_items = (plan.graded && !few && wide_symbols * 2 > all_symbols) ? (uint32_t)plan.big_items : 0u;
     const entro_status st = launch_decode_any(ws, cfg, dt, live, ditems, (uint32_t)items, dtables, s, nullptr, sink);
+    ws->big_items = 0;
     if (few && st == ENTRO_OK) {
         ws->kept = true;
         ws->kept_ntensors = ntensors;

@@ -133,6 +133,7 @@ struct Workspace {
     // call finds descriptors and tables already in place and is one launch.  reserve_device
     // (every call that fills the area goes through it) forgets it.
     static constexpr int kKeptTensors = ENTRO_STATIC_MAX_TENSORS;
+    uint32_t big_items = 0;    // set around a launch: its first so many work items are the full-size ones (0: none to stripe)
     bool kept = false;
     int kept_ntensors = 0, kept_live = 0, kept_sink = 0;
     uint32_t kept_items = 0;
