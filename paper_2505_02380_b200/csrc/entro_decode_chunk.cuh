@@ -557,7 +557,8 @@ __device__ __forceinline__ uint32_t rows_single(uint32_t start, uint32_t* status
 // 8-bit alphabets whose groups of four almost never fail, turns per chunk that come in N's,
 // values that are stored: 8 N symbols, 2 N groups of four, under one check.  Each eight leave
 // as soon as they are decoded (their registers are free for the next eight); if any of the
-// groups failed, all are done again one group at a time and written again.
+// groups failed, the eights from the first one with a failed group onwards are done again one
+// group at a time and written again.
 // kWide: every eight are one group of eight lookups on one view (streams of at most 2 bit per
 // symbol) instead of two groups of four; a failure is repaired in fours all the same.
 template <int K, int N, bool kWide, class Emit>
@@ -582,18 +583,25 @@ __device__ __forceinline__ uint32_t rows_multi(uint32_t start, uint32_t* status,
             if (h + 1 < N) emit(make_uint4(pk[0], pk[1], pk[2], pk[3]));
         }
         if (__builtin_expect((any & 0xffe0u) != 0u, 0)) {
-            // back over all groups: the position moved by the sum of the s, the words by one per flip of bit 5
+            // the eights before the first one with a failed group stand; back over the groups from there
+            // on: the position moved by the sum of their s, the words by one per flip of bit 5
+            int h0 = 0;
+#pragma unroll
+            for (int h = N - 1; h >= 0; --h)
+                if (((s[2 * h] | s[2 * h + 1]) & 0xffe0u) != 0u) h0 = h;
             uint32_t p = r.pos, steps = 0;
 #pragma unroll
             for (int g = 2 * N - 1; g >= 0; --g) {
-                const uint32_t before = p - s[g];
-                steps += ((before ^ p) >> 5) & 1u;
-                p = before;
+                if (g >= 2 * h0) {
+                    const uint32_t before = p - s[g];
+                    steps += ((before ^ p) >> 5) & 1u;
+                    p = before;
+                }
             }
             cur_init(r, (r.next - kCurBytes - 4u * steps) * 8u + (p & 31u));
-            emit.back(N - 1);
+            emit.back((uint32_t)(N - 1 - h0));
 #pragma unroll 1
-            for (int h = 0; h < N; ++h) {
+            for (int h = h0; h < N; ++h) {
 #pragma unroll
                 for (int g = 0; g < 2; ++g) {
                     uint32_t sg;
