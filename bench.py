@@ -39,7 +39,7 @@ NOMINAL_HBM_GBS = 8000.0
 # ncu capture on the 1-layer truncation, 480,260,096 weights; traffic grows in proportion to the
 # weights, so a full launch is this figure times its weights).  See profiles/.  Set an entry to
 # None when the kernel changes until the counters have been taken again.
-NCU_DRAM_BYTES_PER_WEIGHT = {8: 1100.29e6 / 480260096, 4: 967.09e6 / 480260096}
+NCU_DRAM_BYTES_PER_WEIGHT = {8: 1102.38e6 / 480260096, 4: 966.16e6 / 480260096}
 FALLBACK_HBM_GBS = 6650.0
 
 
