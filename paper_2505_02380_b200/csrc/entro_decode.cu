@@ -404,7 +404,7 @@ entro_status validate_desc(const entro_tensor_desc& d, bool need_out = true)
 struct ItemPlan {
     uint64_t total = 0;        // chunks in the launch
     uint64_t seen = 0;         // chunks of the tensors planned so far
-    uint32_t base = 0, tail = 0;
+    uint32_t base = 0, tail = 0, unit = 32;
     bool graded = false;
     uint64_t items = 0;        // work items of the tensors planned so far
     uint64_t big_items = 0;    // of those, the ones before the first tensor with graded (small) items
@@ -422,8 +422,12 @@ ItemPlan plan_items(const DecodeConfig& cfg, const entro_tensor_desc* descs, int
         }
     const uint64_t ctas = (uint64_t)sm_count * cfg.ctas_per_sm;
     uint64_t want = (p.total + ctas * 5 - 1) / (ctas * 5);
-    want = (want + cfg.warps_per_cta - 1) / cfg.warps_per_cta * cfg.warps_per_cta;
-    if (want < (uint64_t)cfg.warps_per_cta) want = cfg.warps_per_cta;
+    p.unit = (uint32_t)cfg.warps_per_cta;
+    // fewer chunks than warps on the GPU: items of two chunks, so that the launch spreads over as
+    // many SMs as it can (a lone warp decodes a chunk several times faster than one of 32 on an SM)
+    if (p.total < ctas * (uint64_t)cfg.warps_per_cta) p.unit = 2;
+    want = (want + p.unit - 1) / p.unit * p.unit;
+    if (want < (uint64_t)p.unit) want = p.unit;
     p.base = want < (uint64_t)cfg.chunks_per_item ? (uint32_t)want : (uint32_t)cfg.chunks_per_item;
     p.tail = p.base / 8 < (uint32_t)cfg.warps_per_cta ? (uint32_t)cfg.warps_per_cta : p.base / 8;
     p.graded = live >= 8 && p.base >= 8u * (uint32_t)cfg.warps_per_cta;   // a tail item still gives every warp a chunk
@@ -450,11 +454,11 @@ uint64_t fill_dev_tensor(const entro_tensor_desc& d, ItemPlan& plan, DevTensor& 
     // 4096-symbol chunks and scale down for larger ones, so that an item is as much work
     uint32_t per_item = (plan.graded && (plan.seen + nc) * 100 > plan.total * 88) ? plan.tail : plan.base;
     if (d.chunk_symbols > 4096u) per_item = (uint32_t)((uint64_t)per_item * 4096u / d.chunk_symbols);
-    if (per_item < 32u) per_item = 32u;
+    if (per_item < plan.unit) per_item = plan.unit;
     // the tensor's items of equal size (a short last item leaves most of a CTA's warps idle),
     // whole rounds of the 32 warps
     const uint64_t pieces = (nc + per_item - 1) / per_item;
-    if (pieces > 1) per_item = (uint32_t)(((nc + pieces - 1) / pieces + 31u) / 32u * 32u);
+    if (pieces > 1) per_item = (uint32_t)(((nc + pieces - 1) / pieces + plan.unit - 1u) / plan.unit * plan.unit);
     t.item_chunks = per_item;
     plan.seen += nc;
     t.raw_symbols = 0;
